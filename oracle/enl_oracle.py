@@ -1,0 +1,188 @@
+"""Python front end of the float64 CPU oracle (``enl_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: imported by the tests, by the smoke check and by the benchmark's
+CPU-baseline leg.  The product package never imports this module, and this module never
+imports the product package.
+
+The oracle keeps its own group container (a dict of plain arrays, no pages): one entry per
+(group id, layer), rows in stored order; an append concatenates at the end (paper, Sec. 3.2:
+new objects are concatenated at the end of their group, existing K/V is untouched).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import Dict, List, Optional, Sequence, Tuple
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "enl_oracle.c")
+_LIB = os.path.join(_HERE, "libenl_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle with gcc (OpenMP, -O2, no fast-math) into ``libenl_oracle.so``."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c99", "-o", _LIB, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        lib = ctypes.CDLL(_LIB)
+        lib.enl_oracle_threads.restype = ctypes.c_int
+        lib.enl_oracle_sel_off.restype = None
+        lib.enl_oracle_attend.restype = ctypes.c_int
+        _lib = lib
+    return _lib
+
+
+def threads() -> int:
+    """Number of OpenMP threads the oracle will use."""
+    return int(_load().enl_oracle_threads())
+
+
+def _bits(x) -> np.ndarray:
+    """bf16 tensor / uint16 array -> contiguous uint16 bit patterns (exact, no rounding)."""
+    if isinstance(x, np.ndarray):
+        if x.dtype != np.uint16:
+            raise TypeError("numpy inputs must already be uint16 bf16 bit patterns")
+        return np.ascontiguousarray(x)
+    import torch  # local: only tensors need it
+
+    if x.dtype != torch.bfloat16:
+        raise TypeError("tensor inputs must be bfloat16")
+    return np.ascontiguousarray(x.detach().cpu().contiguous().view(torch.int16).numpy().view(np.uint16))
+
+
+def sel_off(sel_len: Sequence[int]) -> np.ndarray:
+    """Exclusive prefix sum of the selected groups' lengths, length n_sel + 1 (int64)."""
+    n = len(sel_len)
+    a = np.ascontiguousarray(np.asarray(sel_len, dtype=np.int32))
+    out = np.zeros(n + 1, dtype=np.int64)
+    _load().enl_oracle_sel_off(
+        ctypes.c_int(n), a.ctypes.data_as(ctypes.c_void_p), out.ctypes.data_as(ctypes.c_void_p)
+    )
+    return out
+
+
+def attend_slots(
+    n_q_heads: int,
+    n_kv_heads: int,
+    head_dim: int,
+    slots_k: Sequence,
+    slots_v: Sequence,
+    q,
+    k_new,
+    v_new,
+    rows: Optional[Sequence[int]] = None,
+    want_mass: bool = True,
+) -> Tuple[np.ndarray, Optional[np.ndarray]]:
+    """Attention of one episode over explicit slot arrays.
+
+    ``slots_k[s]`` / ``slots_v[s]``: ``[len_s, Hkv, D]`` bf16; ``q``: ``[n_q, Hq, D]``;
+    ``k_new`` / ``v_new``: ``[n_new, Hkv, D]``.  Returns ``(out [n_rows, Hq, D] f64,
+    mass [n_rows, Hq, n_sel + 1] f64)``; ``rows`` picks query rows (default: all).
+    """
+    lib = _load()
+    n_sel = len(slots_k)
+    kb = [_bits(k) for k in slots_k]
+    vb = [_bits(v) for v in slots_v]
+    lens = np.asarray([k.shape[0] if k.ndim == 3 else 0 for k in kb], dtype=np.int32)
+    for k, v in zip(kb, vb):
+        assert k.shape == v.shape
+        assert k.shape[0] == 0 or k.shape[1:] == (n_kv_heads, head_dim)
+    qb, knb, vnb = _bits(q), _bits(k_new), _bits(v_new)
+    n_q, n_new = qb.shape[0], knb.shape[0]
+    assert qb.shape[1:] == (n_q_heads, head_dim)
+    assert knb.shape == vnb.shape and (n_new == 0 or knb.shape[1:] == (n_kv_heads, head_dim))
+    if rows is None:
+        rows_a = np.arange(n_q, dtype=np.int32)
+    else:
+        rows_a = np.ascontiguousarray(np.asarray(rows, dtype=np.int32))
+    n_rows = int(rows_a.shape[0])
+    out = np.zeros((n_rows, n_q_heads, head_dim), dtype=np.float64)
+    mass = np.zeros((n_rows, n_q_heads, n_sel + 1), dtype=np.float64) if want_mass else None
+    PtrArr = ctypes.c_void_p * max(n_sel, 1)
+    kp = PtrArr(*[k.ctypes.data for k in kb]) if n_sel else PtrArr()
+    vp = PtrArr(*[v.ctypes.data for v in vb]) if n_sel else PtrArr()
+    rc = lib.enl_oracle_attend(
+        ctypes.c_int(n_q_heads), ctypes.c_int(n_kv_heads), ctypes.c_int(head_dim),
+        ctypes.c_int(n_sel), lens.ctypes.data_as(ctypes.c_void_p), kp, vp,
+        ctypes.c_int(n_q), ctypes.c_int(n_new),
+        qb.ctypes.data_as(ctypes.c_void_p), knb.ctypes.data_as(ctypes.c_void_p),
+        vnb.ctypes.data_as(ctypes.c_void_p),
+        ctypes.c_int(n_rows), rows_a.ctypes.data_as(ctypes.c_void_p),
+        out.ctypes.data_as(ctypes.c_void_p),
+        mass.ctypes.data_as(ctypes.c_void_p) if mass is not None else None,
+    )
+    if rc != 0:
+        raise ValueError("enl_oracle_attend rejected its arguments")
+    return out, mass
+
+
+class OracleCache:
+    """The oracle's own group store: ``(group, layer) -> (K bits, V bits)``, no pages."""
+
+    def __init__(self, n_layers: int, n_q_heads: int, n_kv_heads: int, head_dim: int):
+        self.n_layers, self.n_q_heads = n_layers, n_q_heads
+        self.n_kv_heads, self.head_dim = n_kv_heads, head_dim
+        self._g: Dict[Tuple[int, int], Tuple[np.ndarray, np.ndarray]] = {}
+
+    def group_store(self, group_id: int, layer: int, k, v, append: bool = False) -> None:
+        kb, vb = _bits(k), _bits(v)
+        kb = kb.reshape(-1, self.n_kv_heads, self.head_dim)
+        vb = vb.reshape(-1, self.n_kv_heads, self.head_dim)
+        key = (int(group_id), int(layer))
+        if append and key in self._g:
+            k0, v0 = self._g[key]
+            kb, vb = np.concatenate([k0, kb], axis=0), np.concatenate([v0, vb], axis=0)
+        self._g[key] = (kb, vb)
+
+    def group_len(self, group_id: int, layer: int) -> int:
+        return int(self._g[(int(group_id), int(layer))][0].shape[0])
+
+    def attend(
+        self,
+        layer: int,
+        sel_ids: Sequence[int],
+        q,
+        k_new,
+        v_new,
+        rows: Optional[Sequence[int]] = None,
+        want_mass: bool = True,
+    ):
+        """One episode.  Returns ``(out, mass, sel_off)``; slots follow ``sel_ids`` order."""
+        ks = [self._g[(int(g), int(layer))][0] for g in sel_ids]
+        vs = [self._g[(int(g), int(layer))][1] for g in sel_ids]
+        out, mass = attend_slots(self.n_q_heads, self.n_kv_heads, self.head_dim, ks, vs,
+                                 q, k_new, v_new, rows=rows, want_mass=want_mass)
+        return out, mass, sel_off([k.shape[0] for k in ks])
+
+    def attend_batch(
+        self,
+        layer: int,
+        sel_ids: Sequence[int],
+        cu_sel: Sequence[int],
+        cu_q: Sequence[int],
+        cu_new: Sequence[int],
+        q,
+        k_new,
+        v_new,
+        rows_per_episode: Optional[List[Optional[Sequence[int]]]] = None,
+    ):
+        """Varlen batch of independent episodes: a plain loop over ``attend``."""
+        res = []
+        for b in range(len(cu_q) - 1):
+            ids = list(sel_ids[cu_sel[b]:cu_sel[b + 1]])
+            rows = rows_per_episode[b] if rows_per_episode is not None else None
+            res.append(self.attend(layer, ids, q[cu_q[b]:cu_q[b + 1]],
+                                   k_new[cu_new[b]:cu_new[b + 1]], v_new[cu_new[b]:cu_new[b + 1]],
+                                   rows=rows))
+        return res
