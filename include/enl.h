@@ -1,0 +1,169 @@
+/*
+ * enl.h -- C ABI of the selective-KV attention library for navigation-map memory (B200, sm_100a).
+ *
+ * The paper (EfficientNav, arXiv 2510.18546) states the problem this boundary follows:
+ *   - Sec. 3.2 "Discrete Memory Caching": the navigation map is clustered into groups, each
+ *     group's KV cache is computed on its own and kept; any subset, in any order, is re-used
+ *     without recomputation; new objects are concatenated at the END of their group.
+ *   - App. C "Detailed Planning Example": the planner's prompt is the selected groups followed
+ *     by the new tokens (instruction + trajectory).
+ *   - App. A "LLM inference and KV Cache": Attn = softmax(Q K^T / sqrt(D)) V; decoding
+ *     concatenates the new token's K/V to what is already there.
+ *   - Sec. 3.3 "Attention-based Memory Clustering": the attention between new tokens and an
+ *     existing group decides clustering; this library returns the un-averaged primitive, the
+ *     post-softmax probability mass that each query row puts on each selected group.
+ *
+ * All K/V/Q/O tensors are bf16, row-major, DEVICE memory owned by the caller and kept alive
+ * until the stream reaches the call.  Index arrays (select list, prefix counts) are HOST
+ * memory and are consumed before the call returns.  The library owns the page pool, the
+ * group tables, the gather-plan buffers and the split-KV scratch, all allocated in
+ * enl_cache_create; enl_attend and enl_group_store allocate no device memory.
+ *
+ * Every device operation is enqueued on the stream the caller passes (a cudaStream_t cast to
+ * void*; NULL = the legacy default stream).  No call synchronises the device except
+ * enl_cache_create, enl_cache_free and enl_cache_status.  Validation happens on the host
+ * before anything is enqueued: a call that returns an error has enqueued nothing and has
+ * left the cache unchanged.
+ *
+ * No position encoding is applied here: cached K is stored as the caller produced it (already
+ * rotated at whatever positions the caller assigned to the group), so results do not depend
+ * on the order of the select list except for the order of the mass slots.
+ */
+#ifndef ENL_H
+#define ENL_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct enl_cache enl_cache_t;            /* opaque */
+
+enum { ENL_BF16 = 1 };
+enum { ENL_DEVICE_NONE = -1 };                   /* bookkeeping-only cache: tables, no GPU   */
+enum { ENL_REPLACE = 0, ENL_APPEND = 1 };        /* enl_group_store modes                    */
+
+enum {                                            /* enl_attend_args_t.flags                  */
+    ENL_PLAN_ONLY = 1u                            /* validate + build the gather plan + fill  */
+                                                  /* sel_off_out, enqueue nothing             */
+};
+
+enum {                                            /* return codes                             */
+    ENL_OK         =  0,
+    ENL_E_INVAL    = -1,   /* null pointer, bad shape, n_q > n_new, duplicate id in a list ...  */
+    ENL_E_NOGROUP  = -2,   /* group id out of range, or never stored for that layer            */
+    ENL_E_NOMEM    = -3,   /* page pool, plan buffers or a create-time allocation exhausted    */
+    ENL_E_CUDA     = -4,   /* a CUDA call failed, or a GPU operation on a bookkeeping cache    */
+    ENL_E_TIMEOUT  = -5    /* a bounded wait inside a kernel expired (see enl_cache_status)    */
+};
+
+typedef struct {
+    int32_t n_layers, n_q_heads, n_kv_heads;     /* n_q_heads = n_kv_heads * {1,2,4,8,16}    */
+    int32_t head_dim;                            /* 64 or 128                                */
+    int32_t page_tokens;                         /* 0 = library default (16); only 16 today  */
+    int32_t max_groups;                          /* group ids are 0 .. max_groups-1          */
+    int64_t max_tokens;                          /* pool capacity, tokens summed over groups */
+    int32_t dtype;                               /* ENL_BF16                                 */
+    int32_t device;                              /* CUDA ordinal, or ENL_DEVICE_NONE         */
+    int32_t max_batch;                           /* episodes per enl_attend; 0 = 64          */
+    int32_t max_q_tokens;                        /* query rows per enl_attend; 0 = 16384     */
+    int64_t scratch_bytes;                       /* split-KV scratch; 0 = 64 MiB             */
+} enl_cache_desc_t;
+
+/*
+ * Sec. 3.2: create the store that keeps every group's K/V.  Allocates, on desc->device, the
+ * K and V page pools for all layers ([layer][page][kv head][page_tokens][head_dim] bf16,
+ * zero-filled), the plan buffers and the scratch.  Synchronises the device.
+ * Errors: ENL_E_INVAL (bad shape), ENL_E_NOMEM (allocation failed), ENL_E_CUDA.
+ */
+int enl_cache_create(const enl_cache_desc_t *desc, enl_cache_t **out);
+
+/*
+ * Sec. 3.2: write one group's K/V for one layer ("compute KV cache of each group individually"
+ * and keep it), or append rows after the group's current end ("concatenate the information of
+ * new objects at the end of the group"; existing rows are not touched).
+ *   k_dev, v_dev : [n_tokens][n_kv_heads][head_dim] bf16, device; may be NULL only on a
+ *                  bookkeeping-only cache.
+ *   mode         : ENL_REPLACE sets the group's length for this layer to n_tokens;
+ *                  ENL_APPEND adds n_tokens rows after the current length.
+ * Pages are shared by all layers of a group, so a group's length must agree across the layers
+ * that are attended (checked in enl_attend).  n_tokens = 0 is legal (an empty group).
+ * Errors: ENL_E_INVAL, ENL_E_NOGROUP (id out of range), ENL_E_NOMEM (pool exhausted; state
+ * unchanged), ENL_E_CUDA.
+ */
+int enl_group_store(enl_cache_t *c, int32_t group_id, int32_t layer, int32_t n_tokens,
+                    const void *k_dev, const void *v_dev, int32_t mode, void *cuda_stream);
+
+typedef struct {
+    int32_t layer;
+    int32_t batch;                     /* independent episodes in this call, >= 1              */
+    const int32_t *sel_ids;            /* HOST [n_sel]: selected group ids, episode by episode */
+    const int32_t *cu_sel;             /* HOST [batch+1] prefix counts into sel_ids            */
+    const int32_t *cu_q;               /* HOST [batch+1] prefix counts of query rows           */
+    const int32_t *cu_new;             /* HOST [batch+1] prefix counts of new-token keys       */
+                                       /*   all three may be NULL when batch == 1              */
+    int32_t n_sel, n_q, n_new;         /* totals over the batch                                */
+    const void *q;                     /* device bf16 [n_q][n_q_heads][head_dim]               */
+    const void *k_new, *v_new;         /* device bf16 [n_new][n_kv_heads][head_dim]            */
+    void *out;                         /* device bf16 [n_q][n_q_heads][head_dim]               */
+    float *group_mass;                 /* device fp32 or NULL.  Row r (global over the batch), */
+                                       /*   q head h, slot s of its episode at                 */
+                                       /*   (r*n_q_heads + h)*mass_stride + s; slot s < G_b is */
+                                       /*   the s-th id of the episode's list, slot G_b the    */
+                                       /*   new tokens; entries past G_b are not written       */
+    int32_t mass_stride;               /* >= max_b(G_b) + 1                                    */
+    int32_t *sel_off_out;              /* HOST or NULL, [n_sel + batch]: per episode the       */
+                                       /*   exclusive prefix sum (G_b + 1 entries, in tokens)  */
+                                       /*   of its selected groups' lengths                    */
+    int32_t split_hint;                /* 0 = library chooses the number of KV splits,         */
+                                       /*   k >= 1 = use k splits (clamped to what fits)       */
+    uint32_t flags;                    /* ENL_PLAN_ONLY                                        */
+} enl_attend_args_t;
+
+/*
+ * App. A + App. C + Sec. 3.3: for every episode b, query row r and q head h (reading kv head
+ * h / (n_q_heads / n_kv_heads)):
+ *   keys   = the stored rows of the episode's selected groups, in list order, then the new
+ *            keys 0 .. c with c = (n_new_b - n_q_b) + r  (prefill: n_q_b = n_new_b; a decode
+ *            step passes n_q_b = 1 and the grown new-token buffer);
+ *   out    = softmax(q . keys / sqrt(head_dim)) . values           (fp32 accumulate, bf16 out)
+ *   mass   = the same probabilities summed per slot (fp32); every row sums to 1.
+ * A group appears at most once in an episode's list (the retrieval's x_i is 0 or 1, Sec. 3.4);
+ * an empty list is legal (plain causal attention), so is a zero-length group (mass 0).
+ * Errors: ENL_E_INVAL, ENL_E_NOGROUP, ENL_E_NOMEM (plan larger than the plan buffers),
+ * ENL_E_CUDA.  Kernel-side bounded waits report through enl_cache_status.
+ */
+int enl_attend(enl_cache_t *c, const enl_attend_args_t *args, void *cuda_stream);
+
+/* Releases everything enl_cache_create allocated.  Synchronises the device.  NULL is a no-op. */
+int enl_cache_free(enl_cache_t *c);
+
+/* ---- helpers (not part of the four calls above) ---------------------------------------- */
+
+/* Static text for a return code. */
+const char *enl_strerror(int code);
+
+/* Current length in tokens of a group for a layer, -1 if never stored, ENL_E_* on a bad id. */
+int32_t enl_group_len(const enl_cache_t *c, int32_t group_id, int32_t layer);
+
+/* Synchronises the device and returns ENL_OK, or ENL_E_TIMEOUT if any kernel of this cache
+ * gave up on a bounded wait since the last call (the flag is then cleared). */
+int enl_cache_status(enl_cache_t *c);
+
+/*
+ * Read-back of the gather plan built by the last enl_attend (host copy), for tests of the
+ * integer book-keeping.  Each array pointer may be NULL; counts are always written.
+ *   stream_pages[i], stream_meta[i] : page id and (slot << 8 | valid tokens) of KV-stream entry i
+ *   ep_stream_off[b], ep_cached_tiles[b] : first entry and number of 128-key tiles of episode b
+ *   n_splits : KV splits chosen;  n_items : CTAs of the attention launch
+ */
+int enl_plan_inspect(const enl_cache_t *c, int32_t cap_entries, int32_t *stream_pages,
+                     int32_t *stream_meta, int32_t *n_entries, int32_t cap_batch,
+                     int32_t *ep_stream_off, int32_t *ep_cached_tiles, int32_t *n_splits,
+                     int32_t *n_items);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ENL_H */

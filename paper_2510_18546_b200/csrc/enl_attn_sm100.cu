@@ -1,0 +1,585 @@
+// Selective-KV flash attention with fused per-group mass, sm_100a (tcgen05 + TMEM + TMA).
+//
+// What it computes (paper, App. A: softmax(Q K^T / sqrt(D)) V; App. C: the prompt is the selected
+// groups followed by the new tokens; Sec. 3.3: attention between new tokens and a group):
+// one CTA takes two Q tiles of 128 rows each -- (128/rep) consecutive query tokens x the rep q heads
+// that read one kv head -- and walks the key stream of its episode: the selected groups' pages in
+// list order (eight 16-token pages per 128-key tile, fetched as separate TMA boxes from wherever the
+// pages lie in the pool), then the new-token keys up to the causal limit.  Per tile:
+//   S_i = Q_i K^T            tcgen05.mma, operands in shared memory, accumulator in TMEM
+//   p   = exp2(S * c - m)    one thread per row, fp32; padding and causally hidden columns -> 0
+//   O_i += P_i V             tcgen05.mma, P (bf16) read from TMEM, V from shared memory
+// The row sum of p is split by the slot (selected group, or the new tokens) each 16-key page belongs
+// to; when a slot ends its log2-sum-exp is parked in the mass buffer, and after the last tile the row
+// turns those into probabilities.  With KV splits every split writes partial results that a second
+// kernel merges.
+//
+// Roles: warps 0-3 softmax of Q tile 0, warps 4-7 softmax of Q tile 1, warp 8 TMA producer,
+// warp 9 MMA issuer (and TMEM owner).  TMEM columns: S0 [0,128) S1 [128,256) O0 [256,384) O1 [384,512);
+// P_i overwrites the first 64 columns of S_i.
+#include <cuda_bf16.h>
+
+#include "enl_internal.h"
+#include "tmem_ops.cuh"
+
+namespace enl {
+namespace {
+
+constexpr int kThreads      = 320;
+constexpr int kProducerWarp = 8;
+constexpr int kMmaWarp      = 9;
+constexpr uint32_t kTmemCols = 512;
+constexpr float kRescaleThreshold = 8.0f;     // log2 units: p stays below 2^8 between max updates
+constexpr unsigned long long kWaitLimitNs = 1000ull * 1000ull * 1000ull;
+
+template <int D>
+struct Cfg {
+    static constexpr int kHalves    = D / 64;             // 64-channel (128-byte) column blocks
+    static constexpr int kHalfBytes = 128 * 128;          // 128 rows x 128 B
+    static constexpr int kTileBytes = kHalves * kHalfBytes;
+    static constexpr int kStages    = (D == 128) ? 5 : 8;
+    static constexpr int kBarOff    = (kQTiles + kStages) * kTileBytes;
+    static constexpr int kSmemBytes = kBarOff + 512 + 1024;   // barriers + alignment slack
+};
+
+// ---- small PTX wrappers ------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p)
+{
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait: gives up after kWaitLimitNs or when another role has raised the abort flag.
+// The result is made warp-uniform so that warp-collective tcgen05 instructions stay converged.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                          int32_t *status)
+{
+    bool ok = mbar_try_wait(bar, parity);
+    if (!ok) {
+        const unsigned long long t0 = global_ns();
+        uint32_t spins = 0;
+        while (!(ok = mbar_try_wait(bar, parity))) {
+            if ((++spins & 63u) == 0u) {
+                if (*abort_flag) break;
+                if (global_ns() - t0 > kWaitLimitNs) {
+                    *abort_flag = 1;
+                    atomicExch(status, 1);
+                    break;
+                }
+            }
+        }
+    }
+    return __all_sync(0xffffffffu, ok);
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tm, int x, int y, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *tm, int x, int y, int z, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after()  { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]
+__device__ __forceinline__ void mma_ss(uint32_t d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem]
+__device__ __forceinline__ void mma_ts(uint32_t d, uint32_t a, uint64_t bdesc, uint32_t idesc, uint32_t acc)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d), "r"(a), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ float ex2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float lg2(float x)
+{
+    float y;
+    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle, rows of 128 B, 8-row groups 1024 B apart.
+// K-major operand (the contraction dimension is contiguous): LBO unused.
+// MN-major operand: LBO = distance between 64-element column blocks.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes)
+{
+    uint64_t d = 0;
+    d |= static_cast<uint64_t>((addr & 0x3FFFFu) >> 4);               // start address
+    d |= static_cast<uint64_t>((lbo_bytes >> 4) & 0x3FFFu) << 16;      // leading byte offset
+    d |= static_cast<uint64_t>(1024u >> 4) << 32;                      // stride byte offset
+    d |= static_cast<uint64_t>(1) << 46;                               // descriptor version (sm_100)
+    d |= static_cast<uint64_t>(2) << 61;                               // 128-byte swizzle
+    return d;
+}
+// Instruction descriptor, kind::f16: bf16 x bf16 -> fp32, M = 128.
+__host__ __device__ constexpr uint32_t make_idesc(int n, bool b_mn_major)
+{
+    return (1u << 4)                              // D format fp32
+         | (1u << 7) | (1u << 10)                 // A, B format bf16
+         | ((b_mn_major ? 1u : 0u) << 16)         // B major
+         | (static_cast<uint32_t>(n >> 3) << 17)  // N
+         | (static_cast<uint32_t>(128 >> 4) << 24);  // M
+}
+
+constexpr float kNegInf = -__builtin_huge_valf();
+
+// ---- the kernel ----------------------------------------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant__ AttnParams p)
+{
+    using C = Cfg<D>;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t sbase = (raw + 1023u) & ~1023u;               // 1024-B aligned (swizzle atoms)
+    uint8_t *smem = smem_raw + (sbase - raw);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    // shared-memory map
+    auto q_addr     = [&](int i) { return sbase + static_cast<uint32_t>(i * C::kTileBytes); };
+    auto stage_addr = [&](int s) { return sbase + static_cast<uint32_t>((kQTiles + s) * C::kTileBytes); };
+    const uint32_t bar0 = sbase + C::kBarOff;
+    const uint32_t bar_q_full = bar0;
+    auto bar_kv_full  = [&](int s) { return bar0 + 8u * (1 + s); };
+    auto bar_kv_empty = [&](int s) { return bar0 + 8u * (1 + C::kStages + s); };
+    auto bar_s_full   = [&](int i) { return bar0 + 8u * (1 + 2 * C::kStages + i); };
+    auto bar_p_full   = [&](int i) { return bar0 + 8u * (3 + 2 * C::kStages + i); };
+    auto bar_o_done   = [&](int i) { return bar0 + 8u * (5 + 2 * C::kStages + i); };
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + C::kBarOff + 8 * (7 + 2 * C::kStages));
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+    // work item
+    const Item it = p.items[blockIdx.x];
+    const EpInfo ep = p.eps[it.ep];
+    const int rep = p.rep;
+    const int tile_tokens = kTileRows / rep;
+    const int t_hi = min(it.t0 + kQTiles * tile_tokens, ep.n_q);        // exclusive
+    const int n_qt = (t_hi - it.t0 > tile_tokens) ? 2 : 1;
+    const int c_max = ep.n_new - ep.n_q + t_hi - 1;                      // last new key any row sees
+    const int n_new_tiles = c_max / kTileKeys + 1;
+    const int total_tiles = ep.n_ctiles + n_new_tiles;
+    const int j_beg = static_cast<int>(static_cast<long long>(total_tiles) * it.split / p.n_splits);
+    const int j_end = static_cast<int>(static_cast<long long>(total_tiles) * (it.split + 1) / p.n_splits);
+    const int n_tiles = j_end - j_beg;
+
+    // ---- set-up ----
+    if (threadIdx.x == 0) {
+        *abort_flag = 0;
+        mbar_init(bar_q_full, 1);
+        for (int s = 0; s < C::kStages; ++s) { mbar_init(bar_kv_full(s), 1); mbar_init(bar_kv_empty(s), 1); }
+        for (int i = 0; i < kQTiles; ++i) {
+            mbar_init(bar_s_full(i), 1);
+            mbar_init(bar_p_full(i), 4);          // one arrival per softmax warp
+            mbar_init(bar_o_done(i), 1);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == kMmaWarp) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    bool ok = true;
+
+    if (warp == kProducerWarp) {
+        // ================= TMA producer =================
+        if (n_tiles > 0) {
+            if (lane == 0) {
+                mbar_expect_tx(bar_q_full, static_cast<uint32_t>(n_qt * C::kTileBytes));
+                for (int i = 0; i < n_qt; ++i)
+                    for (int hf = 0; hf < C::kHalves; ++hf)
+                        tma_load_3d(q_addr(i) + hf * C::kHalfBytes, &p.tm_q, hf * 64, it.kvh * rep,
+                                    ep.q_off + it.t0 + i * tile_tokens, bar_q_full);
+            }
+            int fill = 0;
+            for (int j = j_beg; j < j_end && ok; ++j) {
+                const bool cached = j < ep.n_ctiles;
+                int page = 0;
+                if (cached && lane < kPagesPerTile)
+                    page = p.stream[ep.stream_off + j * kPagesPerTile + lane].x;
+                for (int kv = 0; kv < 2; ++kv, ++fill) {
+                    const int st = fill % C::kStages;
+                    if (fill >= C::kStages) {
+                        ok = mbar_wait(bar_kv_empty(st), static_cast<uint32_t>((fill / C::kStages - 1) & 1),
+                                       abort_flag, p.status);
+                        if (!ok) break;
+                    }
+                    const uint32_t full = bar_kv_full(st);
+                    if (lane == 0) mbar_expect_tx(full, static_cast<uint32_t>(C::kTileBytes));
+                    __syncwarp();
+                    const uint32_t dst = stage_addr(st);
+                    if (cached) {
+                        if (lane < kPagesPerTile) {
+                            const CUtensorMap *tm = kv ? &p.tm_vpool : &p.tm_kpool;
+                            const int row = (page * p.Hkv + it.kvh) * kPageTokens;
+                            for (int hf = 0; hf < C::kHalves; ++hf)
+                                tma_load_2d(dst + hf * C::kHalfBytes + lane * (kPageTokens * 128), tm,
+                                            hf * 64, row, full);
+                        }
+                    } else if (lane == 0) {
+                        const CUtensorMap *tm = kv ? &p.tm_vnew : &p.tm_knew;
+                        const int krow = ep.new_off + (j - ep.n_ctiles) * kTileKeys;
+                        for (int hf = 0; hf < C::kHalves; ++hf)
+                            tma_load_3d(dst + hf * C::kHalfBytes, tm, hf * 64, it.kvh, krow, full);
+                    }
+                }
+            }
+            // error path only: let the copies already in flight land before the CTA retires
+            if (!ok) {
+                const int first = fill > C::kStages ? fill - C::kStages : 0;
+                for (int f = first; f < fill; ++f) {
+                    const unsigned long long t0 = global_ns();
+                    while (!mbar_try_wait(bar_kv_full(f % C::kStages), static_cast<uint32_t>((f / C::kStages) & 1)) &&
+                           global_ns() - t0 < 2000000ull) { }
+                }
+            }
+        }
+    } else if (warp == kMmaWarp) {
+        // ================= MMA issuer =================
+        if (n_tiles > 0) {
+            constexpr uint32_t idesc_qk = make_idesc(kTileKeys, false);
+            constexpr uint32_t idesc_pv = make_idesc(D, true);
+            auto tmem_s = [&](int i) { return tmem_base + static_cast<uint32_t>(i * 128); };
+            auto tmem_o = [&](int i) { return tmem_base + static_cast<uint32_t>(256 + i * 128); };
+            auto issue_qk = [&](int i, int st) {
+                if (lane == 0) {
+#pragma unroll
+                    for (int kk = 0; kk < D / 16; ++kk) {
+                        const uint32_t off = static_cast<uint32_t>((kk >> 2) * C::kHalfBytes + (kk & 3) * 32);
+                        mma_ss(tmem_s(i), smem_desc(q_addr(i) + off, 16), smem_desc(stage_addr(st) + off, 16),
+                               idesc_qk, kk > 0 ? 1u : 0u);
+                    }
+                    tc_commit(bar_s_full(i));
+                }
+                __syncwarp();
+            };
+            auto issue_pv = [&](int i, int st, bool first_tile) {
+                if (lane == 0) {
+#pragma unroll
+                    for (int kk = 0; kk < kTileKeys / 16; ++kk) {
+                        mma_ts(tmem_o(i), tmem_s(i) + static_cast<uint32_t>(kk * 8),
+                               smem_desc(stage_addr(st) + static_cast<uint32_t>(kk * 16 * 128), C::kHalfBytes),
+                               idesc_pv, (first_tile && kk == 0) ? 0u : 1u);
+                    }
+                }
+                __syncwarp();
+            };
+            auto commit_to = [&](uint32_t bar) {
+                if (lane == 0) tc_commit(bar);
+                __syncwarp();
+            };
+            auto wait_full = [&](int f) {
+                return mbar_wait(bar_kv_full(f % C::kStages), static_cast<uint32_t>((f / C::kStages) & 1),
+                                 abort_flag, p.status);
+            };
+
+            ok = mbar_wait(bar_q_full, 0, abort_flag, p.status);
+            if (ok) ok = wait_full(0);
+            if (ok) {
+                tc_fence_after();
+                for (int i = 0; i < n_qt; ++i) issue_qk(i, 0);
+                commit_to(bar_kv_empty(0));
+            }
+            for (int jj = 0; jj < n_tiles && ok; ++jj) {
+                const int fv = 2 * jj + 1, fk = 2 * jj + 2;             // ring slots of V_jj and K_{jj+1}
+                const bool more = jj + 1 < n_tiles;
+                ok = wait_full(fv);
+                if (ok && more) ok = wait_full(fk);
+                if (!ok) break;
+                for (int i = 0; i < n_qt; ++i) {
+                    ok = mbar_wait(bar_p_full(i), static_cast<uint32_t>(jj & 1), abort_flag, p.status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_pv(i, fv % C::kStages, jj == 0);
+                    if (i == n_qt - 1) commit_to(bar_kv_empty(fv % C::kStages));
+                    if (!more) commit_to(bar_o_done(i));
+                    if (more) {
+                        issue_qk(i, fk % C::kStages);
+                        if (i == n_qt - 1) commit_to(bar_kv_empty(fk % C::kStages));
+                    }
+                }
+            }
+        }
+    } else if ((warp >> 2) < n_qt) {
+        // ================= softmax / epilogue, one thread per row =================
+        const int i = warp >> 2;
+        const int r = (warp & 3) * 32 + lane;
+        const int t = it.t0 + i * tile_tokens + r / rep;          // episode-relative query token
+        const int h = it.kvh * rep + r % rep;
+        const bool row_valid = t < ep.n_q;
+        const int c = min(ep.n_new - ep.n_q + t, ep.n_new - 1);  // last visible new key
+        const int G = ep.n_slots;
+        const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;
+        const uint32_t t_s = tmem_base + lane_sel + static_cast<uint32_t>(i * 128);
+        const uint32_t t_o = tmem_base + lane_sel + static_cast<uint32_t>(256 + i * 128);
+        const bool split_mode = p.n_splits > 1;
+        const long long grow = static_cast<long long>(ep.q_off) + t;   // global query row
+        const long long rh = (split_mode ? (static_cast<long long>(it.split) * p.n_q_total + grow) : grow) * p.Hq + h;
+        float *slot_out = nullptr;
+        if (row_valid) {
+            if (split_mode) { if (p.part_slot) slot_out = p.part_slot + rh * p.mass_stride; }
+            else if (p.mass) slot_out = p.mass + rh * p.mass_stride;
+        }
+        const float scale = p.scale_log2;
+
+        float m = kNegInf, l = 0.f, acc = 0.f;
+        int cur_slot = -1;
+
+        for (int jj = 0; jj < n_tiles; ++jj) {
+            const int j = j_beg + jj;
+            const bool cached = j < ep.n_ctiles;
+            int meta[kPagesPerTile];
+            if (cached) {
+                const int4 *e4 = reinterpret_cast<const int4 *>(p.stream + ep.stream_off + j * kPagesPerTile);
+#pragma unroll
+                for (int e = 0; e < kPagesPerTile / 2; ++e) {
+                    const int4 v = __ldg(e4 + e);
+                    meta[2 * e] = v.y;
+                    meta[2 * e + 1] = v.w;
+                }
+            } else {
+#pragma unroll
+                for (int e = 0; e < kPagesPerTile; ++e) meta[e] = (G << 8) | kPageTokens;
+            }
+            ok = mbar_wait(bar_s_full(i), static_cast<uint32_t>(jj & 1), abort_flag, p.status);
+            if (!ok) break;
+            tc_fence_after();
+
+            uint32_t su[128];
+            tmem_ld128_wait(t_s, su);
+            float s[128];
+#pragma unroll
+            for (int x = 0; x < 128; ++x) s[x] = __uint_as_float(su[x]);
+
+            // hide page padding (cached tiles) or keys after the causal limit (new-token tiles)
+            if (cached) {
+#pragma unroll
+                for (int e = 0; e < kPagesPerTile; ++e) {
+                    const int nv = meta[e] & 0xff;
+                    if (nv < kPageTokens) {
+#pragma unroll
+                        for (int x = 0; x < kPageTokens; ++x)
+                            if (x >= nv) s[e * kPageTokens + x] = kNegInf;
+                    }
+                }
+            } else {
+                const int lim = c - (j - ep.n_ctiles) * kTileKeys;
+                if (__any_sync(0xffffffffu, lim < kTileKeys - 1)) {
+#pragma unroll
+                    for (int x = 0; x < 128; ++x)
+                        if (x > lim) s[x] = kNegInf;
+                }
+            }
+
+            float mx = s[0];
+#pragma unroll
+            for (int x = 1; x < 128; ++x) mx = fmaxf(mx, s[x]);
+            const float m_cand = mx * scale;
+            const bool need = m_cand > m + kRescaleThreshold;       // also true when m == -inf < m_cand
+            if (__any_sync(0xffffffffu, need)) {
+                const float m_new = fmaxf(m, m_cand);
+                const float alpha = (m_new == kNegInf) ? 1.f : ex2(m - m_new);
+                l *= alpha;
+                acc *= alpha;
+                m = m_new;
+                if (jj > 0) {                                        // O_i holds the tiles so far
+#pragma unroll
+                    for (int k = 0; k < D / 32; ++k) {
+                        uint32_t o[32];
+                        tmem_ld32_wait(t_o + k * 32, o);
+#pragma unroll
+                        for (int x = 0; x < 32; ++x) o[x] = __float_as_uint(__uint_as_float(o[x]) * alpha);
+                        tmem_st32(t_o + k * 32, o);
+                    }
+                }
+            }
+            const float m_use = (m == kNegInf) ? 0.f : m;
+
+#pragma unroll
+            for (int e = 0; e < kPagesPerTile; ++e) {
+                float bs = 0.f;
+#pragma unroll
+                for (int x = 0; x < kPageTokens; ++x) {
+                    const float pv = ex2(fmaf(s[e * kPageTokens + x], scale, -m_use));
+                    s[e * kPageTokens + x] = pv;
+                    bs += pv;
+                }
+                const int slot = meta[e] >> 8;
+                if (slot != cur_slot) {
+                    if (slot_out && cur_slot >= 0) slot_out[cur_slot] = lg2(acc) + m_use;
+                    acc = 0.f;
+                    cur_slot = slot;
+                }
+                acc += bs;
+                l += bs;
+            }
+
+            // P (bf16 pairs, even key in the low half) over the first 64 columns of S_i
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                uint32_t pk[16];
+#pragma unroll
+                for (int x = 0; x < 16; ++x) {
+                    const __nv_bfloat162 b = __floats2bfloat162_rn(s[k * 32 + 2 * x], s[k * 32 + 2 * x + 1]);
+                    pk[x] = *reinterpret_cast<const uint32_t *>(&b);
+                }
+                tmem_st16(t_s + k * 16, pk);
+            }
+            tmem_st_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_p_full(i));
+        }
+
+        // ---- per-row results ----
+        const float m_use = (m == kNegInf) ? 0.f : m;
+        if (ok) {
+            if (slot_out && cur_slot >= 0) slot_out[cur_slot] = lg2(acc) + m_use;
+            const float lse = (l > 0.f) ? m_use + lg2(l) : kNegInf;
+            if (split_mode) {
+                if (row_valid) {
+                    // slots this split did not walk contribute nothing
+                    int first = G + 1, last = -1;
+                    if (n_tiles > 0) {
+                        first = (j_beg < ep.n_ctiles)
+                                    ? (p.stream[ep.stream_off + j_beg * kPagesPerTile].y >> 8) : G;
+                        last = (j_end > ep.n_ctiles)
+                                   ? G : (p.stream[ep.stream_off + j_end * kPagesPerTile - 1].y >> 8);
+                    }
+                    if (slot_out)
+                        for (int sl = 0; sl <= G; ++sl)
+                            if (sl < first || sl > last) slot_out[sl] = kNegInf;
+                    p.part_lse[rh] = lse;
+                }
+            } else if (slot_out) {
+                for (int sl = 0; sl <= G; ++sl) slot_out[sl] = ex2(slot_out[sl] - lse);
+            }
+            if (n_tiles > 0) {
+                ok = mbar_wait(bar_o_done(i), 0, abort_flag, p.status);
+                if (ok) {
+                    tc_fence_after();
+                    const float inv = (l > 0.f) ? 1.f / l : 0.f;
+#pragma unroll
+                    for (int k = 0; k < D / 32; ++k) {
+                        uint32_t o[32];
+                        tmem_ld32_wait(t_o + k * 32, o);
+                        if (row_valid) {
+                            if (split_mode) {
+                                float4 *dst = reinterpret_cast<float4 *>(p.part_o + rh * D + k * 32);
+#pragma unroll
+                                for (int x = 0; x < 8; ++x)
+                                    dst[x] = make_float4(__uint_as_float(o[4 * x]) * inv, __uint_as_float(o[4 * x + 1]) * inv,
+                                                         __uint_as_float(o[4 * x + 2]) * inv, __uint_as_float(o[4 * x + 3]) * inv);
+                            } else {
+                                uint4 *dst = reinterpret_cast<uint4 *>(
+                                    static_cast<__nv_bfloat16 *>(p.out) + rh * D + k * 32);
+#pragma unroll
+                                for (int x = 0; x < 4; ++x) {
+                                    uint32_t w[4];
+#pragma unroll
+                                    for (int y = 0; y < 4; ++y) {
+                                        const __nv_bfloat162 b = __floats2bfloat162_rn(
+                                            __uint_as_float(o[8 * x + 2 * y]) * inv,
+                                            __uint_as_float(o[8 * x + 2 * y + 1]) * inv);
+                                        w[y] = *reinterpret_cast<const uint32_t *>(&b);
+                                    }
+                                    dst[x] = make_uint4(w[0], w[1], w[2], w[3]);
+                                }
+                            }
+                        }
+                    }
+                }
+            }
+        }
+    }
+
+    // ---- teardown ----
+    tc_fence_before();
+    __syncthreads();
+    if (warp == kMmaWarp) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    }
+}
+
+}  // namespace
+
+size_t attention_smem_bytes(int head_dim)
+{
+    return head_dim == 128 ? Cfg<128>::kSmemBytes : Cfg<64>::kSmemBytes;
+}
+
+cudaError_t prepare_attention(int head_dim)
+{
+    if (head_dim == 128)
+        return cudaFuncSetAttribute(attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<128>::kSmemBytes);
+    if (head_dim == 64)
+        return cudaFuncSetAttribute(attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<64>::kSmemBytes);
+    return cudaErrorInvalidValue;
+}
+
+cudaError_t launch_attention(const AttnParams &p, int head_dim, int n_items, cudaStream_t st)
+{
+    if (n_items <= 0) return cudaSuccess;
+    if (head_dim == 128)
+        attn_kernel<128><<<n_items, kThreads, Cfg<128>::kSmemBytes, st>>>(p);
+    else if (head_dim == 64)
+        attn_kernel<64><<<n_items, kThreads, Cfg<64>::kSmemBytes, st>>>(p);
+    else
+        return cudaErrorInvalidValue;
+    return cudaGetLastError();
+}
+
+}  // namespace enl

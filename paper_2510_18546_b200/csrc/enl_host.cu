@@ -1,0 +1,578 @@
+// Host side of the library: the paged per-group KV store, the gather plan and the four C-ABI calls.
+// Everything here is integer book-keeping plus launches; all arithmetic of the method runs in kernels.
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/enl.h"
+#include "enl_internal.h"
+
+using namespace enl;
+
+namespace {
+
+struct Group {
+    std::vector<int32_t> pages;       // shared by all layers: positions 16*i .. 16*i+15 live in pages[i]
+    std::vector<int32_t> len;         // per layer, -1 = never stored
+};
+
+struct DeviceGuard {
+    int prev = -1;
+    bool switched = false;
+    explicit DeviceGuard(int dev)
+    {
+        if (dev < 0) return;
+        if (cudaGetDevice(&prev) == cudaSuccess && prev != dev) {
+            cudaSetDevice(dev);
+            switched = true;
+        }
+    }
+    ~DeviceGuard()
+    {
+        if (switched) cudaSetDevice(prev);
+    }
+};
+
+using EncodeTiledFn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                   CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
+// bf16 tensor map with 128-byte swizzle; dims/box innermost first, strides in bytes for dims 1..rank-1.
+bool encode_map(CUtensorMap *tm, const void *base, int rank, const cuuint64_t *dims, const cuuint64_t *strides,
+                const cuuint32_t *box)
+{
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, static_cast<cuuint32_t>(rank), const_cast<void *>(base), dims,
+              strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+}  // namespace
+
+struct enl_cache {
+    enl_cache_desc_t d{};
+    bool gpu = false;
+    int rep = 1;
+    int64_t n_pages = 0;
+    size_t layer_bytes = 0;                 // one layer of one pool
+    uint8_t *kpool = nullptr, *vpool = nullptr;
+    std::vector<int32_t> free_pages;        // stack of free page ids (page 0 is never in it)
+    std::vector<Group> groups;
+    std::vector<CUtensorMap> tm_k, tm_v;    // per layer
+    uint64_t epoch = 0;                     // bumped by every store
+
+    // gather plan: host image (pinned when there is a GPU), device copy, capacities
+    int32_t cap_entries = 0, cap_items = 0;
+    uint8_t *plan_host = nullptr, *plan_dev = nullptr;
+    size_t off_eps = 0, off_items = 0, off_stream = 0, off_rowslots = 0, plan_bytes = 0;
+    cudaEvent_t plan_copied = nullptr;
+    bool plan_valid = false, plan_on_device = false;
+    uint64_t plan_epoch = 0;
+    int32_t plan_split_hint = 0;
+    bool plan_has_mass = false;
+    std::vector<int32_t> key_sel, key_cu, key_len;   // what the current plan was built from
+    int32_t plan_entries = 0, plan_items = 0, plan_splits = 1, plan_batch = 0, plan_max_slots = 0;
+    std::vector<int32_t> seen;              // duplicate detection stamps
+    int32_t stamp = 0;
+
+    float *scratch = nullptr;
+    int32_t *status_dev = nullptr;
+
+    EpInfo *h_eps() { return reinterpret_cast<EpInfo *>(plan_host + off_eps); }
+    Item *h_items() { return reinterpret_cast<Item *>(plan_host + off_items); }
+    int2 *h_stream() { return reinterpret_cast<int2 *>(plan_host + off_stream); }
+    int32_t *h_rowslots() { return reinterpret_cast<int32_t *>(plan_host + off_rowslots); }
+};
+
+namespace {
+
+void destroy(enl_cache *c)
+{
+    if (!c) return;
+    if (c->gpu) {
+        DeviceGuard g(c->d.device);
+        cudaDeviceSynchronize();
+        if (c->kpool) cudaFree(c->kpool);
+        if (c->vpool) cudaFree(c->vpool);
+        if (c->plan_dev) cudaFree(c->plan_dev);
+        if (c->plan_host) cudaFreeHost(c->plan_host);
+        if (c->scratch) cudaFree(c->scratch);
+        if (c->status_dev) cudaFree(c->status_dev);
+        if (c->plan_copied) cudaEventDestroy(c->plan_copied);
+    } else {
+        delete[] c->plan_host;
+    }
+    delete c;
+}
+
+int tokens_per_cta(const enl_cache *c) { return kQTiles * (kTileRows / c->rep); }
+
+}  // namespace
+
+extern "C" const char *enl_strerror(int code)
+{
+    switch (code) {
+        case ENL_OK: return "ok";
+        case ENL_E_INVAL: return "invalid argument";
+        case ENL_E_NOGROUP: return "group id out of range or group never stored for this layer";
+        case ENL_E_NOMEM: return "out of pool pages, plan space or memory";
+        case ENL_E_CUDA: return "CUDA error, or GPU operation on a bookkeeping-only cache";
+        case ENL_E_TIMEOUT: return "a bounded wait inside a kernel expired";
+        default: return "unknown error";
+    }
+}
+
+extern "C" int enl_cache_create(const enl_cache_desc_t *desc, enl_cache_t **out)
+{
+    if (!desc || !out) return ENL_E_INVAL;
+    *out = nullptr;
+    enl_cache_desc_t d = *desc;
+    if (d.page_tokens == 0) d.page_tokens = kPageTokens;
+    if (d.max_batch == 0) d.max_batch = 64;
+    if (d.max_q_tokens == 0) d.max_q_tokens = 16384;
+    if (d.scratch_bytes == 0) d.scratch_bytes = 64ll << 20;
+    if (d.n_layers <= 0 || d.n_q_heads <= 0 || d.n_kv_heads <= 0 || d.n_q_heads % d.n_kv_heads != 0)
+        return ENL_E_INVAL;
+    const int rep = d.n_q_heads / d.n_kv_heads;
+    if (rep != 1 && rep != 2 && rep != 4 && rep != 8 && rep != 16) return ENL_E_INVAL;
+    if (d.head_dim != 64 && d.head_dim != 128) return ENL_E_INVAL;
+    if (d.page_tokens != kPageTokens || d.dtype != ENL_BF16) return ENL_E_INVAL;
+    if (d.max_groups <= 0 || d.max_tokens <= 0 || d.max_batch < 0 || d.max_q_tokens < 0 || d.scratch_bytes < 0)
+        return ENL_E_INVAL;
+    if (d.device < 0 && d.device != ENL_DEVICE_NONE) return ENL_E_INVAL;
+
+    enl_cache *c = new (std::nothrow) enl_cache;
+    if (!c) return ENL_E_NOMEM;
+    c->d = d;
+    c->rep = rep;
+    c->gpu = d.device >= 0;
+    // every group may waste up to one page of padding; page 0 stays the all-zero page
+    c->n_pages = (d.max_tokens + kPageTokens - 1) / kPageTokens + d.max_groups + 1;
+    if (c->n_pages * d.n_kv_heads * kPageTokens > 0x7fffffffll) { delete c; return ENL_E_INVAL; }
+    c->layer_bytes = static_cast<size_t>(c->n_pages) * d.n_kv_heads * kPageTokens * d.head_dim * 2;
+    c->groups.resize(d.max_groups);
+    c->seen.assign(d.max_groups, 0);
+    c->free_pages.reserve(c->n_pages);
+    for (int64_t pg = c->n_pages - 1; pg >= 1; --pg) c->free_pages.push_back(static_cast<int32_t>(pg));
+
+    const int tpc = tokens_per_cta(c);
+    c->cap_entries = static_cast<int32_t>(std::min<int64_t>(2 * c->n_pages + kPagesPerTile * (d.max_batch + 1), 0x7ffffff0));
+    c->cap_items = std::max(4096, (d.max_q_tokens / tpc + d.max_batch + 1) * d.n_kv_heads);
+    auto align256 = [](size_t x) { return (x + 255) & ~static_cast<size_t>(255); };
+    c->off_eps = 0;
+    c->off_items = align256(c->off_eps + sizeof(EpInfo) * d.max_batch);
+    c->off_stream = align256(c->off_items + sizeof(Item) * c->cap_items);
+    c->off_rowslots = align256(c->off_stream + sizeof(int2) * c->cap_entries);
+    c->plan_bytes = align256(c->off_rowslots + sizeof(int32_t) * d.max_q_tokens);
+
+    if (!c->gpu) {
+        c->plan_host = new (std::nothrow) uint8_t[c->plan_bytes];
+        if (!c->plan_host) { destroy(c); return ENL_E_NOMEM; }
+        *out = c;
+        return ENL_OK;
+    }
+
+    int n_dev = 0;
+    if (cudaGetDeviceCount(&n_dev) != cudaSuccess || d.device >= n_dev) { cudaGetLastError(); delete c; return ENL_E_CUDA; }
+    DeviceGuard g(d.device);
+    if (!get_encode_fn()) { delete c; return ENL_E_CUDA; }
+    const size_t pool_bytes = c->layer_bytes * d.n_layers;
+    bool okm = cudaMalloc(&c->kpool, pool_bytes) == cudaSuccess && cudaMalloc(&c->vpool, pool_bytes) == cudaSuccess &&
+               cudaMalloc(&c->plan_dev, c->plan_bytes) == cudaSuccess &&
+               cudaMallocHost(&c->plan_host, c->plan_bytes) == cudaSuccess &&
+               cudaMalloc(&c->scratch, static_cast<size_t>(d.scratch_bytes)) == cudaSuccess &&
+               cudaMalloc(&c->status_dev, sizeof(int32_t)) == cudaSuccess;
+    if (!okm) { cudaGetLastError(); destroy(c); return ENL_E_NOMEM; }
+    bool okc = cudaMemset(c->kpool, 0, pool_bytes) == cudaSuccess && cudaMemset(c->vpool, 0, pool_bytes) == cudaSuccess &&
+               cudaMemset(c->status_dev, 0, sizeof(int32_t)) == cudaSuccess &&
+               cudaEventCreateWithFlags(&c->plan_copied, cudaEventDisableTiming) == cudaSuccess &&
+               cudaEventRecord(c->plan_copied, 0) == cudaSuccess;
+    if (!okc) { cudaGetLastError(); destroy(c); return ENL_E_CUDA; }
+
+    c->tm_k.resize(d.n_layers);
+    c->tm_v.resize(d.n_layers);
+    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(d.head_dim),
+                                static_cast<cuuint64_t>(c->n_pages) * d.n_kv_heads * kPageTokens};
+    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(d.head_dim) * 2};
+    const cuuint32_t box[2] = {64, kPageTokens};
+    for (int l = 0; l < d.n_layers; ++l) {
+        if (!encode_map(&c->tm_k[l], c->kpool + c->layer_bytes * l, 2, dims, strides, box) ||
+            !encode_map(&c->tm_v[l], c->vpool + c->layer_bytes * l, 2, dims, strides, box)) {
+            destroy(c);
+            return ENL_E_CUDA;
+        }
+    }
+    if (prepare_attention(d.head_dim) != cudaSuccess) { cudaGetLastError(); destroy(c); return ENL_E_CUDA; }
+    if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); destroy(c); return ENL_E_CUDA; }
+    *out = c;
+    return ENL_OK;
+}
+
+extern "C" int enl_cache_free(enl_cache_t *c)
+{
+    destroy(c);
+    return ENL_OK;
+}
+
+extern "C" int32_t enl_group_len(const enl_cache_t *c, int32_t group_id, int32_t layer)
+{
+    if (!c) return ENL_E_INVAL;
+    if (group_id < 0 || group_id >= c->d.max_groups) return ENL_E_NOGROUP;
+    if (layer < 0 || layer >= c->d.n_layers) return ENL_E_INVAL;
+    const Group &g = c->groups[group_id];
+    return g.len.empty() ? -1 : g.len[layer];
+}
+
+extern "C" int enl_cache_status(enl_cache_t *c)
+{
+    if (!c) return ENL_E_INVAL;
+    if (!c->gpu) return ENL_OK;
+    DeviceGuard g(c->d.device);
+    if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return ENL_E_CUDA; }
+    int32_t st = 0;
+    if (cudaMemcpy(&st, c->status_dev, sizeof st, cudaMemcpyDeviceToHost) != cudaSuccess) return ENL_E_CUDA;
+    if (st != 0) {
+        cudaMemset(c->status_dev, 0, sizeof st);
+        return ENL_E_TIMEOUT;
+    }
+    return ENL_OK;
+}
+
+extern "C" int enl_group_store(enl_cache_t *c, int32_t group_id, int32_t layer, int32_t n_tokens, const void *k_dev,
+                               const void *v_dev, int32_t mode, void *cuda_stream)
+{
+    if (!c) return ENL_E_INVAL;
+    if (group_id < 0 || group_id >= c->d.max_groups) return ENL_E_NOGROUP;
+    if (layer < 0 || layer >= c->d.n_layers || n_tokens < 0) return ENL_E_INVAL;
+    if (mode != ENL_REPLACE && mode != ENL_APPEND) return ENL_E_INVAL;
+    if (c->gpu && n_tokens > 0) {
+        if (!k_dev || !v_dev) return ENL_E_INVAL;
+        if ((reinterpret_cast<uintptr_t>(k_dev) | reinterpret_cast<uintptr_t>(v_dev)) & 15) return ENL_E_INVAL;
+    }
+    Group &g = c->groups[group_id];
+    const int32_t old_len = g.len.empty() ? -1 : g.len[layer];
+    const int64_t new_len64 = (mode == ENL_APPEND && old_len > 0) ? static_cast<int64_t>(old_len) + n_tokens : n_tokens;
+    if (new_len64 > 0x3fffffff) return ENL_E_INVAL;
+    const int32_t new_len = static_cast<int32_t>(new_len64);
+    const int32_t first_pos = new_len - n_tokens;
+    const int need_pages = ceil_div(new_len, kPageTokens);
+    const int have = static_cast<int>(g.pages.size());
+    if (need_pages > have && static_cast<size_t>(need_pages - have) > c->free_pages.size()) return ENL_E_NOMEM;
+
+    // commit the table change
+    if (g.len.empty()) g.len.assign(c->d.n_layers, -1);
+    for (int i = have; i < need_pages; ++i) {
+        g.pages.push_back(c->free_pages.back());
+        c->free_pages.pop_back();
+    }
+    g.len[layer] = new_len;
+    int keep = 0;
+    for (int l = 0; l < c->d.n_layers; ++l) keep = std::max(keep, ceil_div(std::max(g.len[l], 0), kPageTokens));
+    while (static_cast<int>(g.pages.size()) > keep) {       // pages no layer needs any more
+        c->free_pages.push_back(g.pages.back());
+        g.pages.pop_back();
+    }
+    ++c->epoch;
+
+    if (!c->gpu || n_tokens == 0) return ENL_OK;
+    DeviceGuard dg(c->d.device);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const size_t row_bytes = static_cast<size_t>(c->d.n_kv_heads) * c->d.head_dim * 2;
+    int pos = first_pos;
+    while (pos < new_len) {
+        PageRun run;
+        run.first_page = pos / kPageTokens;
+        const int last_page = std::min((new_len - 1) / kPageTokens, run.first_page + kScatterPages - 1);
+        for (int i = run.first_page; i <= last_page; ++i) run.ids[i - run.first_page] = g.pages[i];
+        const int end = std::min(new_len, (last_page + 1) * kPageTokens);
+        const size_t src_off = static_cast<size_t>(pos - first_pos) * row_bytes;
+        if (launch_page_scatter(c->kpool + c->layer_bytes * layer, c->vpool + c->layer_bytes * layer,
+                                static_cast<const uint8_t *>(k_dev) + src_off,
+                                static_cast<const uint8_t *>(v_dev) + src_off, run, pos, end - pos,
+                                c->d.n_kv_heads, c->d.head_dim, st) != cudaSuccess) {
+            cudaGetLastError();
+            return ENL_E_CUDA;
+        }
+        pos = end;
+    }
+    return ENL_OK;
+}
+
+extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda_stream)
+{
+    if (!c || !a) return ENL_E_INVAL;
+    const enl_cache_desc_t &d = c->d;
+    const bool plan_only = (a->flags & ENL_PLAN_ONLY) != 0;
+    if (a->flags & ~static_cast<uint32_t>(ENL_PLAN_ONLY)) return ENL_E_INVAL;
+    if (!c->gpu && !plan_only) return ENL_E_CUDA;
+    if (a->layer < 0 || a->layer >= d.n_layers) return ENL_E_INVAL;
+    if (a->batch < 1 || a->batch > d.max_batch) return ENL_E_INVAL;
+    if (a->n_sel < 0 || a->n_q < 1 || a->n_new < a->n_q || a->n_q > d.max_q_tokens) return ENL_E_INVAL;
+    if (a->n_sel > 0 && !a->sel_ids) return ENL_E_INVAL;
+    if (a->split_hint < 0) return ENL_E_INVAL;
+    const int B = a->batch;
+    if (B > 1 && (!a->cu_sel || !a->cu_q || !a->cu_new)) return ENL_E_INVAL;
+    const int32_t one_sel[2] = {0, a->n_sel}, one_q[2] = {0, a->n_q}, one_new[2] = {0, a->n_new};
+    const int32_t *cu_sel = a->cu_sel ? a->cu_sel : one_sel;
+    const int32_t *cu_q = a->cu_q ? a->cu_q : one_q;
+    const int32_t *cu_new = a->cu_new ? a->cu_new : one_new;
+    if (cu_sel[0] != 0 || cu_q[0] != 0 || cu_new[0] != 0) return ENL_E_INVAL;
+    if (cu_sel[B] != a->n_sel || cu_q[B] != a->n_q || cu_new[B] != a->n_new) return ENL_E_INVAL;
+    int max_slots = 0;
+    for (int b = 0; b < B; ++b) {
+        const int ns = cu_sel[b + 1] - cu_sel[b], nq = cu_q[b + 1] - cu_q[b], nn = cu_new[b + 1] - cu_new[b];
+        if (ns < 0 || nq < 1 || nn < nq) return ENL_E_INVAL;
+        max_slots = std::max(max_slots, ns);
+    }
+    if (!plan_only) {
+        if (!a->q || !a->k_new || !a->v_new || !a->out) return ENL_E_INVAL;
+        const uintptr_t al = reinterpret_cast<uintptr_t>(a->q) | reinterpret_cast<uintptr_t>(a->k_new) |
+                             reinterpret_cast<uintptr_t>(a->v_new) | reinterpret_cast<uintptr_t>(a->out);
+        if (al & 15) return ENL_E_INVAL;
+        if (a->group_mass && (reinterpret_cast<uintptr_t>(a->group_mass) & 3)) return ENL_E_INVAL;
+    }
+    if (a->group_mass && a->mass_stride < max_slots + 1) return ENL_E_INVAL;
+
+    // ---- select list: ids, duplicates, lengths (Sec. 3.4: a group is selected at most once) ----
+    std::vector<int32_t> sel_len(a->n_sel);
+    for (int b = 0; b < B; ++b) {
+        if (++c->stamp == 0x7fffffff) { std::fill(c->seen.begin(), c->seen.end(), 0); c->stamp = 1; }
+        for (int s = cu_sel[b]; s < cu_sel[b + 1]; ++s) {
+            const int32_t gid = a->sel_ids[s];
+            if (gid < 0 || gid >= d.max_groups) return ENL_E_NOGROUP;
+            const Group &g = c->groups[gid];
+            if (g.len.empty() || g.len[a->layer] < 0) return ENL_E_NOGROUP;
+            if (c->seen[gid] == c->stamp) return ENL_E_INVAL;
+            c->seen[gid] = c->stamp;
+            sel_len[s] = g.len[a->layer];
+        }
+    }
+    if (a->sel_off_out) {
+        int32_t *o = a->sel_off_out;
+        for (int b = 0; b < B; ++b) {
+            int32_t acc = 0;
+            *o++ = 0;
+            for (int s = cu_sel[b]; s < cu_sel[b + 1]; ++s) { acc += sel_len[s]; *o++ = acc; }
+        }
+    }
+
+    // ---- gather plan: reuse when nothing it was built from has changed ----
+    std::vector<int32_t> cu_key;
+    cu_key.reserve(3 * (B + 1));
+    cu_key.insert(cu_key.end(), cu_sel, cu_sel + B + 1);
+    cu_key.insert(cu_key.end(), cu_q, cu_q + B + 1);
+    cu_key.insert(cu_key.end(), cu_new, cu_new + B + 1);
+    const bool has_mass = a->group_mass != nullptr;
+    const bool reuse = c->plan_valid && c->plan_epoch == c->epoch && c->plan_split_hint == a->split_hint &&
+                       c->plan_has_mass == has_mass && c->key_cu == cu_key && c->key_len == sel_len &&
+                       c->key_sel.size() == static_cast<size_t>(a->n_sel) &&
+                       (a->n_sel == 0 || std::memcmp(c->key_sel.data(), a->sel_ids, sizeof(int32_t) * a->n_sel) == 0);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    DeviceGuard dg(c->gpu ? d.device : -1);
+
+    if (!reuse) {
+        // size check first, so that a failed call leaves the previous plan intact
+        const int tpc = tokens_per_cta(c);
+        int64_t n_entries = 0, base_items = 0;
+        int min_tiles = 0x7fffffff;
+        for (int b = 0; b < B; ++b) {
+            int64_t e = 0;
+            for (int s = cu_sel[b]; s < cu_sel[b + 1]; ++s) e += std::max(1, ceil_div(sel_len[s], kPageTokens));
+            e = (e + kPagesPerTile - 1) / kPagesPerTile * kPagesPerTile;
+            n_entries += e;
+            const int nq = cu_q[b + 1] - cu_q[b], nn = cu_new[b + 1] - cu_new[b];
+            base_items += static_cast<int64_t>(ceil_div(nq, tpc)) * d.n_kv_heads;
+            // fewest tiles any CTA of this episode walks: its first token block
+            const int c_first = nn - nq + std::min(tpc, nq) - 1;
+            min_tiles = std::min<int64_t>(min_tiles, e / kPagesPerTile + c_first / kTileKeys + 1);
+        }
+        if (n_entries > c->cap_entries || base_items > c->cap_items) return ENL_E_NOMEM;
+
+        int n_splits = 1;
+        if (a->split_hint >= 1) n_splits = a->split_hint;
+        else if (base_items < 120) n_splits = std::max(1, std::min(static_cast<int>(148 / base_items), min_tiles / 2));
+        n_splits = std::min<int64_t>(n_splits, std::max<int64_t>(1, c->cap_items / base_items));
+        n_splits = std::min(n_splits, 64);
+        const int slot_stride = max_slots + 1;
+        while (n_splits > 1) {
+            const int64_t per_rh = d.head_dim + 1 + (has_mass ? slot_stride : 0);
+            if (static_cast<int64_t>(n_splits) * a->n_q * d.n_q_heads * per_rh * 4 <= d.scratch_bytes) break;
+            --n_splits;
+        }
+
+        if (c->gpu && cudaEventSynchronize(c->plan_copied) != cudaSuccess) { cudaGetLastError(); return ENL_E_CUDA; }
+        c->plan_valid = false;
+        EpInfo *eps = c->h_eps();
+        int2 *stream = c->h_stream();
+        int32_t *rowslots = c->h_rowslots();
+        int32_t ne = 0;
+        for (int b = 0; b < B; ++b) {
+            EpInfo &e = eps[b];
+            e.stream_off = ne;
+            e.n_slots = cu_sel[b + 1] - cu_sel[b];
+            e.q_off = cu_q[b];
+            e.n_q = cu_q[b + 1] - cu_q[b];
+            e.new_off = cu_new[b];
+            e.n_new = cu_new[b + 1] - cu_new[b];
+            e.pad = 0;
+            for (int s = cu_sel[b]; s < cu_sel[b + 1]; ++s) {
+                const int slot = s - cu_sel[b];
+                const Group &g = c->groups[a->sel_ids[s]];
+                const int len = sel_len[s], np = ceil_div(len, kPageTokens);
+                if (np == 0) stream[ne++] = make_int2(kZeroPage, slot << 8);
+                for (int i = 0; i < np; ++i) {
+                    const int nv = std::min(kPageTokens, len - i * kPageTokens);
+                    stream[ne++] = make_int2(g.pages[i], (slot << 8) | nv);
+                }
+            }
+            while ((ne - e.stream_off) % kPagesPerTile) stream[ne++] = make_int2(kZeroPage, (e.n_slots - 1) << 8);
+            e.n_ctiles = (ne - e.stream_off) / kPagesPerTile;
+            for (int r = e.q_off; r < e.q_off + e.n_q; ++r) rowslots[r] = e.n_slots;
+        }
+        // CTAs, heaviest first (late token blocks see more new-token tiles)
+        struct Work { Item it; int tiles; };
+        std::vector<Work> work;
+        work.reserve(static_cast<size_t>(base_items) * n_splits);
+        for (int b = 0; b < B; ++b) {
+            const EpInfo &e = eps[b];
+            for (int t0 = 0; t0 < e.n_q; t0 += tpc) {
+                const int t_hi = std::min(t0 + tpc, e.n_q);
+                const int tiles = e.n_ctiles + (e.n_new - e.n_q + t_hi - 1) / kTileKeys + 1;
+                for (int h = 0; h < d.n_kv_heads; ++h)
+                    for (int sp = 0; sp < n_splits; ++sp) work.push_back({Item{b, h, t0, sp}, tiles});
+            }
+        }
+        std::stable_sort(work.begin(), work.end(), [](const Work &x, const Work &y) { return x.tiles > y.tiles; });
+        Item *items = c->h_items();
+        for (size_t i = 0; i < work.size(); ++i) items[i] = work[i].it;
+
+        c->plan_entries = ne;
+        c->plan_items = static_cast<int32_t>(work.size());
+        c->plan_splits = n_splits;
+        c->plan_batch = B;
+        c->plan_max_slots = max_slots;
+        c->plan_epoch = c->epoch;
+        c->plan_split_hint = a->split_hint;
+        c->plan_has_mass = has_mass;
+        c->key_sel.assign(a->sel_ids, a->sel_ids + a->n_sel);
+        c->key_cu = cu_key;
+        c->key_len = sel_len;
+        c->plan_valid = true;
+        c->plan_on_device = false;
+    }
+    if (plan_only) return ENL_OK;
+
+    if (!c->plan_on_device) {
+        // one copy covers episodes, items, stream and row->slots (unused gaps travel too; they are small)
+        const size_t used_stream = c->off_stream + sizeof(int2) * c->plan_entries;
+        bool okc = cudaMemcpyAsync(c->plan_dev, c->plan_host, c->off_stream, cudaMemcpyHostToDevice, st) == cudaSuccess &&
+                   cudaMemcpyAsync(c->plan_dev + c->off_stream, c->plan_host + c->off_stream, used_stream - c->off_stream,
+                                   cudaMemcpyHostToDevice, st) == cudaSuccess &&
+                   cudaMemcpyAsync(c->plan_dev + c->off_rowslots, c->plan_host + c->off_rowslots,
+                                   sizeof(int32_t) * a->n_q, cudaMemcpyHostToDevice, st) == cudaSuccess &&
+                   cudaEventRecord(c->plan_copied, st) == cudaSuccess;
+        if (!okc) { cudaGetLastError(); c->plan_valid = false; return ENL_E_CUDA; }
+        c->plan_on_device = true;
+    }
+
+    AttnParams p;
+    std::memset(&p, 0, sizeof p);
+    {
+        const cuuint64_t qd[3] = {static_cast<cuuint64_t>(d.head_dim), static_cast<cuuint64_t>(d.n_q_heads),
+                                  static_cast<cuuint64_t>(a->n_q)};
+        const cuuint64_t qs[2] = {static_cast<cuuint64_t>(d.head_dim) * 2,
+                                  static_cast<cuuint64_t>(d.head_dim) * 2 * d.n_q_heads};
+        const cuuint32_t qb[3] = {64, static_cast<cuuint32_t>(c->rep), static_cast<cuuint32_t>(kTileRows / c->rep)};
+        const cuuint64_t nd[3] = {static_cast<cuuint64_t>(d.head_dim), static_cast<cuuint64_t>(d.n_kv_heads),
+                                  static_cast<cuuint64_t>(a->n_new)};
+        const cuuint64_t ns[2] = {static_cast<cuuint64_t>(d.head_dim) * 2,
+                                  static_cast<cuuint64_t>(d.head_dim) * 2 * d.n_kv_heads};
+        const cuuint32_t nb[3] = {64, 1, kTileKeys};
+        if (!encode_map(&p.tm_q, a->q, 3, qd, qs, qb) || !encode_map(&p.tm_knew, a->k_new, 3, nd, ns, nb) ||
+            !encode_map(&p.tm_vnew, a->v_new, 3, nd, ns, nb))
+            return ENL_E_CUDA;
+    }
+    p.tm_kpool = c->tm_k[a->layer];
+    p.tm_vpool = c->tm_v[a->layer];
+    p.items = reinterpret_cast<const Item *>(c->plan_dev + c->off_items);
+    p.eps = reinterpret_cast<const EpInfo *>(c->plan_dev + c->off_eps);
+    p.stream = reinterpret_cast<const int2 *>(c->plan_dev + c->off_stream);
+    p.out = a->out;
+    p.mass = a->group_mass;
+    p.status = c->status_dev;
+    p.n_q_total = a->n_q;
+    p.Hq = d.n_q_heads;
+    p.Hkv = d.n_kv_heads;
+    p.rep = c->rep;
+    p.mass_stride = a->mass_stride;
+    p.n_splits = c->plan_splits;
+    p.scale_log2 = 1.4426950408889634f / sqrtf(static_cast<float>(d.head_dim));
+    const int slot_stride = c->plan_max_slots + 1;
+    if (p.n_splits > 1) {
+        const size_t rows = static_cast<size_t>(p.n_splits) * a->n_q * d.n_q_heads;
+        p.part_o = c->scratch;
+        p.part_lse = c->scratch + rows * d.head_dim;
+        p.part_slot = has_mass ? c->scratch + rows * (d.head_dim + 1) : nullptr;
+        p.mass_stride = slot_stride;                 // the partial slot buffer is packed
+    }
+    if (launch_attention(p, d.head_dim, c->plan_items, st) != cudaSuccess) { cudaGetLastError(); return ENL_E_CUDA; }
+    if (p.n_splits > 1) {
+        CombineParams cp;
+        cp.part_o = p.part_o;
+        cp.part_lse = p.part_lse;
+        cp.part_slot = p.part_slot;
+        cp.out = a->out;
+        cp.mass = a->group_mass;
+        cp.row_slots = reinterpret_cast<const int32_t *>(c->plan_dev + c->off_rowslots);
+        cp.n_q_total = a->n_q;
+        cp.Hq = d.n_q_heads;
+        cp.D = d.head_dim;
+        cp.slot_stride = slot_stride;
+        cp.mass_stride = a->mass_stride;
+        cp.n_splits = p.n_splits;
+        if (launch_combine(cp, st) != cudaSuccess) { cudaGetLastError(); return ENL_E_CUDA; }
+    }
+    return ENL_OK;
+}
+
+extern "C" int enl_plan_inspect(const enl_cache_t *cc, int32_t cap_entries, int32_t *stream_pages, int32_t *stream_meta,
+                                int32_t *n_entries, int32_t cap_batch, int32_t *ep_stream_off,
+                                int32_t *ep_cached_tiles, int32_t *n_splits, int32_t *n_items)
+{
+    enl_cache *c = const_cast<enl_cache *>(cc);
+    if (!c || !c->plan_valid) return ENL_E_INVAL;
+    if (n_entries) *n_entries = c->plan_entries;
+    if (n_splits) *n_splits = c->plan_splits;
+    if (n_items) *n_items = c->plan_items;
+    const int2 *s = c->h_stream();
+    for (int i = 0; i < c->plan_entries && i < cap_entries; ++i) {
+        if (stream_pages) stream_pages[i] = s[i].x;
+        if (stream_meta) stream_meta[i] = s[i].y;
+    }
+    const EpInfo *e = c->h_eps();
+    for (int b = 0; b < c->plan_batch && b < cap_batch; ++b) {
+        if (ep_stream_off) ep_stream_off[b] = e[b].stream_off;
+        if (ep_cached_tiles) ep_cached_tiles[b] = e[b].n_ctiles;
+    }
+    return ENL_OK;
+}

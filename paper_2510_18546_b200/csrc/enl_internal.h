@@ -1,0 +1,85 @@
+// Internal declarations shared by the host side and the kernels of the library.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace enl {
+
+constexpr int kPageTokens = 16;     // tokens per page: one TMA box of 16 rows x 128 B per 64 channels
+constexpr int kTileKeys   = 128;    // keys per KV tile (8 pages)
+constexpr int kPagesPerTile = kTileKeys / kPageTokens;
+constexpr int kTileRows   = 128;    // query rows per Q tile = (128 / rep) tokens x rep q heads of one kv head
+constexpr int kQTiles     = 2;      // Q tiles per CTA (they share every K/V tile the CTA loads)
+constexpr int kZeroPage   = 0;      // page 0 is never handed out: all zeros, target of null stream entries
+
+// One episode of an attend call.
+struct EpInfo {
+    int32_t stream_off;     // first KV-stream entry (multiple of kPagesPerTile)
+    int32_t n_ctiles;       // cached tiles (128 keys each, last one padded with null entries)
+    int32_t n_slots;        // selected groups G_b; mass slot G_b = new tokens
+    int32_t q_off, n_q;     // first query row (global) and count
+    int32_t new_off, n_new; // first new-token key (global) and count
+    int32_t pad;
+};
+
+// One CTA of the attention launch.
+struct Item {
+    int32_t ep;             // episode
+    int32_t kvh;            // kv head
+    int32_t t0;             // first query token (episode-relative) of the CTA's two Q tiles
+    int32_t split;          // KV split index in [0, n_splits)
+};
+
+// Kernel parameters (passed by value as a __grid_constant__).
+struct AttnParams {
+    CUtensorMap tm_q;       // [n_q][Hq][D]      box {64, rep, 128/rep}
+    CUtensorMap tm_knew;    // [n_new][Hkv][D]   box {64, 1, 128}
+    CUtensorMap tm_vnew;
+    CUtensorMap tm_kpool;   // [pages*Hkv*16][D] box {64, 16}   (one layer)
+    CUtensorMap tm_vpool;
+    const Item   *items;
+    const EpInfo *eps;
+    const int2   *stream;   // {page id, slot << 8 | valid tokens}
+    void   *out;            // bf16 [n_q][Hq][D]
+    float  *mass;           // fp32 or null
+    float  *part_o;         // split mode: [split][row][Hq][D] fp32 (normalised by the split's own sum)
+    float  *part_lse;       // split mode: [split][row][Hq] log2-sum-exp of the split
+    float  *part_slot;      // split mode: [split][row][Hq][mass_stride] per-slot log2-sum-exp
+    int32_t *status;        // device word: nonzero = a bounded wait expired
+    int32_t n_q_total;      // rows over the batch
+    int32_t Hq, Hkv, rep;   // rep = Hq / Hkv
+    int32_t mass_stride;
+    int32_t n_splits;
+    float   scale_log2;     // log2(e) / sqrt(D)
+};
+
+struct CombineParams {
+    const float *part_o, *part_lse, *part_slot;
+    void  *out;
+    float *mass;
+    const int32_t *row_slots;   // [n_q_total]: G_b of the row's episode
+    int32_t n_q_total, Hq, D;
+    int32_t slot_stride;        // row stride of part_slot
+    int32_t mass_stride;        // row stride of mass
+    int32_t n_splits;
+};
+
+// launchers (defined in the .cu files of the kernels)
+cudaError_t launch_attention(const AttnParams &p, int head_dim, int n_items, cudaStream_t st);
+cudaError_t launch_combine(const CombineParams &p, cudaStream_t st);
+// Page ids of (part of) one group, passed by value to the scatter kernel.
+constexpr int kScatterPages = 64;
+struct PageRun {
+    int32_t ids[kScatterPages];   // ids[i] = page holding group positions (first_page + i)*16 ..
+    int32_t first_page;           // index within the group of ids[0]
+};
+cudaError_t launch_page_scatter(void *kpool_layer, void *vpool_layer, const void *k, const void *v,
+                                const PageRun &run, int first_pos, int n_tokens,
+                                int Hkv, int D, cudaStream_t st);
+size_t attention_smem_bytes(int head_dim);
+// Opts the attention kernel into its dynamic shared memory size on the current device.
+cudaError_t prepare_attention(int head_dim);
+
+}  // namespace enl

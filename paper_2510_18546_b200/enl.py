@@ -1,0 +1,172 @@
+"""Thin ctypes binding over ``libenl.so``: same names as the C ABI, argument marshalling only.
+
+Every step of the path (page scatter, gather plan upload, attention, split merge) runs inside the
+library; nothing here computes.  There is no fallback: if the library is missing, loading raises.
+Tensors are torch CUDA tensors (device memory and streams are torch's); index lists are host arrays.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libenl.so")
+
+ENL_BF16 = 1
+ENL_DEVICE_NONE = -1
+ENL_REPLACE, ENL_APPEND = 0, 1
+ENL_PLAN_ONLY = 1
+ENL_OK, ENL_E_INVAL, ENL_E_NOGROUP, ENL_E_NOMEM, ENL_E_CUDA, ENL_E_TIMEOUT = 0, -1, -2, -3, -4, -5
+
+EXPORTS = ("enl_cache_create", "enl_group_store", "enl_attend", "enl_cache_free", "enl_strerror",
+           "enl_group_len", "enl_cache_status", "enl_plan_inspect")
+
+
+class CacheDesc(ctypes.Structure):
+    _fields_ = [("n_layers", ctypes.c_int32), ("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
+                ("head_dim", ctypes.c_int32), ("page_tokens", ctypes.c_int32), ("max_groups", ctypes.c_int32),
+                ("max_tokens", ctypes.c_int64), ("dtype", ctypes.c_int32), ("device", ctypes.c_int32),
+                ("max_batch", ctypes.c_int32), ("max_q_tokens", ctypes.c_int32), ("scratch_bytes", ctypes.c_int64)]
+
+
+class AttendArgs(ctypes.Structure):
+    _fields_ = [("layer", ctypes.c_int32), ("batch", ctypes.c_int32),
+                ("sel_ids", ctypes.c_void_p), ("cu_sel", ctypes.c_void_p), ("cu_q", ctypes.c_void_p),
+                ("cu_new", ctypes.c_void_p),
+                ("n_sel", ctypes.c_int32), ("n_q", ctypes.c_int32), ("n_new", ctypes.c_int32),
+                ("q", ctypes.c_void_p), ("k_new", ctypes.c_void_p), ("v_new", ctypes.c_void_p),
+                ("out", ctypes.c_void_p), ("group_mass", ctypes.c_void_p), ("mass_stride", ctypes.c_int32),
+                ("sel_off_out", ctypes.c_void_p), ("split_hint", ctypes.c_int32), ("flags", ctypes.c_uint32)]
+
+
+class EnlError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__(f"{what}: {strerror(code)} ({code})")
+        self.code = code
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads the library (raises OSError if it has not been built: there is no other path)."""
+    global _lib
+    if _lib is None:
+        L = ctypes.CDLL(LIB_PATH)
+        L.enl_cache_create.argtypes = [ctypes.POINTER(CacheDesc), ctypes.POINTER(ctypes.c_void_p)]
+        L.enl_cache_create.restype = ctypes.c_int
+        L.enl_group_store.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
+                                      ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p]
+        L.enl_group_store.restype = ctypes.c_int
+        L.enl_attend.argtypes = [ctypes.c_void_p, ctypes.POINTER(AttendArgs), ctypes.c_void_p]
+        L.enl_attend.restype = ctypes.c_int
+        L.enl_cache_free.argtypes = [ctypes.c_void_p]
+        L.enl_cache_free.restype = ctypes.c_int
+        L.enl_strerror.argtypes = [ctypes.c_int]
+        L.enl_strerror.restype = ctypes.c_char_p
+        L.enl_group_len.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32]
+        L.enl_group_len.restype = ctypes.c_int32
+        L.enl_cache_status.argtypes = [ctypes.c_void_p]
+        L.enl_cache_status.restype = ctypes.c_int
+        L.enl_plan_inspect.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p,
+                                       ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p,
+                                       ctypes.c_void_p, ctypes.c_void_p]
+        L.enl_plan_inspect.restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+def strerror(code: int) -> str:
+    return lib().enl_strerror(int(code)).decode()
+
+
+def _ptr(t) -> Optional[int]:
+    return None if t is None else int(t.data_ptr())
+
+
+def _i32(a) -> Optional[np.ndarray]:
+    return None if a is None else np.ascontiguousarray(np.asarray(a, dtype=np.int32))
+
+
+def _np_ptr(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def enl_cache_create(n_layers: int, n_q_heads: int, n_kv_heads: int, head_dim: int, max_groups: int,
+                     max_tokens: int, device: int = 0, max_batch: int = 0, max_q_tokens: int = 0,
+                     scratch_bytes: int = 0, page_tokens: int = 0, dtype: int = ENL_BF16) -> int:
+    """Returns the opaque cache handle."""
+    d = CacheDesc(n_layers, n_q_heads, n_kv_heads, head_dim, page_tokens, max_groups, max_tokens, dtype,
+                  device, max_batch, max_q_tokens, scratch_bytes)
+    h = ctypes.c_void_p()
+    rc = lib().enl_cache_create(ctypes.byref(d), ctypes.byref(h))
+    if rc != ENL_OK:
+        raise EnlError(rc, "enl_cache_create")
+    return h.value
+
+
+def enl_group_store(cache: int, group_id: int, layer: int, k, v, mode: int = ENL_REPLACE,
+                    stream: int = 0, n_tokens: Optional[int] = None) -> None:
+    """``k``/``v``: ``[n, Hkv, D]`` bf16 CUDA tensors (or None with ``n_tokens`` on a bookkeeping cache)."""
+    n = int(k.shape[0]) if k is not None else int(n_tokens)
+    rc = lib().enl_group_store(cache, group_id, layer, n, _ptr(k), _ptr(v), mode, stream or None)
+    if rc != ENL_OK:
+        raise EnlError(rc, "enl_group_store")
+
+
+def enl_attend(cache: int, layer: int, sel_ids: Sequence[int], q, k_new, v_new, out, group_mass=None,
+               cu_sel=None, cu_q=None, cu_new=None, n_q: Optional[int] = None, n_new: Optional[int] = None,
+               mass_stride: Optional[int] = None, want_sel_off: bool = False, split_hint: int = 0,
+               flags: int = 0, stream: int = 0):
+    """One attend call.  Returns ``sel_off`` (numpy int32 ``[n_sel + batch]``) when asked, else None."""
+    sel = _i32(sel_ids)
+    cs, cq, cn = _i32(cu_sel), _i32(cu_q), _i32(cu_new)
+    batch = 1 if cq is None else len(cq) - 1
+    nq = int(n_q) if n_q is not None else int(q.shape[0])
+    nn = int(n_new) if n_new is not None else int(k_new.shape[0])
+    so = np.zeros(len(sel) + batch, np.int32) if want_sel_off else None
+    a = AttendArgs()
+    a.layer, a.batch = layer, batch
+    a.sel_ids, a.cu_sel, a.cu_q, a.cu_new = _np_ptr(sel), _np_ptr(cs), _np_ptr(cq), _np_ptr(cn)
+    a.n_sel, a.n_q, a.n_new = len(sel), nq, nn
+    a.q, a.k_new, a.v_new, a.out = _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out)
+    a.group_mass = _ptr(group_mass)
+    a.mass_stride = int(mass_stride) if mass_stride is not None else (
+        int(group_mass.shape[-1]) if group_mass is not None else 0)
+    a.sel_off_out = _np_ptr(so)
+    a.split_hint, a.flags = split_hint, flags
+    rc = lib().enl_attend(cache, ctypes.byref(a), stream or None)
+    if rc != ENL_OK:
+        raise EnlError(rc, "enl_attend")
+    return so
+
+
+def enl_cache_free(cache: int) -> None:
+    lib().enl_cache_free(cache)
+
+
+def enl_group_len(cache: int, group_id: int, layer: int) -> int:
+    return int(lib().enl_group_len(cache, group_id, layer))
+
+
+def enl_cache_status(cache: int) -> int:
+    return int(lib().enl_cache_status(cache))
+
+
+def enl_plan_inspect(cache: int, cap_entries: int = 1 << 16, cap_batch: int = 256):
+    """Host copy of the last gather plan: dict with stream pages/meta, per-episode offsets, splits, items."""
+    pages = np.zeros(cap_entries, np.int32)
+    meta = np.zeros(cap_entries, np.int32)
+    off = np.zeros(cap_batch, np.int32)
+    tiles = np.zeros(cap_batch, np.int32)
+    ne, ns, ni = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32()
+    rc = lib().enl_plan_inspect(cache, cap_entries, _np_ptr(pages), _np_ptr(meta), ctypes.byref(ne), cap_batch,
+                                _np_ptr(off), _np_ptr(tiles), ctypes.byref(ns), ctypes.byref(ni))
+    if rc != ENL_OK:
+        raise EnlError(rc, "enl_plan_inspect")
+    n = min(ne.value, cap_entries)
+    return dict(pages=pages[:n], meta=meta[:n], n_entries=ne.value, ep_stream_off=off, ep_cached_tiles=tiles,
+                n_splits=ns.value, n_items=ni.value)

@@ -1,0 +1,108 @@
+"""GPU parity, small shapes: the CUDA library (through the C ABI) against the float64 oracle,
+element by element, on sizes that span several tiles and ragged tails."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2510_18546_b200 import enl, synth
+from tests.helpers import Session, check_close
+
+pytestmark = pytest.mark.gpu
+
+
+def run_case(wl, split_hint=0, layer=0):
+    with Session(wl, [layer]) as s:
+        q, kn, vn = wl.new_qkv(layer, s.device)
+        out, mass, sel_off = s.attend(0, q, kn, vn, split_hint=split_hint)
+        torch.cuda.synchronize()
+        assert enl.enl_cache_status(s.cache) == enl.ENL_OK
+        cs, cq, cn = wl.cu()
+        so = 0
+        for b in range(wl.batch):
+            qo, mo, off = s.oracle(0, b, q[cq[b]:cq[b + 1]], kn[cn[b]:cn[b + 1]], vn[cn[b]:cn[b + 1]])
+            G = len(wl.sel_local[b])
+            check_close(out[cq[b]:cq[b + 1]], qo, mass[cq[b]:cq[b + 1], :, :G + 1], mo,
+                        what=f"{wl.name} ep{b} split{split_hint}")
+            assert list(sel_off[so:so + G + 1]) == [int(x) for x in off]      # bit-exact book-keeping
+            so += G + 1
+            rs = mass[cq[b]:cq[b + 1], :, :G + 1].sum(-1)
+            assert (rs - 1).abs().max().item() < 1e-3
+
+
+def test_tiny_config():
+    run_case(synth.make("tiny"))
+
+
+@pytest.mark.parametrize("split", [2, 3])
+def test_tiny_config_kv_split(split):
+    run_case(synth.make("tiny"), split_hint=split)
+
+
+SMALL = {
+    # ragged groups, several tiles, rows not a multiple of the CTA's 64 tokens
+    "ragged_d128": dict(Hq=8, Hkv=2, D=128, pool=[[1, 50, 16, 33, 7, 120, 15, 17]], sel=[[5, 0, 3, 7, 1]],
+                        n_q=[77], n_new=[77]),
+    "ragged_d64": dict(Hq=8, Hkv=2, D=64, pool=[[9, 31, 64, 2]], sel=[[3, 2, 1, 0]], n_q=[130], n_new=[130]),
+    # queries aligned with the LAST new keys (chunked prefill / multi-token decode)
+    "nq_lt_nnew": dict(Hq=8, Hkv=2, D=128, pool=[[40, 41, 42]], sel=[[2, 0]], n_q=[5], n_new=[200]),
+    "empty_select": dict(Hq=4, Hkv=1, D=128, pool=[[10]], sel=[[]], n_q=[150], n_new=[150]),
+    "one_decode_token": dict(Hq=32, Hkv=8, D=128, pool=[[300, 17, 256]], sel=[[0, 1, 2]], n_q=[1], n_new=[1]),
+    "decode_grown": dict(Hq=32, Hkv=8, D=128, pool=[[300, 17, 256]], sel=[[2, 0]], n_q=[1], n_new=[37]),
+    "rep1": dict(Hq=2, Hkv=2, D=64, pool=[[20, 20]], sel=[[1, 0]], n_q=[140], n_new=[140]),
+    "rep8": dict(Hq=8, Hkv=1, D=128, pool=[[20, 45]], sel=[[0, 1]], n_q=[40], n_new=[40]),
+    "varlen_batch": dict(Hq=8, Hkv=2, D=128, pool=[[30, 60, 90], [5, 5, 5, 5], [200]],
+                         sel=[[2, 0], [0, 1, 2, 3], []], n_q=[70, 3, 129], n_new=[70, 10, 129]),
+}
+
+
+@pytest.mark.parametrize("name", sorted(SMALL))
+@pytest.mark.parametrize("split", [0, 2])
+def test_small_shapes(name, split):
+    c = SMALL[name]
+    wl = synth.make_small(7, 1, c["Hq"], c["Hkv"], c["D"], c["pool"], c["sel"], c["n_q"], c["n_new"], name=name)
+    run_case(wl, split_hint=split)
+
+
+def test_zero_length_group_has_zero_mass():
+    wl = synth.make_small(8, 1, 8, 2, 64, [[12, 0, 20]], [[0, 1, 2]], [33], [33], name="zero_len")
+    with Session(wl, [0]) as s:
+        q, kn, vn = wl.new_qkv(0, s.device)
+        out, mass, sel_off = s.attend(0, q, kn, vn)
+        torch.cuda.synchronize()
+        assert list(sel_off) == [0, 12, 12, 32]
+        assert mass[:, :, 1].abs().max().item() == 0.0
+        qo, mo, _ = s.oracle(0, 0, q, kn, vn)
+        check_close(out, qo, mass, mo, what="zero_len")
+
+
+def test_select_order_permutes_mass_only():
+    wl = synth.make_small(9, 1, 8, 2, 128, [[33, 70, 18, 5]], [[0, 1, 2, 3]], [64], [64], name="perm")
+    with Session(wl, [0]) as s:
+        q, kn, vn = wl.new_qkv(0, s.device)
+        o1, m1, _ = s.attend(0, q, kn, vn)
+        perm = [2, 0, 3, 1]
+        o2, m2, off2 = s.attend(0, q, kn, vn, sel_override=perm)
+        torch.cuda.synchronize()
+        assert list(off2) == [0, 18, 51, 56, 126]
+        assert (o1.float() - o2.float()).abs().max().item() <= 2e-2
+        assert (m1[..., perm] - m2[..., :4]).abs().max().item() <= 1e-3
+        assert (m1[..., 4] - m2[..., 4]).abs().max().item() <= 1e-3
+
+
+def test_append_keeps_existing_rows():
+    """Sec. 3.2: rows appended at the end of a group; a later attend sees old + new rows in order."""
+    wl = synth.make_small(10, 1, 8, 2, 128, [[45, 30]], [[0, 1]], [20], [20], name="append")
+    with Session(wl, [0], extra_tokens=64) as s:
+        g = torch.Generator(device=s.device).manual_seed(3)
+        ka = (torch.randn(21, 2, 128, generator=g, device=s.device)).to(torch.bfloat16)
+        va = (torch.randn(21, 2, 128, generator=g, device=s.device)).to(torch.bfloat16)
+        enl.enl_group_store(s.cache, 0, 0, ka, va, mode=enl.ENL_APPEND)
+        assert enl.enl_group_len(s.cache, 0, 0) == 66
+        ks, vs = s.host_kv[(0, 0)]
+        s.host_kv[(0, 0)] = ([torch.cat([ks[0], ka.cpu()]), ks[1]], [torch.cat([vs[0], va.cpu()]), vs[1]])
+        q, kn, vn = wl.new_qkv(0, s.device)
+        out, mass, sel_off = s.attend(0, q, kn, vn)
+        torch.cuda.synchronize()
+        assert list(sel_off) == [0, 66, 96]
+        qo, mo, _ = s.oracle(0, 0, q, kn, vn)
+        check_close(out, qo, mass, mo, what="append")
