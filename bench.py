@@ -1,0 +1,404 @@
+#!/usr/bin/env python
+"""Benchmark of the selective-KV attention hot path.
+
+A "step" is one planning step of the workload: for every layer one group store (the K/V of one
+group rewritten in place, Sec. 3.2), the gather plan (built at the first layer, reused by the
+others), and one `enl_attend` per layer (attention + fused per-group mass, plus the split merge
+when KV splits are used).  Layers run sequentially on one stream, as in the planner.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload planner|long|long_scoring|concurrent|decode|tiny]
+    python bench.py --impl reference      # the float64 CPU oracle, timed on the host cores
+
+Prints ONE JSON line.  `value` is algorithmic TFLOP/s for prefill workloads (QK^T and PV, causal half
+counted once, padding and masked work not credited) and algorithmic GB/s for the decode workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+# dram__bytes_read.sum + dram__bytes_write.sum per attention launch from the ncu capture summarised in
+# profiles/ (same kernel, same workload shape); None until a capture exists for the workload.
+NCU_TRAFFIC_BYTES = {}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        d["_source"] = "measured"
+        return d
+    d = dict(FALLBACK_PEAKS)
+    d["_source"] = "fallback"
+    return d
+
+
+# ---- algorithmic work ---------------------------------------------------------------------------
+def prefill_flops_per_layer(wl) -> float:
+    f = 0.0
+    for b in range(wl.batch):
+        S, tn, nn = wl.selected_tokens(b), wl.n_q[b], wl.n_new[b]
+        vis_new = tn * (nn - tn) + tn * (tn + 1) / 2.0
+        f += 4.0 * wl.n_q_heads * wl.head_dim * (tn * S + vis_new)
+    return f
+
+
+def kv_bytes_per_token(wl) -> int:
+    return 2 * wl.n_kv_heads * wl.head_dim * 2
+
+
+def prefill_bytes_per_layer(wl) -> float:
+    by = 0.0
+    for b in range(wl.batch):
+        S, tn, nn, G = wl.selected_tokens(b), wl.n_q[b], wl.n_new[b], len(wl.sel_local[b])
+        by += (S + nn) * kv_bytes_per_token(wl) + 2 * tn * wl.n_q_heads * wl.head_dim * 2 + 4 * tn * wl.n_q_heads * (G + 1)
+    return by
+
+
+def decode_bytes_per_layer(wl, t: int) -> float:
+    return (wl.selected_tokens(0) + t + 1) * kv_bytes_per_token(wl)
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self._stop, self._t = index, [], threading.Event(), None
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                o = subprocess.run(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                                    "-i", str(self.index)], capture_output=True, text=True, timeout=5).stdout.strip()
+                if o:
+                    self.rows.append([x.strip() for x in o.splitlines()[0].split(",")])
+            except Exception:
+                pass
+            self._stop.wait(0.1)
+
+    def __enter__(self):
+        self._t = threading.Thread(target=self._run, daemon=True)
+        self._t.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        self._t.join(timeout=10)
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except Exception:
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ---- the oracle arm (also the cpu_baseline leg) -------------------------------------------------
+def oracle_sample(wl, seconds_target: float = 12.0):
+    """Times the float64 oracle, as it stands, on a bounded sample of the workload: layer 0, episode 0,
+    all q heads, as many query rows as fit the time target.  Returns (value in the metric's unit, dict)."""
+    from oracle import enl_oracle as orc
+    b, layer = 0, 0
+    k, v = wl.pool_kv(layer, b, "cpu")
+    offs = wl.pool_offsets(b)
+    ks = [k[offs[g]:offs[g + 1]] for g in wl.sel_local[b]]
+    vs = [v[offs[g]:offs[g + 1]] for g in wl.sel_local[b]]
+    q, kn, vn = wl.new_qkv(layer, "cpu")
+    S = wl.selected_tokens(b)
+    if wl.decode_steps:
+        t = wl.decode_steps - 1
+        q, kn, vn = q[t:t + 1], kn[:t + 1], vn[:t + 1]
+        rows = [0]
+    else:
+        q, kn, vn = q[:wl.n_q[b]], kn[:wl.n_new[b]], vn[:wl.n_new[b]]
+        rows = None
+    # calibrate on a few rows, then size the sample
+    n_q, n_new = q.shape[0], kn.shape[0]
+    probe = [n_q - 1] if rows is None else rows
+    t0 = time.perf_counter()
+    orc.attend_slots(wl.n_q_heads, wl.n_kv_heads, wl.head_dim, ks, vs, q, kn, vn, rows=probe)
+    dt_probe = time.perf_counter() - t0
+    if rows is None:
+        n = int(max(1, min(n_q, seconds_target / max(dt_probe, 1e-4))))
+        rows = sorted(set(np.linspace(0, n_q - 1, n).astype(int).tolist()))
+    t0 = time.perf_counter()
+    orc.attend_slots(wl.n_q_heads, wl.n_kv_heads, wl.head_dim, ks, vs, q, kn, vn, rows=rows)
+    dt = time.perf_counter() - t0
+    if wl.decode_steps:
+        work = decode_bytes_per_layer(wl, wl.decode_steps - 1)
+        value, unit = work / dt / 1e9, "GB/s"
+    else:
+        work = sum(4.0 * wl.n_q_heads * wl.head_dim * (S + (n_new - n_q) + r + 1) for r in rows)
+        value, unit = work / dt / 1e12, "TFLOP/s"
+    info = {"value": value, "unit": unit, "cores": orc.threads(), "kind": "oracle",
+            "sample": f"layer 0, episode 0, {len(rows)} of {n_q} query rows x {wl.n_q_heads} heads, "
+                      f"{S} cached + {n_new} new keys, {dt:.2f} s"}
+    return value, unit, dt, info
+
+
+def run_reference(args, wl, rank):
+    if rank != 0:
+        return
+    times = []
+    info = None
+    for i in range(args.warmup + args.steps):
+        value, unit, dt, info = oracle_sample(wl, seconds_target=max(1.0, 60.0 / (args.warmup + args.steps)))
+        if i >= args.warmup:
+            times.append((value, dt))
+    value = float(np.mean([t[0] for t in times]))
+    line = {"impl": "reference", "metric": metric_name(wl), "value": value, "unit": unit, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": float(np.mean([t[1] for t in times]) * 1e3),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": wl.name, "note": "each step is a bounded sample of the workload (see cpu_baseline.sample)"},
+            "cpu_baseline": dict(info, value=value),
+            "e2e": {"value": value, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def metric_name(wl):
+    if wl.decode_steps:
+        return "selective-KV decode attention HBM GB/s (one decode step, all layers)"
+    return "selective-KV attention TFLOP/s (one planning step, all layers)"
+
+
+# ---- the CUDA arm --------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (profiling)")
+    ap.add_argument("--impl", default="enl", choices=["enl", "reference"])
+    ap.add_argument("--workload", default="planner")
+    ap.add_argument("--split", type=int, default=0, help="KV splits (0 = library chooses)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "enl":
+        args.warmup = 3
+
+    from paper_2510_18546_b200 import synth
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    wl = synth.make(args.workload)
+    if args.layers > 0:
+        wl.n_layers = args.layers
+    if args.impl == "reference":
+        run_reference(args, wl, rank)
+        return
+
+    from paper_2510_18546_b200 import enl
+    from paper_2510_18546_b200.dist import init_process_group, max_over_ranks, barrier
+    dev = torch.device(f"cuda:{local}")
+    torch.cuda.set_device(dev)
+    init_process_group(world, rank, backend="nccl")
+    # weak scaling: every rank runs its own replica of the workload (episodes are independent; no
+    # data-path collective).  Rank r draws its values from seed + r.
+    wl.seed += rank
+
+    L = wl.n_layers
+    tq = wl.decode_steps if wl.decode_steps else int(sum(wl.n_q))
+    cache = enl.enl_cache_create(L, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.n_groups, wl.pool_tokens,
+                                 device=local, max_batch=wl.batch, max_q_tokens=max(tq, 1))
+    stream = torch.cuda.current_stream(dev).cuda_stream
+    store_src = []                       # per layer: (group id, K, V) rewritten every step
+    for layer in range(L):
+        for b in range(wl.batch):
+            k, v = wl.pool_kv(layer, b, dev)
+            offs = wl.pool_offsets(b)
+            for g in range(len(wl.pool_lens[b])):
+                enl.enl_group_store(cache, wl.group_base[b] + g, layer, k[offs[g]:offs[g + 1]], v[offs[g]:offs[g + 1]])
+            if b == 0:
+                g = int(wl.sel_local[0][0]) if len(wl.sel_local[0]) else 0
+                store_src.append((wl.group_base[0] + g, k[offs[g]:offs[g + 1]].clone(), v[offs[g]:offs[g + 1]].clone()))
+        torch.cuda.synchronize(dev)
+    qs, kns, vns = [], [], []
+    for layer in range(L):
+        q, kn, vn = wl.new_qkv(layer, dev)
+        qs.append(q); kns.append(kn); vns.append(vn)
+    sel = wl.sel_ids()
+    cs, cq, cn = wl.cu()
+    multi = wl.batch > 1
+    G = int(np.max(np.diff(cs))) if len(sel) else 0
+    outs = [torch.empty(tq if not wl.decode_steps else 1, wl.n_q_heads, wl.head_dim, dtype=torch.bfloat16, device=dev)
+            for _ in range(L)]
+    masses = [torch.empty(outs[0].shape[0], wl.n_q_heads, G + 1, dtype=torch.float32, device=dev) for _ in range(L)]
+
+    def attend(layer, q, kn, vn, out, mass, t=None):
+        if wl.decode_steps:
+            enl.enl_attend(cache, layer, sel, q[t:t + 1], kn, vn, out, mass, n_q=1, n_new=t + 1,
+                           split_hint=args.split, stream=stream)
+        else:
+            enl.enl_attend(cache, layer, sel, q, kn, vn, out, mass, cu_sel=cs if multi else None,
+                           cu_q=cq if multi else None, cu_new=cn if multi else None, split_hint=args.split,
+                           stream=stream)
+
+    def step(i, timed_events=None):
+        t = (i % wl.decode_steps) if wl.decode_steps else None
+        for layer in range(L):
+            gid, k, v = store_src[layer]
+            enl.enl_group_store(cache, gid, layer, k, v, stream=stream)
+        for layer in range(L):
+            if timed_events is not None:
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+            attend(layer, qs[layer], kns[layer], vns[layer], outs[layer], masses[layer], t)
+            if timed_events is not None:
+                e1.record()
+                timed_events.append((e0, e1))
+        return t
+
+    for i in range(args.warmup):
+        step(i)
+    torch.cuda.synchronize(dev)
+    plan = enl.enl_plan_inspect(cache)
+    n_splits = plan["n_splits"]
+    barrier()
+    torch.cuda.synchronize(dev)
+    e_beg, e_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as clk:
+        e_beg.record()
+        for i in range(args.steps):
+            step(args.warmup + i)
+        e_end.record()
+        torch.cuda.synchronize(dev)
+    barrier()
+    ms_total = max_over_ranks(e_beg.elapsed_time(e_end))
+    ms_step = ms_total / args.steps
+    status = enl.enl_cache_status(cache)
+
+    # the dominant kernel's own duration: events around every enl_attend call of a few more steps
+    evs = []
+    n_inst = max(1, min(5, args.steps))
+    for i in range(n_inst):
+        step(args.warmup + args.steps + i, evs)
+    torch.cuda.synchronize(dev)
+    attend_ms = float(np.mean([a.elapsed_time(b) for a, b in evs]))
+
+    if wl.decode_steps:
+        ts = [(args.warmup + i) % wl.decode_steps for i in range(args.steps)]
+        work_step = float(np.mean([decode_bytes_per_layer(wl, t) for t in ts])) * L
+        value, unit, bound = work_step * world / (ms_step * 1e-3) / 1e9, "GB/s", "hbm"
+        per_launch = work_step / L
+        achieved = per_launch / (attend_ms * 1e-3) / 1e9
+    else:
+        work_step = prefill_flops_per_layer(wl) * L
+        value, unit, bound = work_step * world / (ms_step * 1e-3) / 1e12, "TFLOP/s", "tensor"
+        per_launch = work_step / L
+        achieved = per_launch / (attend_ms * 1e-3) / 1e12
+    peaks = load_peaks()
+    peak = peaks["hbm_gbs"] if bound == "hbm" else peaks["bf16_tflops_sustained"]
+    roofline = {"bound": bound, "achieved": achieved, "peak": peak, "unit": unit, "frac": achieved / peak,
+                "traffic": NCU_TRAFFIC_BYTES.get(wl.name), "peak_source": peaks["_source"] +
+                (" (sustained bf16 GEMM)" if bound == "tensor" else " (copy bandwidth)"),
+                "kernel": f"attn_kernel<{wl.head_dim}>" + (" + combine_kernel" if n_splits > 1 else ""),
+                "launch_ms": attend_ms,
+                "algorithmic_per_launch": per_launch}
+
+    # ---- end to end through the C ABI with host buffers ----
+    e2e = None
+    if not args.no_e2e:
+        hq = [x.cpu().pin_memory() for x in qs]
+        hk = [x.cpu().pin_memory() for x in kns]
+        hv = [x.cpu().pin_memory() for x in vns]
+        ho = [torch.empty_like(o, device="cpu").pin_memory() for o in outs]
+        hm = [torch.empty_like(m, device="cpu").pin_memory() for m in masses]
+        dq, dk, dv = torch.empty_like(qs[0]), torch.empty_like(kns[0]), torch.empty_like(vns[0])
+
+        def e2e_step(i):
+            t = (i % wl.decode_steps) if wl.decode_steps else None
+            bi = bo = 0
+            for layer in range(L):
+                gid, k, v = store_src[layer]
+                enl.enl_group_store(cache, gid, layer, k, v, stream=stream)
+            for layer in range(L):
+                if wl.decode_steps:
+                    # the step's inputs: one query row and the new token's K/V row, appended to the
+                    # caller-owned device buffer that already holds the rows of earlier steps
+                    qs[layer][t:t + 1].copy_(hq[layer][t:t + 1], non_blocking=True)
+                    kns[layer][t:t + 1].copy_(hk[layer][t:t + 1], non_blocking=True)
+                    vns[layer][t:t + 1].copy_(hv[layer][t:t + 1], non_blocking=True)
+                    bi += hq[layer][t:t + 1].nbytes + 2 * hk[layer][t:t + 1].nbytes
+                    attend(layer, qs[layer], kns[layer], vns[layer], outs[layer], masses[layer], t)
+                else:
+                    dq.copy_(hq[layer], non_blocking=True)
+                    dk.copy_(hk[layer], non_blocking=True)
+                    dv.copy_(hv[layer], non_blocking=True)
+                    bi += hq[layer].nbytes + hk[layer].nbytes + hv[layer].nbytes
+                    attend(layer, dq, dk, dv, outs[layer], masses[layer], t)
+                ho[layer].copy_(outs[layer], non_blocking=True)
+                hm[layer].copy_(masses[layer], non_blocking=True)
+                bo += ho[layer].nbytes + hm[layer].nbytes
+            return bi, bo
+
+        for i in range(3):
+            e2e_step(i)
+        torch.cuda.synchronize(dev)
+        barrier()
+        n_e2e = max(3, min(args.steps, 10))
+        a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for i in range(n_e2e):
+            bi, bo = e2e_step(args.warmup + i)
+        b_.record()
+        torch.cuda.synchronize(dev)
+        barrier()
+        e2e_ms = max_over_ranks(a.elapsed_time(b_)) / n_e2e
+        scale = 1e9 if wl.decode_steps else 1e12
+        e2e = {"value": work_step * world / (e2e_ms * 1e-3) / scale, "unit": unit, "ms_per_step": e2e_ms,
+               "h2d_bytes_per_step": int(bi), "d2h_bytes_per_step": int(bo), "steps": n_e2e}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        wl0 = synth.make(args.workload)
+        _, _, _, cpu = oracle_sample(wl0)
+
+    launches_per_step = L * (1 + (1 if n_splits > 1 else 0)) + L      # attention (+ merge) + page scatter
+    enl.enl_cache_free(cache)
+    if rank == 0:
+        line = {"metric": metric_name(wl), "value": value, "unit": unit, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                "config": {"workload": wl.name, "layers": L, "q_heads": wl.n_q_heads, "kv_heads": wl.n_kv_heads,
+                           "head_dim": wl.head_dim, "batch": wl.batch, "pool_groups": wl.n_groups,
+                           "selected_groups": int(len(sel)), "selected_tokens": int(sum(wl.selected_tokens(b) for b in range(wl.batch))),
+                           "new_tokens": int(sum(wl.n_new)) if not wl.decode_steps else 1,
+                           "kv_splits": n_splits, "parallelism": f"replicas x{world}",
+                           "l2": "inputs larger than L2: every layer of a step reads its own pages and tensors"},
+                "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e,
+                "gpu_launches": launches_per_step * args.steps, "clocks": clk.summary(),
+                "status": "ok" if status == 0 else enl.strerror(status),
+                "fraction_of_nominal": achieved / (8000.0 if bound == "hbm" else 2250.0)}
+        print(json.dumps(line), flush=True)
+
+
+if __name__ == "__main__":
+    main()
