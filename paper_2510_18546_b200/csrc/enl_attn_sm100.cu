@@ -15,7 +15,8 @@
 // kernel merges.
 //
 // Roles: warps 0-3 softmax of Q tile 0, warps 4-7 softmax of Q tile 1, warp 8 TMA producer,
-// warp 9 MMA issuer (and TMEM owner).  TMEM columns: S0 [0,128) S1 [128,256) O0 [256,384) O1 [384,512);
+// warp 9 MMA issuer (and TMEM owner), warps 10-11 idle (they complete the third warpgroup so that
+// setmaxnreg can move registers from it to the two softmax warpgroups, which hold a 128-column row of S).  TMEM columns: S0 [0,128) S1 [128,256) O0 [256,384) O1 [384,512);
 // P_i overwrites the first 64 columns of S_i.
 #include <cuda_bf16.h>
 
@@ -25,7 +26,9 @@
 namespace enl {
 namespace {
 
-constexpr int kThreads      = 320;
+constexpr int kThreads      = 384;
+constexpr int kRegsSoftmax  = 224;            // 2 softmax warps + 1 other warp per scheduler: 2*224 + 56 <= 512
+constexpr int kRegsOther    = 56;
 constexpr int kProducerWarp = 8;
 constexpr int kMmaWarp      = 9;
 constexpr uint32_t kTmemCols = 512;
@@ -233,7 +236,9 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
 
     bool ok = true;
 
-    if (warp == kProducerWarp) {
+    if (warp >= 8) {
+      asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
+      if (warp == kProducerWarp) {
         // ================= TMA producer =================
         if (n_tiles > 0) {
             if (lane == 0) {
@@ -286,7 +291,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                 }
             }
         }
-    } else if (warp == kMmaWarp) {
+      } else if (warp == kMmaWarp) {
         // ================= MMA issuer =================
         if (n_tiles > 0) {
             constexpr uint32_t idesc_qk = make_idesc(kTileKeys, false);
@@ -352,7 +357,10 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                 }
             }
         }
-    } else if ((warp >> 2) < n_qt) {
+      }
+    } else {
+      asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
+      if ((warp >> 2) < n_qt) {
         // ================= softmax / epilogue, one thread per row =================
         const int i = warp >> 2;
         const int r = (warp & 3) * 32 + lane;
@@ -543,6 +551,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                 }
             }
         }
+      }
     }
 
     // ---- teardown ----

@@ -37,34 +37,56 @@ __device__ __forceinline__ float ex2f(float x)
     return y;
 }
 
-// One block per (query row, q head); thread d merges channel d, then the threads stride over the slots.
+// One warp per (query row, q head): lane l merges channels 4l..4l+3 (D = 128) or 2l, 2l+1 (D = 64),
+// then the lanes stride over the slots.
+template <int D>
 __global__ void combine_kernel(const CombineParams p)
 {
-    const long long rh = blockIdx.x;                       // row * Hq + head
-    const int row = static_cast<int>(rh / p.Hq);
+    constexpr int V = D / 32;                               // channels per lane
+    const int lane = threadIdx.x & 31;
+    const long long rh = blockIdx.x * static_cast<long long>(blockDim.x >> 5) + (threadIdx.x >> 5);
     const long long split_stride = static_cast<long long>(p.n_q_total) * p.Hq;
+    if (rh >= split_stride) return;
+    const int row = static_cast<int>(rh / p.Hq);
     const float ninf = -__builtin_huge_valf();
 
-    float mx = ninf;
-    for (int k = 0; k < p.n_splits; ++k) mx = fmaxf(mx, p.part_lse[k * split_stride + rh]);
-    float sum = 0.f;
-    for (int k = 0; k < p.n_splits; ++k) {
-        const float v = p.part_lse[k * split_stride + rh];
-        if (v != ninf) sum += ex2f(v - mx);
-    }
+    // every lane needs every split's log-sum-exp: lane k loads split k (and k + 32), then shuffles
+    float my0 = lane < p.n_splits ? p.part_lse[lane * split_stride + rh] : ninf;
+    float my1 = lane + 32 < p.n_splits ? p.part_lse[(lane + 32) * split_stride + rh] : ninf;
+    float mx = fmaxf(my0, my1);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    float sum = (my0 != ninf ? ex2f(my0 - mx) : 0.f) + (my1 != ninf ? ex2f(my1 - mx) : 0.f);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
     const float lse = mx + log2f(sum);
+    const float w0 = my0 != ninf ? ex2f(my0 - lse) : 0.f;
+    const float w1 = my1 != ninf ? ex2f(my1 - lse) : 0.f;
 
-    for (int d = threadIdx.x; d < p.D; d += blockDim.x) {
-        float o = 0.f;
-        for (int k = 0; k < p.n_splits; ++k) {
-            const float v = p.part_lse[k * split_stride + rh];
-            if (v != ninf) o += ex2f(v - lse) * p.part_o[(k * split_stride + rh) * p.D + d];
+    float acc[V];
+#pragma unroll
+    for (int x = 0; x < V; ++x) acc[x] = 0.f;
+    for (int k = 0; k < p.n_splits; ++k) {
+        const float w = __shfl_sync(0xffffffffu, k < 32 ? w0 : w1, k & 31);
+        if (w != 0.f) {
+            const float *src = p.part_o + (k * split_stride + rh) * D + lane * V;
+            if constexpr (V == 4) {
+                const float4 v = *reinterpret_cast<const float4 *>(src);
+                acc[0] += w * v.x; acc[1] += w * v.y; acc[2] += w * v.z; acc[3] += w * v.w;
+            } else {
+                const float2 v = *reinterpret_cast<const float2 *>(src);
+                acc[0] += w * v.x; acc[1] += w * v.y;
+            }
         }
-        static_cast<__nv_bfloat16 *>(p.out)[rh * p.D + d] = __float2bfloat16_rn(o);
     }
+    __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(p.out) + rh * D + lane * V;
+#pragma unroll
+    for (int x = 0; x < V; x += 2)
+        *reinterpret_cast<__nv_bfloat162 *>(dst + x) = __floats2bfloat162_rn(acc[x], acc[x + 1]);
+
     if (p.mass) {
         const int G = p.row_slots[row];
-        for (int s = threadIdx.x; s <= G; s += blockDim.x) {
+        for (int s = lane; s <= G; s += 32) {
             float w = 0.f;
             for (int k = 0; k < p.n_splits; ++k) {
                 const float v = p.part_slot[(k * split_stride + rh) * p.slot_stride + s];
@@ -95,9 +117,12 @@ cudaError_t launch_page_scatter(void *kpool_layer, void *vpool_layer, const void
 
 cudaError_t launch_combine(const CombineParams &p, cudaStream_t st)
 {
-    const long long blocks = static_cast<long long>(p.n_q_total) * p.Hq;
-    if (blocks <= 0) return cudaSuccess;
-    combine_kernel<<<static_cast<int>(blocks), 128, 0, st>>>(p);
+    const long long pairs = static_cast<long long>(p.n_q_total) * p.Hq;
+    if (pairs <= 0) return cudaSuccess;
+    const int warps = 8;
+    const int blocks = static_cast<int>((pairs + warps - 1) / warps);
+    if (p.D == 128) combine_kernel<128><<<blocks, warps * 32, 0, st>>>(p);
+    else combine_kernel<64><<<blocks, warps * 32, 0, st>>>(p);
     return cudaGetLastError();
 }
 
