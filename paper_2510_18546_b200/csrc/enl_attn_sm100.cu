@@ -147,6 +147,36 @@ __device__ __forceinline__ float lg2(float x)
     return y;
 }
 
+// 3-input max and packed 2 x fp32 arithmetic (one issue slot for two lanes of work)
+__device__ __forceinline__ float fmax3(float a, float b, float c)
+{
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t pack2(float lo, float hi)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float &lo, float &hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b)
+{
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+
 // Shared-memory matrix descriptor, 128-byte swizzle, rows of 128 B, 8-row groups 1024 B apart.
 // K-major operand (the contraction dimension is contiguous): LBO unused.
 // MN-major operand: LBO = distance between 64-element column blocks.
@@ -171,6 +201,16 @@ __host__ __device__ constexpr uint32_t make_idesc(int n, bool b_mn_major)
 }
 
 constexpr float kNegInf = -__builtin_huge_valf();
+
+// Optional phase timestamps of CTA 0 (development builds only; never compiled into the library).
+#ifdef ENL_TRACE
+__device__ long long g_trace[3][96][8];
+#define ENL_TR(role, tile, slot) do { if (blockIdx.x == 0 && lane == 0 && (tile) < 96) g_trace[role][tile][slot] = clock64(); } while (0)
+#define ENL_PIN(x) asm volatile("" : "+f"(x) :: "memory")
+#else
+#define ENL_TR(role, tile, slot) do { } while (0)
+#define ENL_PIN(x) do { } while (0)
+#endif
 
 // ---- the kernel ----------------------------------------------------------------------------
 template <int D>
@@ -253,7 +293,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                 const bool cached = j < ep.n_ctiles;
                 int page = 0;
                 if (cached && lane < kPagesPerTile)
-                    page = p.stream[ep.stream_off + j * kPagesPerTile + lane].x;
+                    page = p.stream_page[ep.stream_off + j * kPagesPerTile + lane];
                 for (int kv = 0; kv < 2; ++kv, ++fill) {
                     const int st = fill % C::kStages;
                     if (fill >= C::kStages) {
@@ -344,9 +384,11 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                 if (ok && more) ok = wait_full(fk);
                 if (!ok) break;
                 for (int i = 0; i < n_qt; ++i) {
+                    ENL_TR(2, jj, 4 * i);
                     ok = mbar_wait(bar_p_full(i), static_cast<uint32_t>(jj & 1), abort_flag, p.status);
                     if (!ok) break;
                     tc_fence_after();
+                    ENL_TR(2, jj, 4 * i + 1);
                     issue_pv(i, fv % C::kStages, jj == 0);
                     if (i == n_qt - 1) commit_to(bar_kv_empty(fv % C::kStages));
                     if (!more) commit_to(bar_o_done(i));
@@ -385,28 +427,56 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
         float m = kNegInf, l = 0.f, acc = 0.f;
         int cur_slot = -1;
 
+        // (slot << 8 | valid keys) of the eight pages of a tile; fetched one tile ahead so that the
+        // loads are in flight while this tile is processed
+        auto load_meta = [&](int j, int (&dst)[kPagesPerTile]) {
+            if (j < ep.n_ctiles) {
+                const int4 *e4 = reinterpret_cast<const int4 *>(p.stream_meta + ep.stream_off + j * kPagesPerTile);
+                const int4 a = __ldg(e4), b = __ldg(e4 + 1);
+                dst[0] = a.x; dst[1] = a.y; dst[2] = a.z; dst[3] = a.w;
+                dst[4] = b.x; dst[5] = b.y; dst[6] = b.z; dst[7] = b.w;
+            } else {
+#pragma unroll
+                for (int e = 0; e < kPagesPerTile; ++e) dst[e] = (G << 8) | kPageTokens;
+            }
+        };
+        int meta_next[kPagesPerTile];
+        load_meta(j_beg, meta_next);
+
         for (int jj = 0; jj < n_tiles; ++jj) {
             const int j = j_beg + jj;
             const bool cached = j < ep.n_ctiles;
             int meta[kPagesPerTile];
-            if (cached) {
-                const int4 *e4 = reinterpret_cast<const int4 *>(p.stream + ep.stream_off + j * kPagesPerTile);
 #pragma unroll
-                for (int e = 0; e < kPagesPerTile / 2; ++e) {
-                    const int4 v = __ldg(e4 + e);
-                    meta[2 * e] = v.y;
-                    meta[2 * e + 1] = v.w;
-                }
-            } else {
-#pragma unroll
-                for (int e = 0; e < kPagesPerTile; ++e) meta[e] = (G << 8) | kPageTokens;
-            }
+            for (int e = 0; e < kPagesPerTile; ++e) meta[e] = meta_next[e];
+            if (jj + 1 < n_tiles) load_meta(j + 1, meta_next);
+            if ((warp & 3) == 0) ENL_TR(i, jj, 0);
             ok = mbar_wait(bar_s_full(i), static_cast<uint32_t>(jj & 1), abort_flag, p.status);
             if (!ok) break;
             tc_fence_after();
+            if ((warp & 3) == 0) ENL_TR(i, jj, 1);
 
             uint32_t su[128];
+#ifdef ENL_TRACE_LD
+            {
+                uint32_t c0[32], c1[32], c2[32], c3[32];
+                tmem_ld32_wait(t_s, c0);
+                if ((warp & 3) == 0) ENL_TR(i, jj, 2);
+                tmem_ld32_wait(t_s + 32, c1);
+                if ((warp & 3) == 0) ENL_TR(i, jj, 6);
+                tmem_ld32_wait(t_s + 64, c2);
+                if ((warp & 3) == 0) ENL_TR(i, jj, 7);
+                tmem_ld32_wait(t_s + 96, c3);
+                if ((warp & 3) == 0) ENL_TR(i, jj, 3);
+#pragma unroll
+                for (int x = 0; x < 32; ++x) { su[x] = c0[x]; su[32 + x] = c1[x]; su[64 + x] = c2[x]; su[96 + x] = c3[x]; }
+            }
+#define ENL_TR2(a, b, c) do { } while (0)
+#else
             tmem_ld128_wait(t_s, su);
+            if ((warp & 3) == 0) ENL_TR(i, jj, 2);
+#define ENL_TR2(a, b, c) ENL_TR(a, b, c)
+#endif
             float s[128];
 #pragma unroll
             for (int x = 0; x < 128; ++x) s[x] = __uint_as_float(su[x]);
@@ -431,9 +501,25 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                 }
             }
 
-            float mx = s[0];
 #pragma unroll
-            for (int x = 1; x < 128; ++x) mx = fmaxf(mx, s[x]);
+            for (int x = 0; x < 128; x += 8) ENL_PIN(s[x]);
+            if ((warp & 3) == 0) ENL_TR2(i, jj, 6);
+            // row maximum: eight independent chains of 3-input max, one per 16-key page
+            float mx;
+            {
+                float pm[kPagesPerTile];
+#pragma unroll
+                for (int e = 0; e < kPagesPerTile; ++e) {
+                    const int b = e * kPageTokens;
+                    float a = fmax3(s[b], s[b + 1], s[b + 2]);
+#pragma unroll
+                    for (int x = 3; x < 15; x += 2) a = fmax3(a, s[b + x], s[b + x + 1]);
+                    pm[e] = fmaxf(a, s[b + 15]);
+                }
+                mx = fmax3(fmax3(pm[0], pm[1], pm[2]), fmax3(pm[3], pm[4], pm[5]), fmaxf(pm[6], pm[7]));
+            }
+            ENL_PIN(mx);
+            if ((warp & 3) == 0) ENL_TR2(i, jj, 7);
             const float m_cand = mx * scale;
             const bool need = m_cand > m + kRescaleThreshold;       // also true when m == -inf < m_cand
             if (__any_sync(0xffffffffu, need)) {
@@ -453,27 +539,46 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                     }
                 }
             }
-            const float m_use = (m == kNegInf) ? 0.f : m;
+            float m_use = (m == kNegInf) ? 0.f : m;
+            ENL_PIN(m_use);
+            if ((warp & 3) == 0) ENL_TR2(i, jj, 3);
 
+            const uint64_t sc2 = pack2(scale, scale), nm2 = pack2(-m_use, -m_use);
+            float bs[kPagesPerTile];                               // sum of p over each page
 #pragma unroll
             for (int e = 0; e < kPagesPerTile; ++e) {
-                float bs = 0.f;
+                uint64_t pr[kPageTokens / 2];
 #pragma unroll
-                for (int x = 0; x < kPageTokens; ++x) {
-                    const float pv = ex2(fmaf(s[e * kPageTokens + x], scale, -m_use));
-                    s[e * kPageTokens + x] = pv;
-                    bs += pv;
+                for (int x = 0; x < kPageTokens / 2; ++x) {
+                    const int b = e * kPageTokens + 2 * x;
+                    float a0, a1;
+                    unpack2(fma2(pack2(s[b], s[b + 1]), sc2, nm2), a0, a1);
+                    s[b] = ex2(a0);
+                    s[b + 1] = ex2(a1);
+                    pr[x] = pack2(s[b], s[b + 1]);
                 }
+                const uint64_t q0 = add2(add2(pr[0], pr[1]), add2(pr[2], pr[3]));
+                const uint64_t q1 = add2(add2(pr[4], pr[5]), add2(pr[6], pr[7]));
+                float b0, b1;
+                unpack2(add2(q0, q1), b0, b1);
+                bs[e] = b0 + b1;
+            }
+            // credit the page sums to their slots; a slot that ends parks its log2-sum-exp
+#pragma unroll
+            for (int e = 0; e < kPagesPerTile; ++e) {
                 const int slot = meta[e] >> 8;
                 if (slot != cur_slot) {
                     if (slot_out && cur_slot >= 0) slot_out[cur_slot] = lg2(acc) + m_use;
                     acc = 0.f;
                     cur_slot = slot;
                 }
-                acc += bs;
-                l += bs;
+                acc += bs[e];
+                l += bs[e];
             }
 
+            ENL_PIN(l);
+            ENL_PIN(acc);
+            if ((warp & 3) == 0) ENL_TR(i, jj, 4);
             // P (bf16 pairs, even key in the low half) over the first 64 columns of S_i
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
@@ -489,6 +594,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_p_full(i));
+            if ((warp & 3) == 0) ENL_TR(i, jj, 5);
         }
 
         // ---- per-row results ----
@@ -502,9 +608,9 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                     int first = G + 1, last = -1;
                     if (n_tiles > 0) {
                         first = (j_beg < ep.n_ctiles)
-                                    ? (p.stream[ep.stream_off + j_beg * kPagesPerTile].y >> 8) : G;
+                                    ? (p.stream_meta[ep.stream_off + j_beg * kPagesPerTile] >> 8) : G;
                         last = (j_end > ep.n_ctiles)
-                                   ? G : (p.stream[ep.stream_off + j_end * kPagesPerTile - 1].y >> 8);
+                                   ? G : (p.stream_meta[ep.stream_off + j_end * kPagesPerTile - 1] >> 8);
                     }
                     if (slot_out)
                         for (int sl = 0; sl <= G; ++sl)
@@ -564,6 +670,13 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
 }
 
 }  // namespace
+
+#ifdef ENL_TRACE
+extern "C" int enl_debug_trace(long long *out)
+{
+    return cudaMemcpyFromSymbol(out, g_trace, sizeof(g_trace)) == cudaSuccess ? 0 : -1;
+}
+#endif
 
 size_t attention_smem_bytes(int head_dim)
 {

@@ -84,7 +84,7 @@ struct enl_cache {
     // gather plan: host image (pinned when there is a GPU), device copy, capacities
     int32_t cap_entries = 0, cap_items = 0;
     uint8_t *plan_host = nullptr, *plan_dev = nullptr;
-    size_t off_eps = 0, off_items = 0, off_stream = 0, off_rowslots = 0, plan_bytes = 0;
+    size_t off_eps = 0, off_items = 0, off_stream = 0, off_meta = 0, off_rowslots = 0, plan_bytes = 0;
     cudaEvent_t plan_copied = nullptr;
     bool plan_valid = false, plan_on_device = false;
     uint64_t plan_epoch = 0;
@@ -100,7 +100,8 @@ struct enl_cache {
 
     EpInfo *h_eps() { return reinterpret_cast<EpInfo *>(plan_host + off_eps); }
     Item *h_items() { return reinterpret_cast<Item *>(plan_host + off_items); }
-    int2 *h_stream() { return reinterpret_cast<int2 *>(plan_host + off_stream); }
+    int32_t *h_stream() { return reinterpret_cast<int32_t *>(plan_host + off_stream); }
+    int32_t *h_meta() { return reinterpret_cast<int32_t *>(plan_host + off_meta); }
     int32_t *h_rowslots() { return reinterpret_cast<int32_t *>(plan_host + off_rowslots); }
 };
 
@@ -182,7 +183,8 @@ extern "C" int enl_cache_create(const enl_cache_desc_t *desc, enl_cache_t **out)
     c->off_eps = 0;
     c->off_items = align256(c->off_eps + sizeof(EpInfo) * d.max_batch);
     c->off_stream = align256(c->off_items + sizeof(Item) * c->cap_items);
-    c->off_rowslots = align256(c->off_stream + sizeof(int2) * c->cap_entries);
+    c->off_meta = align256(c->off_stream + sizeof(int32_t) * c->cap_entries);
+    c->off_rowslots = align256(c->off_meta + sizeof(int32_t) * c->cap_entries);
     c->plan_bytes = align256(c->off_rowslots + sizeof(int32_t) * d.max_q_tokens);
 
     if (!c->gpu) {
@@ -423,7 +425,8 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
         if (c->gpu && cudaEventSynchronize(c->plan_copied) != cudaSuccess) { cudaGetLastError(); return ENL_E_CUDA; }
         c->plan_valid = false;
         EpInfo *eps = c->h_eps();
-        int2 *stream = c->h_stream();
+        int32_t *stream = c->h_stream();
+        int32_t *smeta = c->h_meta();
         int32_t *rowslots = c->h_rowslots();
         int32_t ne = 0;
         for (int b = 0; b < B; ++b) {
@@ -439,13 +442,14 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
                 const int slot = s - cu_sel[b];
                 const Group &g = c->groups[a->sel_ids[s]];
                 const int len = sel_len[s], np = ceil_div(len, kPageTokens);
-                if (np == 0) stream[ne++] = make_int2(kZeroPage, slot << 8);
+                if (np == 0) { stream[ne] = kZeroPage; smeta[ne++] = slot << 8; }
                 for (int i = 0; i < np; ++i) {
                     const int nv = std::min(kPageTokens, len - i * kPageTokens);
-                    stream[ne++] = make_int2(g.pages[i], (slot << 8) | nv);
+                    stream[ne] = g.pages[i];
+                    smeta[ne++] = (slot << 8) | nv;
                 }
             }
-            while ((ne - e.stream_off) % kPagesPerTile) stream[ne++] = make_int2(kZeroPage, (e.n_slots - 1) << 8);
+            while ((ne - e.stream_off) % kPagesPerTile) { stream[ne] = kZeroPage; smeta[ne++] = (e.n_slots - 1) << 8; }
             e.n_ctiles = (ne - e.stream_off) / kPagesPerTile;
             for (int r = e.q_off; r < e.q_off + e.n_q; ++r) rowslots[r] = e.n_slots;
         }
@@ -484,10 +488,13 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
 
     if (!c->plan_on_device) {
         // one copy covers episodes, items, stream and row->slots (unused gaps travel too; they are small)
-        const size_t used_stream = c->off_stream + sizeof(int2) * c->plan_entries;
+        const size_t ent_bytes = sizeof(int32_t) * c->plan_entries;
         bool okc = cudaMemcpyAsync(c->plan_dev, c->plan_host, c->off_stream, cudaMemcpyHostToDevice, st) == cudaSuccess &&
-                   cudaMemcpyAsync(c->plan_dev + c->off_stream, c->plan_host + c->off_stream, used_stream - c->off_stream,
-                                   cudaMemcpyHostToDevice, st) == cudaSuccess &&
+                   (ent_bytes == 0 ||
+                    (cudaMemcpyAsync(c->plan_dev + c->off_stream, c->plan_host + c->off_stream, ent_bytes,
+                                     cudaMemcpyHostToDevice, st) == cudaSuccess &&
+                     cudaMemcpyAsync(c->plan_dev + c->off_meta, c->plan_host + c->off_meta, ent_bytes,
+                                     cudaMemcpyHostToDevice, st) == cudaSuccess)) &&
                    cudaMemcpyAsync(c->plan_dev + c->off_rowslots, c->plan_host + c->off_rowslots,
                                    sizeof(int32_t) * a->n_q, cudaMemcpyHostToDevice, st) == cudaSuccess &&
                    cudaEventRecord(c->plan_copied, st) == cudaSuccess;
@@ -516,7 +523,8 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
     p.tm_vpool = c->tm_v[a->layer];
     p.items = reinterpret_cast<const Item *>(c->plan_dev + c->off_items);
     p.eps = reinterpret_cast<const EpInfo *>(c->plan_dev + c->off_eps);
-    p.stream = reinterpret_cast<const int2 *>(c->plan_dev + c->off_stream);
+    p.stream_page = reinterpret_cast<const int32_t *>(c->plan_dev + c->off_stream);
+    p.stream_meta = reinterpret_cast<const int32_t *>(c->plan_dev + c->off_meta);
     p.out = a->out;
     p.mass = a->group_mass;
     p.status = c->status_dev;
@@ -564,10 +572,10 @@ extern "C" int enl_plan_inspect(const enl_cache_t *cc, int32_t cap_entries, int3
     if (n_entries) *n_entries = c->plan_entries;
     if (n_splits) *n_splits = c->plan_splits;
     if (n_items) *n_items = c->plan_items;
-    const int2 *s = c->h_stream();
+    const int32_t *s = c->h_stream(), *m = c->h_meta();
     for (int i = 0; i < c->plan_entries && i < cap_entries; ++i) {
-        if (stream_pages) stream_pages[i] = s[i].x;
-        if (stream_meta) stream_meta[i] = s[i].y;
+        if (stream_pages) stream_pages[i] = s[i];
+        if (stream_meta) stream_meta[i] = m[i];
     }
     const EpInfo *e = c->h_eps();
     for (int b = 0; b < c->plan_batch && b < cap_batch; ++b) {

@@ -41,7 +41,8 @@ struct AttnParams {
     CUtensorMap tm_vpool;
     const Item   *items;
     const EpInfo *eps;
-    const int2   *stream;   // {page id, slot << 8 | valid tokens}
+    const int32_t *stream_page;   // KV stream: page id of every entry
+    const int32_t *stream_meta;   // KV stream: slot << 8 | valid tokens
     void   *out;            // bf16 [n_q][Hq][D]
     float  *mass;           // fp32 or null
     float  *part_o;         // split mode: [split][row][Hq][D] fp32 (normalised by the split's own sum)
