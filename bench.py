@@ -120,45 +120,54 @@ class ClockSampler:
 
 
 # ---- the oracle arm (also the cpu_baseline leg) -------------------------------------------------
-def oracle_sample(wl, seconds_target: float = 12.0):
-    """Times the float64 oracle, as it stands, on a bounded sample of the workload: layer 0, episode 0,
-    all q heads, as many query rows as fit the time target.  Returns (value in the metric's unit, dict)."""
+def oracle_sample(wl, seconds_target: float = 15.0):
+    """Times the float64 oracle, as it stands, on a bounded sample of the workload: episode 0, all q heads,
+    layer after layer (for a decode workload: step after step of layer 0) until about `seconds_target`
+    seconds of CPU work have been done; a layer too long for that contributes evenly spaced query rows.
+    Returns (value in the metric's unit, unit, seconds, dict)."""
     from oracle import enl_oracle as orc
-    b, layer = 0, 0
-    k, v = wl.pool_kv(layer, b, "cpu")
-    offs = wl.pool_offsets(b)
-    ks = [k[offs[g]:offs[g + 1]] for g in wl.sel_local[b]]
-    vs = [v[offs[g]:offs[g + 1]] for g in wl.sel_local[b]]
-    q, kn, vn = wl.new_qkv(layer, "cpu")
+    b = 0
     S = wl.selected_tokens(b)
+    offs = wl.pool_offsets(b)
+    work, dt, n_calls, n_rows = 0.0, 0.0, 0, 0
+    layer, t_dec = 0, wl.decode_steps - 1 if wl.decode_steps else 0
+    row_budget = None
+    while dt < seconds_target and layer < wl.n_layers:
+        k, v = wl.pool_kv(layer, b, "cpu")
+        ks = [k[offs[g]:offs[g + 1]] for g in wl.sel_local[b]]
+        vs = [v[offs[g]:offs[g + 1]] for g in wl.sel_local[b]]
+        q, kn, vn = wl.new_qkv(layer, "cpu")
+        if wl.decode_steps:
+            q, kn, vn = q[t_dec:t_dec + 1], kn[:t_dec + 1], vn[:t_dec + 1]
+            rows = [0]
+        else:
+            q, kn, vn = q[:wl.n_q[b]], kn[:wl.n_new[b]], vn[:wl.n_new[b]]
+            n_q = q.shape[0]
+            if row_budget is None:
+                # calibrate on the most expensive row, then size one layer's share of the sample
+                t0 = time.perf_counter()
+                orc.attend_slots(wl.n_q_heads, wl.n_kv_heads, wl.head_dim, ks, vs, q, kn, vn, rows=[n_q - 1])
+                row_budget = int(max(1, min(n_q, seconds_target / max(time.perf_counter() - t0, 1e-5))))
+            rows = sorted(set(np.linspace(0, n_q - 1, row_budget).astype(int).tolist()))
+        n_q, n_new = q.shape[0], kn.shape[0]
+        t0 = time.perf_counter()
+        orc.attend_slots(wl.n_q_heads, wl.n_kv_heads, wl.head_dim, ks, vs, q, kn, vn, rows=rows)
+        dt += time.perf_counter() - t0
+        n_calls += 1
+        n_rows += len(rows)
+        if wl.decode_steps:
+            work += decode_bytes_per_layer(wl, t_dec)
+        else:
+            work += sum(4.0 * wl.n_q_heads * wl.head_dim * (S + (n_new - n_q) + r + 1) for r in rows)
+        layer += 1
     if wl.decode_steps:
-        t = wl.decode_steps - 1
-        q, kn, vn = q[t:t + 1], kn[:t + 1], vn[:t + 1]
-        rows = [0]
-    else:
-        q, kn, vn = q[:wl.n_q[b]], kn[:wl.n_new[b]], vn[:wl.n_new[b]]
-        rows = None
-    # calibrate on a few rows, then size the sample
-    n_q, n_new = q.shape[0], kn.shape[0]
-    probe = [n_q - 1] if rows is None else rows
-    t0 = time.perf_counter()
-    orc.attend_slots(wl.n_q_heads, wl.n_kv_heads, wl.head_dim, ks, vs, q, kn, vn, rows=probe)
-    dt_probe = time.perf_counter() - t0
-    if rows is None:
-        n = int(max(1, min(n_q, seconds_target / max(dt_probe, 1e-4))))
-        rows = sorted(set(np.linspace(0, n_q - 1, n).astype(int).tolist()))
-    t0 = time.perf_counter()
-    orc.attend_slots(wl.n_q_heads, wl.n_kv_heads, wl.head_dim, ks, vs, q, kn, vn, rows=rows)
-    dt = time.perf_counter() - t0
-    if wl.decode_steps:
-        work = decode_bytes_per_layer(wl, wl.decode_steps - 1)
         value, unit = work / dt / 1e9, "GB/s"
+        what = f"step {t_dec} of layers 0..{n_calls - 1}"
     else:
-        work = sum(4.0 * wl.n_q_heads * wl.head_dim * (S + (n_new - n_q) + r + 1) for r in rows)
         value, unit = work / dt / 1e12, "TFLOP/s"
+        what = f"layers 0..{n_calls - 1}, {n_rows} query rows in all"
     info = {"value": value, "unit": unit, "cores": orc.threads(), "kind": "oracle",
-            "sample": f"layer 0, episode 0, {len(rows)} of {n_q} query rows x {wl.n_q_heads} heads, "
-                      f"{S} cached + {n_new} new keys, {dt:.2f} s"}
+            "sample": f"episode 0, {what} x {wl.n_q_heads} heads, {S} cached keys, {dt:.1f} s of oracle time"}
     return value, unit, dt, info
 
 
@@ -168,7 +177,7 @@ def run_reference(args, wl, rank):
     times = []
     info = None
     for i in range(args.warmup + args.steps):
-        value, unit, dt, info = oracle_sample(wl, seconds_target=max(1.0, 60.0 / (args.warmup + args.steps)))
+        value, unit, dt, info = oracle_sample(wl, seconds_target=max(1.0, min(15.0, 90.0 / (args.warmup + args.steps))))
         if i >= args.warmup:
             times.append((value, dt))
     value = float(np.mean([t[0] for t in times]))
