@@ -55,7 +55,8 @@ enum {                                            /* return codes               
     ENL_E_NOGROUP  = -2,   /* group id out of range, or never stored for that layer            */
     ENL_E_NOMEM    = -3,   /* page pool, plan buffers or a create-time allocation exhausted    */
     ENL_E_CUDA     = -4,   /* a CUDA call failed, or a GPU operation on a bookkeeping cache    */
-    ENL_E_TIMEOUT  = -5    /* a bounded wait inside a kernel expired (see enl_cache_status)    */
+    ENL_E_TIMEOUT  = -5,   /* a bounded wait inside a kernel expired (see enl_cache_status)    */
+    ENL_E_LIMIT    = -6    /* a size beyond the fixed maxima of enl_attend_static              */
 };
 
 typedef struct {
@@ -162,6 +163,55 @@ int enl_plan_inspect(const enl_cache_t *c, int32_t cap_entries, int32_t *stream_
                      int32_t *stream_meta, int32_t *n_entries, int32_t cap_batch,
                      int32_t *ep_stream_off, int32_t *ep_cached_tiles, int32_t *n_splits,
                      int32_t *n_items);
+
+/* ---- an entry point that allocates nothing ------------------------------------------------ */
+
+#define ENL_STATIC_MAX_SEGMENTS  255                 /* cached segments per call                      */
+#define ENL_STATIC_MAX_KEYS      65536               /* cached keys + new keys per call               */
+#define ENL_STATIC_SCRATCH_BYTES (4u << 20)          /* size of the library's built-in scratch array  */
+
+typedef struct {
+    int32_t n_q_heads, n_kv_heads;     /* n_q_heads = n_kv_heads * {1,2,4,8}                        */
+    int32_t head_dim;                  /* 64 or 128                                                 */
+    int32_t n_seg;                     /* cached segments (groups) in the key stream, may be 0      */
+    const int32_t *seg_len;            /* HOST [n_seg]: tokens per segment, in stream order         */
+    int32_t n_new;                     /* new-token keys the query sees (its own included), >= 1    */
+    const void *q;                     /* device bf16 [n_q_heads][head_dim]: the one query token    */
+    const void *k, *v;                 /* device bf16 [sum(seg_len) + n_new][n_kv_heads][head_dim]: */
+                                       /*   the segments back to back, then the new keys            */
+    void *out;                         /* device bf16 [n_q_heads][head_dim]                         */
+    float *group_mass;                 /* device fp32 [n_q_heads][n_seg + 1] or NULL; slot n_seg =  */
+                                       /*   the new tokens                                          */
+} enl_static_args_t;
+
+/*
+ * (The paper has no counterpart: this entry point exists for deployment reasons only.)
+ * One decode-style query token attends over segments of cached keys plus the new keys, exactly as an
+ * enl_attend call with n_q = 1 would, but WITHOUT touching any allocator: no cache object, no
+ * cudaMalloc / cudaFree, no allocating library routine, no host heap.  It is meant for callers
+ * that are not allowed to allocate once they are running -- a planner tick inside a real-time
+ * control loop with memory fixed at start-up, code hosted by another runtime that owns the whole
+ * device heap, a process whose allocator is sealed after initialisation.  Such callers cannot create
+ * a cache (the paged pool is an allocation), so they pass the key/value stream as ONE contiguous
+ * buffer they own, and the split-KV partial results go to a fixed array of ENL_STATIC_SCRATCH_BYTES
+ * that is part of the library image: every GPU that loads the library carries that array until the
+ * process exits, whether or not this function is ever called.
+ *
+ * The work is split over up to 64 key ranges whose partial outputs, log-sum-exps and per-segment
+ * sums are written to the built-in array and merged by a second kernel into out / group_mass.
+ * Limits: at most ENL_STATIC_MAX_SEGMENTS segments, ENL_STATIC_MAX_KEYS keys in all, 8 q heads per
+ * kv head, and partials that fit the array (n_q_heads * (head_dim + n_seg + 2) * 4 bytes per
+ * 1024 keys); anything larger returns ENL_E_LIMIT and enqueues nothing.
+ *
+ * The first call on a device looks up the array's device address (cudaGetSymbolAddress, with that
+ * device current) and keeps it; make that first call outside any stream capture.  All calls share the
+ * one array and it keeps the previous call's partials: a call overwrites everything it later reads,
+ * so back-to-back calls on one stream are fine, but two calls whose kernels overlap on the GPU
+ * (different streams, no dependency) race on it and give wrong results.  Use one stream, or order the
+ * calls with events.
+ * Errors: ENL_E_INVAL (null pointer, bad shape, negative length), ENL_E_LIMIT, ENL_E_CUDA.
+ */
+int enl_attend_static(const enl_static_args_t *args, void *cuda_stream);
 
 #ifdef __cplusplus
 }

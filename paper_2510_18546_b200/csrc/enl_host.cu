@@ -139,6 +139,7 @@ extern "C" const char *enl_strerror(int code)
         case ENL_E_NOMEM: return "out of pool pages, plan space or memory";
         case ENL_E_CUDA: return "CUDA error, or GPU operation on a bookkeeping-only cache";
         case ENL_E_TIMEOUT: return "a bounded wait inside a kernel expired";
+        case ENL_E_LIMIT: return "size beyond the fixed maxima of the entry point that allocates nothing";
         default: return "unknown error";
     }
 }

@@ -19,10 +19,11 @@ ENL_BF16 = 1
 ENL_DEVICE_NONE = -1
 ENL_REPLACE, ENL_APPEND = 0, 1
 ENL_PLAN_ONLY = 1
-ENL_OK, ENL_E_INVAL, ENL_E_NOGROUP, ENL_E_NOMEM, ENL_E_CUDA, ENL_E_TIMEOUT = 0, -1, -2, -3, -4, -5
+ENL_OK, ENL_E_INVAL, ENL_E_NOGROUP, ENL_E_NOMEM, ENL_E_CUDA, ENL_E_TIMEOUT, ENL_E_LIMIT = 0, -1, -2, -3, -4, -5, -6
+ENL_STATIC_MAX_SEGMENTS, ENL_STATIC_MAX_KEYS, ENL_STATIC_SCRATCH_BYTES = 255, 65536, 4 << 20
 
 EXPORTS = ("enl_cache_create", "enl_group_store", "enl_attend", "enl_cache_free", "enl_strerror",
-           "enl_group_len", "enl_cache_status", "enl_plan_inspect")
+           "enl_group_len", "enl_cache_status", "enl_plan_inspect", "enl_attend_static")
 
 
 class CacheDesc(ctypes.Structure):
@@ -40,6 +41,13 @@ class AttendArgs(ctypes.Structure):
                 ("q", ctypes.c_void_p), ("k_new", ctypes.c_void_p), ("v_new", ctypes.c_void_p),
                 ("out", ctypes.c_void_p), ("group_mass", ctypes.c_void_p), ("mass_stride", ctypes.c_int32),
                 ("sel_off_out", ctypes.c_void_p), ("split_hint", ctypes.c_int32), ("flags", ctypes.c_uint32)]
+
+
+class StaticArgs(ctypes.Structure):
+    _fields_ = [("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32),
+                ("n_seg", ctypes.c_int32), ("seg_len", ctypes.c_void_p), ("n_new", ctypes.c_int32),
+                ("q", ctypes.c_void_p), ("k", ctypes.c_void_p), ("v", ctypes.c_void_p), ("out", ctypes.c_void_p),
+                ("group_mass", ctypes.c_void_p)]
 
 
 class EnlError(RuntimeError):
@@ -75,6 +83,8 @@ def lib() -> ctypes.CDLL:
                                        ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p,
                                        ctypes.c_void_p, ctypes.c_void_p]
         L.enl_plan_inspect.restype = ctypes.c_int
+        L.enl_attend_static.argtypes = [ctypes.POINTER(StaticArgs), ctypes.c_void_p]
+        L.enl_attend_static.restype = ctypes.c_int
         _lib = L
     return _lib
 
@@ -142,6 +152,22 @@ def enl_attend(cache: int, layer: int, sel_ids: Sequence[int], q, k_new, v_new, 
     if rc != ENL_OK:
         raise EnlError(rc, "enl_attend")
     return so
+
+
+def enl_attend_static(seg_len: Sequence[int], n_new: int, q, k, v, out, group_mass=None, stream: int = 0) -> None:
+    """One query token over contiguous caller-owned K/V, for callers that must not allocate: the library
+    keeps its split-KV partials in a fixed built-in device array instead of allocated scratch.
+    ``q``/``out``: ``[Hq, D]`` bf16; ``k``/``v``: ``[sum(seg_len) + n_new, Hkv, D]`` bf16;
+    ``group_mass``: ``[Hq, len(seg_len) + 1]`` fp32 or None.  Calls share the built-in array, so issue
+    them on one stream (or order them); sizes beyond the fixed maxima raise ``ENL_E_LIMIT``."""
+    sl = _i32(seg_len)
+    a = StaticArgs()
+    a.n_q_heads, a.n_kv_heads, a.head_dim = int(q.shape[-2]), int(k.shape[-2]), int(q.shape[-1])
+    a.n_seg, a.seg_len, a.n_new = len(sl), _np_ptr(sl) if len(sl) else None, int(n_new)
+    a.q, a.k, a.v, a.out, a.group_mass = _ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(group_mass)
+    rc = lib().enl_attend_static(ctypes.byref(a), stream or None)
+    if rc != ENL_OK:
+        raise EnlError(rc, "enl_attend_static")
 
 
 def enl_cache_free(cache: int) -> None:
