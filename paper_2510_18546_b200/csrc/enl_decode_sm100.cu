@@ -1,0 +1,624 @@
+// Split-KV attention for one-token decode steps, sm_100a: an HBM-streaming kernel.
+//
+// What it computes (paper, App. A: decoding attends with the one new query over the concatenated K/V;
+// Sec. 3.2: the cached part is the selected groups' K/V; Sec. 3.3: per-group attention mass): for one
+// episode, one kv head and one range of the episode's key stream (16-token pages of the selected groups
+// in list order, then the new-token keys), the partial attention of the rep q heads that read this kv
+// head -- partial output normalised by the range's own sum, the range's log2-sum-exp and a per-slot
+// log2-sum-exp -- which the split merge kernel turns into the output row and the group masses.
+//
+// Every K and V page is read from HBM exactly once: each of the CTA's 12 warps owns a contiguous run of
+// the CTA's pages and a private ring of TMA stages (one page of one head = 16 rows x D bf16, 128-byte
+// swizzle) fed by its lane 0 in the order K0 V0 K1 V1 ...  Per page, all in registers:
+//   S = Q K^T      mma.sync, A = the rep query rows padded to 16, B = the K page (ldmatrix)
+//   p = exp2(S-m)  running maximum per head kept by the warp, O and the sums rescaled when it grows
+//   O += P V       mma.sync, A = P straight from the S accumulators, B = the V page (ldmatrix.trans)
+// A page belongs to one slot (a selected group, or the new tokens), so the slot sums are running sums
+// that are parked, as log2 values, whenever the slot changes.  No CTA barrier inside the stream.
+// At the end the warps are merged through shared memory; with several splits the CTA that finishes
+// last for its (episode, kv head) merges the splits' partial results (a counter per pair, reset by
+// that CTA), so a decode step is one launch.
+// The arithmetic intensity is 4 flop per byte, so the tensor work is noise; the roof is HBM bandwidth.
+// Code outside the streaming loop runs once per CTA from a cold instruction cache (the K/V stream has
+// pushed it out of L2 since the last launch), so those loops are kept rolled: their size is their cost.
+#include <cuda_bf16.h>
+
+#include "enl_internal.h"
+
+namespace enl {
+namespace {
+
+constexpr int kWarps   = 12;                              // one CTA per SM; 384 threads leave 168 registers each
+constexpr int kThreads = kWarps * 32;
+constexpr int kStages  = 4;                               // TMA stages per warp: 192 KB in flight per SM (D = 128)
+constexpr int kMaxRep  = 8;                               // q heads per kv head (rows 8..15 of the MMA stay zero)
+constexpr int kMaxRun  = kDecodeMaxPages / kWarps + 1;    // pages one warp may own
+constexpr float kRescaleThreshold = 8.0f;                 // log2 units
+constexpr unsigned long long kWaitLimitNs = 1000ull * 1000ull * 1000ull;
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p)
+{
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait, warp-uniform result.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int32_t *status)
+{
+    bool ok = mbar_try_wait(bar, parity);
+    if (!ok) {
+        const unsigned long long t0 = global_ns();
+        uint32_t spins = 0;
+        while (!(ok = mbar_try_wait(bar, parity))) {
+            if ((++spins & 63u) == 0u) {
+                if (*abort_flag) break;
+                if (global_ns() - t0 > kWaitLimitNs) {
+                    *abort_flag = 1;
+                    atomicExch(status, 2);
+                    break;
+                }
+            }
+        }
+    }
+    return __all_sync(0xffffffffu, ok);
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tm, int x, int y, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *tm, int x, int y, int z, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4])
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t addr, uint32_t (&r)[4])
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+// D (fp32, m16n8) += A (bf16, m16k16, row) * B (bf16, k16n8, col).  Rows 8..15 of A are always zero here, so
+// the accumulators of those rows (z0, z1) stay zero and one pair serves every product.
+__device__ __forceinline__ void mma_bf16(float &d0, float &d1, float &z0, float &z1, uint32_t a0, uint32_t a2,
+                                         uint32_t b0, uint32_t b1)
+{
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+        : "+f"(d0), "+f"(d1), "+f"(z0), "+f"(z1)
+        : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ float ex2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float lg2(float x)
+{
+    float y;
+    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
+{
+    const __nv_bfloat162 b = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t *>(&b);
+}
+
+constexpr float kNegInf = -__builtin_huge_valf();
+
+// Shared memory: [ring: warp][stage][D*32 B] | per-warp slot log-sums | per-warp (m, l) | split weights | barriers
+template <int D>
+struct DecCfg {
+    static constexpr int kStageBytes = D * kPageTokens * 2;            // one page of one head: 4 KB (D=128) / 2 KB
+    static constexpr int kRingBytes  = kWarps * kStages * kStageBytes;
+    static constexpr int kWslotOff   = kRingBytes;                     // [warp][kMaxRun + 1][kMaxRep] float
+    static constexpr int kWslotBytes = kWarps * (kMaxRun + 1) * kMaxRep * 4;
+    static constexpr int kCslotOff   = kWslotOff + kWslotBytes;        // [kDecodeMaxPages + 1][kMaxRep] float
+    static constexpr int kCslotBytes = (kDecodeMaxPages + 1) * kMaxRep * 4;
+    static constexpr int kMiscOff    = kCslotOff + kCslotBytes;
+    // wm[warp][rep], wl[warp][rep], wfirst[warp], wcnt[warp], cm[rep], cl[rep], weights[rep][kMaxSplits], flags[4]
+    static constexpr int kMiscBytes  = (2 * kWarps * kMaxRep + 2 * kWarps + 2 * kMaxRep + kMaxRep * kMaxSplits + 4) * 4;
+    static constexpr int kBarOff     = (kMiscOff + kMiscBytes + 15) & ~15;
+    static constexpr int kSmemBytes  = kBarOff + kWarps * kStages * 8 + 1024;   // + alignment slack
+};
+
+template <int D>
+__global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_constant__ DecodeParams p)
+{
+    using C = DecCfg<D>;
+    constexpr int kChunks = D / 8;                        // 16-byte chunks per row
+    constexpr int kHalves = D / 64;                       // TMA boxes (64 channels) per page
+    constexpr int kNB     = D / 8;                        // n-blocks of the PV product
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t sbase = (raw + 1023u) & ~1023u;
+    uint8_t *smem = smem_raw + (sbase - raw);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = lane >> 2, tq = lane & 3;               // MMA row group and thread-in-group
+    float *wslot = reinterpret_cast<float *>(smem + C::kWslotOff);
+    float *cslot = reinterpret_cast<float *>(smem + C::kCslotOff);
+    float *wm = reinterpret_cast<float *>(smem + C::kMiscOff);                // [warp][kMaxRep]
+    float *wl = wm + kWarps * kMaxRep;
+    int *wfirst = reinterpret_cast<int *>(wl + kWarps * kMaxRep);             // first slot of the warp's run
+    int *wcnt = wfirst + kWarps;                                              // slots the warp parked
+    float *cm = reinterpret_cast<float *>(wcnt + kWarps);                     // CTA (later: merged) log2-sum-exp reference
+    float *cl = cm + kMaxRep;
+    float *weights = cl + kMaxRep;                                            // [kMaxRep][kMaxSplits]
+    volatile int *flags = reinterpret_cast<volatile int *>(weights + kMaxRep * kMaxSplits);   // [0] abort, [1] last
+    volatile int *abort_flag = flags;
+    const uint32_t bar0 = sbase + C::kBarOff;
+    auto bar_full = [&](int s) { return bar0 + 8u * (warp * kStages + s); };
+    auto stage_addr = [&](int s) { return sbase + static_cast<uint32_t>((warp * kStages + s) * C::kStageBytes); };
+
+    // grid = (splits, kv heads, episodes); a single episode travels in the parameters
+    struct { int ep, kvh, split; } it = {static_cast<int>(blockIdx.z), static_cast<int>(blockIdx.y), static_cast<int>(blockIdx.x)};
+    EpInfo ep;
+    if (gridDim.z == 1) {
+        ep = p.ep0;
+    } else {
+        const int4 *src = reinterpret_cast<const int4 *>(p.eps + it.ep);
+        const int4 e0 = __ldg(src), e1 = __ldg(src + 1);
+        ep.stream_off = e0.x; ep.n_ctiles = e0.y; ep.n_slots = e0.z; ep.q_off = e0.w;
+        ep.n_q = e1.x; ep.new_off = e1.y; ep.n_new = e1.z; ep.pad = e1.w;
+    }
+    if (threadIdx.x == 0) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&p.tm_kpool) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&p.tm_vpool) : "memory");
+    }
+    const int rep = p.rep;
+    const int n_cached = ep.n_ctiles * kPagesPerTile;                         // cached stream entries (padded)
+    const int n_newp = (ep.n_new + kPageTokens - 1) / kPageTokens;            // pages of new-token keys
+    const int total = n_cached + n_newp;
+    const int pg_beg = static_cast<int>(static_cast<long long>(total) * it.split / p.n_splits);
+    const int pg_end = static_cast<int>(static_cast<long long>(total) * (it.split + 1) / p.n_splits);
+    const int n_cta = pg_end - pg_beg;                                        // <= kDecodeMaxPages (host guarantees)
+    // this warp's run of pages, CTA-relative [w_beg, w_end)
+    const int w_beg = n_cta * warp / kWarps, w_end = n_cta * (warp + 1) / kWarps;
+    const int n_w = w_end - w_beg;
+    const int G = ep.n_slots;
+
+    auto entry_meta = [&](int e) -> int {                                     // slot << 8 | valid keys
+        if (e < n_cached) return __ldg(p.stream_meta + ep.stream_off + e);
+        const int i = e - n_cached;
+        return (G << 8) | min(kPageTokens, ep.n_new - i * kPageTokens);
+    };
+
+    if (threadIdx.x == 0) { flags[0] = 0; flags[1] = 0; }
+    if (lane == 0) {
+        for (int s = 0; s < kStages; ++s) mbar_init(bar_full(s), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+
+    // lane j keeps the page id and the meta word of entry j of this warp's run (n_w <= 32): one coalesced
+    // load up front, so that no global load sits between a stage becoming free and its refill
+    int my_page = 0, my_meta = 0;
+    if (lane < n_w) {
+        const int e = pg_beg + w_beg + lane;
+        if (e < n_cached) {
+            my_page = __ldg(p.stream_page + ep.stream_off + e);
+            my_meta = __ldg(p.stream_meta + ep.stream_off + e);
+        } else {
+            my_page = -1 - (e - n_cached);                                   // new-token page, counted from the end
+            my_meta = entry_meta(e);
+        }
+    }
+    // load i of this warp: K page i/2 (i even) or V page i/2 (i odd); `page` as kept by lane i/2
+    auto issue = [&](int i, int page) {
+        const int st = i % kStages;
+        const bool is_v = i & 1;
+        const uint32_t full = bar_full(st), dst = stage_addr(st);
+        mbar_expect_tx(full, static_cast<uint32_t>(C::kStageBytes));
+        if (page >= 0) {
+            const CUtensorMap *tm = is_v ? &p.tm_vpool : &p.tm_kpool;
+            const int row = (page * p.Hkv + it.kvh) * kPageTokens;
+#pragma unroll
+            for (int hf = 0; hf < kHalves; ++hf) tma_load_2d(dst + hf * (kPageTokens * 128), tm, hf * 64, row, full);
+        } else {
+            const CUtensorMap *tm = is_v ? &p.tm_vnew : &p.tm_knew;
+            const int krow = ep.new_off + (-1 - page) * kPageTokens;         // rows past the tensor's end read as zero
+#pragma unroll
+            for (int hf = 0; hf < kHalves; ++hf)
+                tma_load_3d(dst + hf * (kPageTokens * 128), tm, hf * 64, it.kvh, krow, full);
+        }
+    };
+    const int n_loads = 2 * n_w;
+    int issued = 0;
+    for (; issued < min(kStages, n_loads); ++issued) {
+        const int pg = __shfl_sync(0xffffffffu, my_page, issued >> 1);
+        if (lane == 0) issue(issued, pg);
+    }
+
+    // the query rows of this kv head as the A operand of S = Q K^T (rows >= rep stay zero)
+    uint32_t qa[D / 16][2];
+    {
+        const __nv_bfloat16 *qrow = static_cast<const __nv_bfloat16 *>(p.q) +
+                                    (static_cast<long long>(ep.q_off) * p.Hq + it.kvh * rep + g) * D;
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks) {
+            qa[ks][0] = (g < rep) ? *reinterpret_cast<const uint32_t *>(qrow + ks * 16 + 2 * tq) : 0u;
+            qa[ks][1] = (g < rep) ? *reinterpret_cast<const uint32_t *>(qrow + ks * 16 + 8 + 2 * tq) : 0u;
+        }
+    }
+    const float scale = p.scale_log2;
+    bool ok = true;
+    int consumed = 0;                                                        // loads consumed by this warp
+
+    // called by the whole warp after it has read stage (consumed % kStages) for the last time
+    auto release_and_refill = [&]() {
+        const int pg = __shfl_sync(0xffffffffu, my_page, (issued >> 1) & 31);   // also orders the warp's reads
+        if (lane == 0 && issued < n_loads) {
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            issue(issued, pg);
+        }
+        if (issued < n_loads) ++issued;
+        ++consumed;
+    };
+
+    float o[kNB][2];
+#pragma unroll
+    for (int nb = 0; nb < kNB; ++nb) { o[nb][0] = o[nb][1] = 0.f; }
+    float z0 = 0.f, z1 = 0.f;               // accumulators of the unused MMA rows 8..15
+    float m = kNegInf;                      // running reference maximum of row g (same in the four lanes of a quad)
+    float lsum = 0.f, acc = 0.f;            // lane-local parts of the row sum and of the current slot's sum
+    int cur_slot = -1, n_parked = 0;
+    const int slot_first_w = __shfl_sync(0xffffffffu, my_meta, 0) >> 8;
+    float *my_wslot = wslot + warp * (kMaxRun + 1) * kMaxRep;
+    auto park = [&]() {                      // the slot that ends: log2 of its sum, absolute
+        float a = acc;
+        a += __shfl_xor_sync(0xffffffffu, a, 1);
+        a += __shfl_xor_sync(0xffffffffu, a, 2);
+        if (cur_slot >= 0) {
+            if (tq == 0 && g < kMaxRep) my_wslot[n_parked * kMaxRep + g] = (a > 0.f) ? lg2(a) + m : kNegInf;
+            ++n_parked;
+        }
+        acc = 0.f;
+    };
+
+    for (int i = 0; i < n_w && ok; ++i) {
+        // ---- S = Q K^T ----
+        int st = consumed % kStages;
+        ok = mbar_wait(bar_full(st), static_cast<uint32_t>((consumed / kStages) & 1), abort_flag, p.status);
+        if (!ok) break;
+        uint32_t base = stage_addr(st);
+        float c[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
+#pragma unroll
+        for (int nb = 0; nb < 2; ++nb) {
+            const int row = nb * 8 + (lane & 7);                             // token whose 16-byte chunks this lane addresses
+#pragma unroll
+            for (int kq = 0; kq < kChunks / 4; ++kq) {                       // four 8-channel chunks = two k16 steps
+                const int ch = kq * 4 + (lane >> 3);
+                const uint32_t addr = base + (ch >> 3) * (kPageTokens * 128) + row * 128 + (((ch & 7) ^ (row & 7)) << 4);
+                uint32_t b[4];
+                ldsm_x4(addr, b);
+                mma_bf16(c[nb][0], c[nb][1], z0, z1, qa[2 * kq][0], qa[2 * kq][1], b[0], b[1]);
+                mma_bf16(c[nb][0], c[nb][1], z0, z1, qa[2 * kq + 1][0], qa[2 * kq + 1][1], b[2], b[3]);
+            }
+        }
+        const int meta = __shfl_sync(0xffffffffu, my_meta, i);
+        const int nv = meta & 0xff, slot = meta >> 8;
+        const float s0 = (2 * tq < nv) ? c[0][0] * scale : kNegInf;
+        const float s1 = (2 * tq + 1 < nv) ? c[0][1] * scale : kNegInf;
+        const float s2 = (8 + 2 * tq < nv) ? c[1][0] * scale : kNegInf;
+        const float s3 = (8 + 2 * tq + 1 < nv) ? c[1][1] * scale : kNegInf;
+        release_and_refill();
+
+        // ---- p = exp2(S - m), sums ----
+        float mx = fmaxf(fmaxf(s0, s1), fmaxf(s2, s3));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+        if (slot != cur_slot) { park(); cur_slot = slot; }
+        if (__any_sync(0xffffffffu, mx > m + kRescaleThreshold)) {           // also when m is still -inf
+            const float m_new = fmaxf(m, mx);
+            const float alpha = (m == kNegInf) ? 0.f : ex2(m - m_new);      // nothing accumulated yet when m = -inf
+            if (m_new != m) {
+                lsum *= alpha;
+                acc *= alpha;
+            }
+            // rows g (o[.][0..1]) scale by this lane's alpha; rows g + 8 hold only zeros
+            const float a_row = (m_new != m) ? alpha : 1.f;
+#pragma unroll
+            for (int nb = 0; nb < kNB; ++nb) { o[nb][0] *= a_row; o[nb][1] *= a_row; }
+            m = m_new;
+        }
+        const float m_use = (m == kNegInf) ? 0.f : m;
+        const float p0 = ex2(s0 - m_use), p1 = ex2(s1 - m_use), p2 = ex2(s2 - m_use), p3 = ex2(s3 - m_use);
+        const float ps = (p0 + p1) + (p2 + p3);
+        acc += ps;
+        lsum += ps;
+        const uint32_t a0 = pack_bf16(p0, p1), a2 = pack_bf16(p2, p3);
+
+        // ---- O += P V ----
+        st = consumed % kStages;
+        ok = mbar_wait(bar_full(st), static_cast<uint32_t>((consumed / kStages) & 1), abort_flag, p.status);
+        if (!ok) break;
+        base = stage_addr(st);
+        const int row = ((lane >> 3) & 1) * 8 + (lane & 7);                  // token addressed by this lane
+#pragma unroll
+        for (int nq = 0; nq < kNB / 2; ++nq) {                               // two 8-channel n-blocks per ldmatrix
+            const int ch = nq * 2 + (lane >> 4);
+            const uint32_t addr = base + (ch >> 3) * (kPageTokens * 128) + row * 128 + (((ch & 7) ^ (row & 7)) << 4);
+            uint32_t b[4];
+            ldsm_x4_trans(addr, b);
+            mma_bf16(o[2 * nq][0], o[2 * nq][1], z0, z1, a0, a2, b[0], b[1]);
+            mma_bf16(o[2 * nq + 1][0], o[2 * nq + 1][1], z0, z1, a0, a2, b[2], b[3]);
+        }
+        release_and_refill();
+    }
+    park();
+
+    // error path only: let this warp's copies in flight land before the CTA retires
+    if (!ok) {
+        for (int f = consumed; f < issued; ++f) {
+            const unsigned long long t0 = global_ns();
+            while (!mbar_try_wait(bar_full(f % kStages), static_cast<uint32_t>((f / kStages) & 1)) &&
+                   global_ns() - t0 < 2000000ull) { }
+        }
+    }
+    lsum += __shfl_xor_sync(0xffffffffu, lsum, 1);
+    lsum += __shfl_xor_sync(0xffffffffu, lsum, 2);
+    if (tq == 0) { wm[warp * kMaxRep + g] = m; wl[warp * kMaxRep + g] = lsum; }
+    if (lane == 0) { wfirst[warp] = slot_first_w; wcnt[warp] = n_parked; }
+    __syncthreads();                                                         // every stage consumed: the ring is free
+    if (*abort_flag) return;
+
+    // ---- merge the warps: reference maximum, sum, output, slot log-sums of the CTA ----
+    float *obuf = reinterpret_cast<float *>(smem);                           // [warp][kMaxRep][D]
+    if (g < rep) {
+#pragma unroll
+        for (int nb = 0; nb < kNB; ++nb)
+            *reinterpret_cast<float2 *>(obuf + (warp * kMaxRep + g) * D + nb * 8 + 2 * tq) = make_float2(o[nb][0], o[nb][1]);
+    }
+    if (threadIdx.x < rep) {
+        const int h = threadIdx.x;
+        float M = kNegInf;
+#pragma unroll 1
+        for (int w = 0; w < kWarps; ++w) M = fmaxf(M, wm[w * kMaxRep + h]);
+        float Lh = 0.f;
+#pragma unroll 1
+        for (int w = 0; w < kWarps; ++w) {
+            const float mw = wm[w * kMaxRep + h];
+            const float f = (mw == kNegInf) ? 0.f : ex2(mw - M);
+            Lh += wl[w * kMaxRep + h] * f;
+            weights[h * kMaxSplits + w] = f;                                 // warp weights, reused below
+        }
+        cm[h] = M;
+        cl[h] = Lh;
+    }
+    int slot_first = 0x7fffffff, slot_end = 0;                                // slots the CTA's range touched
+#pragma unroll 1
+    for (int w = 0; w < kWarps; ++w)
+        if (wcnt[w] > 0) { slot_first = min(slot_first, wfirst[w]); slot_end = max(slot_end, wfirst[w] + wcnt[w]); }
+    const int n_local = (slot_end > 0) ? slot_end - slot_first : 0;
+    if (n_local == 0) slot_first = 0;
+    for (int idx = threadIdx.x; idx < n_local * rep; idx += kThreads) {
+        const int sl = idx / rep, h = idx % rep, s = slot_first + sl;
+        float mxv = kNegInf;
+#pragma unroll 1
+        for (int w = 0; w < kWarps; ++w) {
+            const int j = s - wfirst[w];
+            if (j >= 0 && j < wcnt[w]) mxv = fmaxf(mxv, wslot[(w * (kMaxRun + 1) + j) * kMaxRep + h]);
+        }
+        float sum = 0.f;
+        if (mxv != kNegInf)
+#pragma unroll 1
+            for (int w = 0; w < kWarps; ++w) {
+                const int j = s - wfirst[w];
+                if (j >= 0 && j < wcnt[w]) sum += ex2(wslot[(w * (kMaxRun + 1) + j) * kMaxRep + h] - mxv);
+            }
+        cslot[sl * kMaxRep + h] = (mxv != kNegInf) ? mxv + lg2(sum) : kNegInf;
+    }
+    __syncthreads();
+
+    const bool single = p.n_splits == 1;
+    const long long row_h0 = static_cast<long long>(ep.q_off) * p.Hq + it.kvh * rep;          // + h: (row, head) index
+    const long long rh0 = static_cast<long long>(it.split) * p.n_q_total * p.Hq + row_h0;     // + h: partial index
+    for (int idx = threadIdx.x; idx < rep * D; idx += kThreads) {
+        const int h = idx / D, ch = idx % D;
+        float v = 0.f;
+#pragma unroll 1
+        for (int w = 0; w < kWarps; ++w) v += obuf[(w * kMaxRep + h) * D + ch] * weights[h * kMaxSplits + w];
+        const float l = cl[h];
+        v = (l > 0.f) ? v / l : 0.f;
+        if (single) static_cast<__nv_bfloat16 *>(p.out)[(row_h0 + h) * D + ch] = __float2bfloat16_rn(v);
+        else p.part_o[(rh0 + h) * D + ch] = v;
+    }
+    if (single) {
+        if (p.mass)
+            for (int idx = threadIdx.x; idx < rep * (G + 1); idx += kThreads) {
+                const int h = idx / (G + 1), s = idx % (G + 1);
+                const float l = cl[h];
+                const float lse = (l > 0.f) ? cm[h] + lg2(l) : kNegInf;
+                float v = 0.f;
+                if (s >= slot_first && s < slot_first + n_local && lse != kNegInf) {
+                    const float x = cslot[(s - slot_first) * kMaxRep + h];
+                    if (x != kNegInf) v = ex2(x - lse);
+                }
+                p.mass[(row_h0 + h) * p.mass_stride + s] = v;
+            }
+        return;
+    }
+    if (threadIdx.x < rep) {
+        const float l = cl[threadIdx.x];
+        p.part_lse[rh0 + threadIdx.x] = (l > 0.f) ? cm[threadIdx.x] + lg2(l) : kNegInf;
+    }
+    if (p.part_slot)                                                         // only the slots this range touched
+        for (int idx = threadIdx.x; idx < rep * n_local; idx += kThreads) {
+            const int h = idx / n_local, sl = idx % n_local;
+            p.part_slot[(rh0 + h) * p.slot_stride + slot_first + sl] = cslot[sl * kMaxRep + h];
+        }
+
+    // ---- the last CTA of this (episode, kv head) merges the splits ----
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int *ctr = p.counters + it.ep * p.Hkv + it.kvh;
+        const int prev = atomicAdd(ctr, 1);
+        if (prev == p.n_splits - 1) {
+            flags[1] = 1;
+            *ctr = 0;                                                        // ready for the next launch
+        }
+    }
+    __syncthreads();
+    if (!flags[1]) return;
+    __threadfence();
+    const long long split_stride = static_cast<long long>(p.n_q_total) * p.Hq;
+    // weights of the splits: one warp per head
+    for (int h = warp; h < rep; h += kWarps) {
+        const float my0 = lane < p.n_splits ? __ldcg(p.part_lse + lane * split_stride + row_h0 + h) : kNegInf;
+        const float my1 = lane + 32 < p.n_splits ? __ldcg(p.part_lse + (lane + 32) * split_stride + row_h0 + h) : kNegInf;
+        float mxv = fmaxf(my0, my1);
+#pragma unroll
+        for (int of = 16; of > 0; of >>= 1) mxv = fmaxf(mxv, __shfl_xor_sync(0xffffffffu, mxv, of));
+        float sum = (my0 != kNegInf ? ex2(my0 - mxv) : 0.f) + (my1 != kNegInf ? ex2(my1 - mxv) : 0.f);
+#pragma unroll
+        for (int of = 16; of > 0; of >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, of);
+        const float lse = (mxv != kNegInf) ? mxv + lg2(sum) : kNegInf;
+        weights[h * kMaxSplits + lane] = (my0 != kNegInf) ? ex2(my0 - lse) : 0.f;
+        if (lane + 32 < kMaxSplits) weights[h * kMaxSplits + lane + 32] = (my1 != kNegInf) ? ex2(my1 - lse) : 0.f;
+        if (lane == 0) cm[h] = lse;
+    }
+    // per-slot table in the idle ring (behind the reduction buffer), zeroed before the barrier
+    constexpr int kRedFloats = kThreads * 4;
+    float *red = reinterpret_cast<float *>(smem);                            // [group][rep * D] partial outputs
+    float *tab = red + kRedFloats;                                           // [rep][G + 1]
+    constexpr int kTabCap = (C::kRingBytes - kRedFloats * 4) / 4;
+    const bool tab_fits = rep * (G + 1) <= kTabCap;
+    if (p.mass && tab_fits)
+        for (int idx = threadIdx.x; idx < rep * (G + 1); idx += kThreads) tab[idx] = 0.f;
+    __syncthreads();
+
+    // output: the rep rows of split k are rep * D contiguous floats; float4 f of split k goes to thread
+    // (k mod groups, f), every load independent of the others
+    const int n_f4 = rep * D / 4;
+    const int groups = max(1, kThreads / n_f4);
+    const int grp = threadIdx.x / n_f4, f = threadIdx.x % n_f4;
+    for (int f0 = 0; f0 < n_f4; f0 += kThreads) {                            // one trip unless rep * D > 1024
+        const int ff = f0 + f;
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (grp < groups && ff < n_f4) {
+            const int h = ff / (D / 4);
+#pragma unroll 4
+            for (int k = grp; k < p.n_splits; k += groups) {
+                const float w = weights[h * kMaxSplits + k];
+                const float4 v = __ldcg(reinterpret_cast<const float4 *>(p.part_o + (k * split_stride + row_h0) * D) + ff);
+                a.x += w * v.x; a.y += w * v.y; a.z += w * v.z; a.w += w * v.w;
+            }
+            *reinterpret_cast<float4 *>(red + (grp * n_f4 + f) * 4) = a;
+        }
+        __syncthreads();
+        if (threadIdx.x < n_f4 && ff < n_f4) {
+            float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int gi = 0; gi < groups; ++gi) {
+                const float4 v = *reinterpret_cast<const float4 *>(red + (gi * n_f4 + f) * 4);
+                t.x += v.x; t.y += v.y; t.z += v.z; t.w += v.w;
+            }
+            uint2 o2;
+            o2.x = pack_bf16(t.x, t.y);
+            o2.y = pack_bf16(t.z, t.w);
+            *reinterpret_cast<uint2 *>(static_cast<__nv_bfloat16 *>(p.out) + row_h0 * D + ff * 4) = o2;
+        }
+        __syncthreads();
+    }
+    if (!p.mass) return;
+    if (tab_fits) {
+        // every split contributes only the slots its range touched
+        for (int k = warp; k < p.n_splits; k += kWarps) {
+            const int kb = static_cast<int>(static_cast<long long>(total) * k / p.n_splits);
+            const int ke = static_cast<int>(static_cast<long long>(total) * (k + 1) / p.n_splits);
+            if (ke <= kb) continue;
+            const int first = entry_meta(kb) >> 8, cnt = (entry_meta(ke - 1) >> 8) - first + 1;
+            for (int idx = lane; idx < cnt * rep; idx += 32) {
+                const int h = idx / cnt, sl = idx % cnt;
+                const float lse = cm[h];
+                const float x = __ldcg(p.part_slot + (k * split_stride + row_h0 + h) * p.slot_stride + first + sl);
+                if (lse != kNegInf && x != kNegInf) atomicAdd(&tab[h * (G + 1) + first + sl], ex2(x - lse));
+            }
+        }
+        __syncthreads();
+        for (int idx = threadIdx.x; idx < rep * (G + 1); idx += kThreads) {
+            const int h = idx / (G + 1), sidx = idx % (G + 1);
+            p.mass[(row_h0 + h) * p.mass_stride + sidx] = tab[idx];
+        }
+    } else {
+        // more slots than the table holds: one thread per (head, slot), splits in order
+        for (int idx = threadIdx.x; idx < rep * (G + 1); idx += kThreads) {
+            const int h = idx / (G + 1), sidx = idx % (G + 1);
+            const float lse = cm[h];
+            float v = 0.f;
+            for (int k = 0; k < p.n_splits; ++k) {
+                const int kb = static_cast<int>(static_cast<long long>(total) * k / p.n_splits);
+                const int ke = static_cast<int>(static_cast<long long>(total) * (k + 1) / p.n_splits);
+                if (ke <= kb) continue;
+                const int first = entry_meta(kb) >> 8, last = entry_meta(ke - 1) >> 8;
+                if (sidx < first || sidx > last) continue;
+                const float x = __ldcg(p.part_slot + (k * split_stride + row_h0 + h) * p.slot_stride + sidx);
+                if (lse != kNegInf && x != kNegInf) v += ex2(x - lse);
+            }
+            p.mass[(row_h0 + h) * p.mass_stride + sidx] = v;
+        }
+    }
+}
+
+}  // namespace
+
+size_t decode_smem_bytes(int head_dim)
+{
+    return head_dim == 128 ? DecCfg<128>::kSmemBytes : DecCfg<64>::kSmemBytes;
+}
+
+cudaError_t prepare_decode(int head_dim)
+{
+    if (head_dim == 128)
+        return cudaFuncSetAttribute(decode_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, DecCfg<128>::kSmemBytes);
+    if (head_dim == 64)
+        return cudaFuncSetAttribute(decode_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, DecCfg<64>::kSmemBytes);
+    return cudaErrorInvalidValue;
+}
+
+cudaError_t launch_decode(const DecodeParams &p, int head_dim, int batch, cudaStream_t st)
+{
+    if (batch <= 0 || p.n_splits <= 0) return cudaSuccess;
+    const dim3 grid(p.n_splits, p.Hkv, batch);
+    if (head_dim == 128)
+        decode_kernel<128><<<grid, kThreads, DecCfg<128>::kSmemBytes, st>>>(p);
+    else if (head_dim == 64)
+        decode_kernel<64><<<grid, kThreads, DecCfg<64>::kSmemBytes, st>>>(p);
+    else
+        return cudaErrorInvalidValue;
+    return cudaGetLastError();
+}
+
+}  // namespace enl

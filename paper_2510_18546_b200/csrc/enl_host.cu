@@ -3,6 +3,7 @@
 #include <algorithm>
 #include <cstdio>
 #include <cstring>
+#include <cstdlib>
 #include <new>
 #include <vector>
 
@@ -60,9 +61,11 @@ bool encode_map(CUtensorMap *tm, const void *base, int rank, const cuuint64_t *d
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) return false;
     cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    static int promo = -1;
+    if (promo < 0) { const char *e = getenv("ENL_L2PROMO"); promo = e ? atoi(e) : 3; }
     return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, static_cast<cuuint32_t>(rank), const_cast<void *>(base), dims,
               strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+              static_cast<CUtensorMapL2promotion>(promo), CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
@@ -90,6 +93,7 @@ struct enl_cache {
     uint64_t plan_epoch = 0;
     int32_t plan_split_hint = 0;
     bool plan_has_mass = false;
+    bool plan_decode = false;               // the plan is for the one-token decode kernel
     std::vector<int32_t> key_sel, key_cu, key_len;   // what the current plan was built from
     int32_t plan_entries = 0, plan_items = 0, plan_splits = 1, plan_batch = 0, plan_max_slots = 0;
     std::vector<int32_t> seen;              // duplicate detection stamps
@@ -97,6 +101,7 @@ struct enl_cache {
 
     float *scratch = nullptr;
     int32_t *status_dev = nullptr;
+    int32_t *counters_dev = nullptr;        // decode: finished splits per (episode, kv head)
 
     EpInfo *h_eps() { return reinterpret_cast<EpInfo *>(plan_host + off_eps); }
     Item *h_items() { return reinterpret_cast<Item *>(plan_host + off_items); }
@@ -119,6 +124,7 @@ void destroy(enl_cache *c)
         if (c->plan_host) cudaFreeHost(c->plan_host);
         if (c->scratch) cudaFree(c->scratch);
         if (c->status_dev) cudaFree(c->status_dev);
+        if (c->counters_dev) cudaFree(c->counters_dev);
         if (c->plan_copied) cudaEventDestroy(c->plan_copied);
     } else {
         delete[] c->plan_host;
@@ -204,10 +210,12 @@ extern "C" int enl_cache_create(const enl_cache_desc_t *desc, enl_cache_t **out)
                cudaMalloc(&c->plan_dev, c->plan_bytes) == cudaSuccess &&
                cudaMallocHost(&c->plan_host, c->plan_bytes) == cudaSuccess &&
                cudaMalloc(&c->scratch, static_cast<size_t>(d.scratch_bytes)) == cudaSuccess &&
-               cudaMalloc(&c->status_dev, sizeof(int32_t)) == cudaSuccess;
+               cudaMalloc(&c->status_dev, sizeof(int32_t)) == cudaSuccess &&
+               cudaMalloc(&c->counters_dev, sizeof(int32_t) * d.max_batch * d.n_kv_heads) == cudaSuccess;
     if (!okm) { cudaGetLastError(); destroy(c); return ENL_E_NOMEM; }
     bool okc = cudaMemset(c->kpool, 0, pool_bytes) == cudaSuccess && cudaMemset(c->vpool, 0, pool_bytes) == cudaSuccess &&
                cudaMemset(c->status_dev, 0, sizeof(int32_t)) == cudaSuccess &&
+               cudaMemset(c->counters_dev, 0, sizeof(int32_t) * d.max_batch * d.n_kv_heads) == cudaSuccess &&
                cudaEventCreateWithFlags(&c->plan_copied, cudaEventDisableTiming) == cudaSuccess &&
                cudaEventRecord(c->plan_copied, 0) == cudaSuccess;
     if (!okc) { cudaGetLastError(); destroy(c); return ENL_E_CUDA; }
@@ -225,7 +233,7 @@ extern "C" int enl_cache_create(const enl_cache_desc_t *desc, enl_cache_t **out)
             return ENL_E_CUDA;
         }
     }
-    if (prepare_attention(d.head_dim) != cudaSuccess) { cudaGetLastError(); destroy(c); return ENL_E_CUDA; }
+    if (prepare_attention(d.head_dim) != cudaSuccess || prepare_decode(d.head_dim) != cudaSuccess) { cudaGetLastError(); destroy(c); return ENL_E_CUDA; }
     if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); destroy(c); return ENL_E_CUDA; }
     *out = c;
     return ENL_OK;
@@ -256,6 +264,8 @@ extern "C" int enl_cache_status(enl_cache_t *c)
     if (cudaMemcpy(&st, c->status_dev, sizeof st, cudaMemcpyDeviceToHost) != cudaSuccess) return ENL_E_CUDA;
     if (st != 0) {
         cudaMemset(c->status_dev, 0, sizeof st);
+        // a decode launch that gave up may have left its split counters half counted
+        cudaMemset(c->counters_dev, 0, sizeof(int32_t) * c->d.max_batch * c->d.n_kv_heads);
         return ENL_E_TIMEOUT;
     }
     return ENL_OK;
@@ -411,16 +421,40 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
         }
         if (n_entries > c->cap_entries || base_items > c->cap_items) return ENL_E_NOMEM;
 
-        int n_splits = 1;
-        if (a->split_hint >= 1) n_splits = a->split_hint;
-        else if (base_items < 120) n_splits = std::max(1, std::min(static_cast<int>(148 / base_items), min_tiles / 2));
-        n_splits = std::min<int64_t>(n_splits, std::max<int64_t>(1, c->cap_items / base_items));
-        n_splits = std::min(n_splits, 64);
         const int slot_stride = max_slots + 1;
-        while (n_splits > 1) {
-            const int64_t per_rh = d.head_dim + 1 + (has_mass ? slot_stride : 0);
-            if (static_cast<int64_t>(n_splits) * a->n_q * d.n_q_heads * per_rh * 4 <= d.scratch_bytes) break;
-            --n_splits;
+        const int64_t per_rh = d.head_dim + 1 + (has_mass ? slot_stride : 0);      // scratch floats per (split, row, head)
+        auto fits = [&](int ns) {
+            return static_cast<int64_t>(ns) * a->n_q * d.n_q_heads * per_rh * 4 <= d.scratch_bytes;
+        };
+        // One query token per episode: the streaming decode kernel, whose CTAs cover at most kDecodeMaxPages
+        // pages each and always hand their partial results to the merge kernel.
+        bool decode = c->rep <= 8;
+        int need = 1, fewest = 0x7fffffff;
+        for (int b = 0; b < B && decode; ++b) {
+            if (cu_q[b + 1] - cu_q[b] != 1) decode = false;
+            int64_t e = 0;
+            for (int s = cu_sel[b]; s < cu_sel[b + 1]; ++s) e += std::max(1, ceil_div(sel_len[s], kPageTokens));
+            e = (e + kPagesPerTile - 1) / kPagesPerTile * kPagesPerTile + ceil_div(cu_new[b + 1] - cu_new[b], kPageTokens);
+            need = std::max<int64_t>(need, (e + kDecodeMaxPages - 1) / kDecodeMaxPages);
+            fewest = std::min<int64_t>(fewest, e);
+        }
+        int n_splits = 1;
+        if (decode) {
+            const int slots = 148;                                                // one CTA per SM, one wave
+            n_splits = a->split_hint >= 1 ? a->split_hint : std::max(1, slots / (B * d.n_kv_heads));
+            n_splits = std::min(std::min(std::max(n_splits, need), fewest), kMaxSplits);
+            while (n_splits > need && !fits(n_splits)) --n_splits;
+            if (n_splits < need || !fits(n_splits) ||
+                static_cast<int64_t>(B) * d.n_kv_heads * n_splits > c->cap_items)
+                decode = false;                                                    // too long for one merge: general kernel
+        }
+        if (!decode) {
+            n_splits = 1;
+            if (a->split_hint >= 1) n_splits = a->split_hint;
+            else if (base_items < 120) n_splits = std::max(1, std::min(static_cast<int>(148 / base_items), min_tiles / 2));
+            n_splits = std::min<int64_t>(n_splits, std::max<int64_t>(1, c->cap_items / base_items));
+            n_splits = std::min(n_splits, kMaxSplits);
+            while (n_splits > 1 && !fits(n_splits)) --n_splits;
         }
 
         if (c->gpu && cudaEventSynchronize(c->plan_copied) != cudaSuccess) { cudaGetLastError(); return ENL_E_CUDA; }
@@ -458,7 +492,10 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
         struct Work { Item it; int tiles; };
         std::vector<Work> work;
         work.reserve(static_cast<size_t>(base_items) * n_splits);
-        for (int b = 0; b < B; ++b) {
+        for (int b = 0; b < B && decode; ++b)
+            for (int h = 0; h < d.n_kv_heads; ++h)
+                for (int sp = 0; sp < n_splits; ++sp) work.push_back({Item{b, h, 0, sp}, eps[b].n_ctiles});
+        for (int b = 0; b < B && !decode; ++b) {
             const EpInfo &e = eps[b];
             for (int t0 = 0; t0 < e.n_q; t0 += tpc) {
                 const int t_hi = std::min(t0 + tpc, e.n_q);
@@ -479,6 +516,7 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
         c->plan_epoch = c->epoch;
         c->plan_split_hint = a->split_hint;
         c->plan_has_mass = has_mass;
+        c->plan_decode = decode;
         c->key_sel.assign(a->sel_ids, a->sel_ids + a->n_sel);
         c->key_cu = cu_key;
         c->key_len = sel_len;
@@ -501,6 +539,44 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
                    cudaEventRecord(c->plan_copied, st) == cudaSuccess;
         if (!okc) { cudaGetLastError(); c->plan_valid = false; return ENL_E_CUDA; }
         c->plan_on_device = true;
+    }
+
+    const int slot_stride = c->plan_max_slots + 1;
+    if (c->plan_decode) {
+        DecodeParams dp;
+        std::memset(&dp, 0, sizeof dp);
+        const cuuint64_t nd[3] = {static_cast<cuuint64_t>(d.head_dim), static_cast<cuuint64_t>(d.n_kv_heads),
+                                  static_cast<cuuint64_t>(a->n_new)};
+        const cuuint64_t ns[2] = {static_cast<cuuint64_t>(d.head_dim) * 2,
+                                  static_cast<cuuint64_t>(d.head_dim) * 2 * d.n_kv_heads};
+        const cuuint32_t nb[3] = {64, 1, kPageTokens};
+        if (!encode_map(&dp.tm_knew, a->k_new, 3, nd, ns, nb) || !encode_map(&dp.tm_vnew, a->v_new, 3, nd, ns, nb))
+            return ENL_E_CUDA;
+        dp.tm_kpool = c->tm_k[a->layer];
+        dp.tm_vpool = c->tm_v[a->layer];
+        dp.ep0 = c->h_eps()[0];
+        dp.eps = reinterpret_cast<const EpInfo *>(c->plan_dev + c->off_eps);
+        dp.stream_page = reinterpret_cast<const int32_t *>(c->plan_dev + c->off_stream);
+        dp.stream_meta = reinterpret_cast<const int32_t *>(c->plan_dev + c->off_meta);
+        dp.q = a->q;
+        dp.out = a->out;
+        dp.mass = a->group_mass;
+        const size_t rows = static_cast<size_t>(c->plan_splits) * a->n_q * d.n_q_heads;
+        dp.part_o = c->scratch;
+        dp.part_lse = c->scratch + rows * d.head_dim;
+        dp.part_slot = has_mass ? c->scratch + rows * (d.head_dim + 1) : nullptr;
+        dp.counters = c->counters_dev;
+        dp.status = c->status_dev;
+        dp.n_q_total = a->n_q;
+        dp.Hq = d.n_q_heads;
+        dp.Hkv = d.n_kv_heads;
+        dp.rep = c->rep;
+        dp.slot_stride = slot_stride;
+        dp.mass_stride = a->mass_stride;
+        dp.n_splits = c->plan_splits;
+        dp.scale_log2 = 1.4426950408889634f / sqrtf(static_cast<float>(d.head_dim));
+        if (launch_decode(dp, d.head_dim, c->plan_batch, st) != cudaSuccess) { cudaGetLastError(); return ENL_E_CUDA; }
+        return ENL_OK;
     }
 
     AttnParams p;
@@ -536,7 +612,6 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
     p.mass_stride = a->mass_stride;
     p.n_splits = c->plan_splits;
     p.scale_log2 = 1.4426950408889634f / sqrtf(static_cast<float>(d.head_dim));
-    const int slot_stride = c->plan_max_slots + 1;
     if (p.n_splits > 1) {
         const size_t rows = static_cast<size_t>(p.n_splits) * a->n_q * d.n_q_heads;
         p.part_o = c->scratch;

@@ -56,6 +56,34 @@ struct AttnParams {
     float   scale_log2;     // log2(e) / sqrt(D)
 };
 
+// Decode (one query token per episode): pages of the key stream one CTA may cover, and the most splits
+// the merge kernel takes.
+constexpr int kDecodeMaxPages = 256;
+constexpr int kMaxSplits      = 64;
+
+struct DecodeParams {
+    CUtensorMap tm_knew;    // [n_new][Hkv][D]   box {64, 1, 16}
+    CUtensorMap tm_vnew;
+    CUtensorMap tm_kpool;   // [pages*Hkv*16][D] box {64, 16}   (one layer)
+    CUtensorMap tm_vpool;
+    EpInfo ep0;             // episode 0 (used when the call has one episode; grid = splits x kv heads x episodes)
+    const EpInfo *eps;
+    const int32_t *stream_page;
+    const int32_t *stream_meta;
+    const void *q;          // bf16 [n_q][Hq][D], one row per episode
+    void   *out;            // bf16 [n_q][Hq][D]
+    float  *mass;           // fp32 or null
+    float  *part_o, *part_lse, *part_slot;      // as in AttnParams; part_slot is null when mass is
+    int32_t *counters;      // [episode][kv head], zero between launches: splits that have finished
+    int32_t *status;
+    int32_t n_q_total;
+    int32_t Hq, Hkv, rep;
+    int32_t slot_stride;    // row stride of part_slot
+    int32_t mass_stride;    // row stride of mass
+    int32_t n_splits;
+    float   scale_log2;
+};
+
 struct CombineParams {
     const float *part_o, *part_lse, *part_slot;
     void  *out;
@@ -70,6 +98,9 @@ struct CombineParams {
 // launchers (defined in the .cu files of the kernels)
 cudaError_t launch_attention(const AttnParams &p, int head_dim, int n_items, cudaStream_t st);
 cudaError_t launch_combine(const CombineParams &p, cudaStream_t st);
+cudaError_t launch_decode(const DecodeParams &p, int head_dim, int batch, cudaStream_t st);
+cudaError_t prepare_decode(int head_dim);
+size_t decode_smem_bytes(int head_dim);
 // Page ids of (part of) one group, passed by value to the scatter kernel.
 constexpr int kScatterPages = 64;
 struct PageRun {

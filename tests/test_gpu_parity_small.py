@@ -50,13 +50,20 @@ SMALL = {
     "decode_grown": dict(Hq=32, Hkv=8, D=128, pool=[[300, 17, 256]], sel=[[2, 0]], n_q=[1], n_new=[37]),
     "rep1": dict(Hq=2, Hkv=2, D=64, pool=[[20, 20]], sel=[[1, 0]], n_q=[140], n_new=[140]),
     "rep8": dict(Hq=8, Hkv=1, D=128, pool=[[20, 45]], sel=[[0, 1]], n_q=[40], n_new=[40]),
+    # one query token per episode: the streaming decode kernel
+    "decode_batch": dict(Hq=8, Hkv=2, D=128, pool=[[30, 60, 90], [5, 5, 5, 5], [200]],
+                         sel=[[2, 0], [0, 1, 2, 3], []], n_q=[1, 1, 1], n_new=[1, 10, 129]),
+    "decode_d64_rep8": dict(Hq=8, Hkv=1, D=64, pool=[[20, 45, 300]], sel=[[0, 1, 2]], n_q=[1], n_new=[33]),
+    "decode_rep1": dict(Hq=2, Hkv=2, D=64, pool=[[20, 0, 20]], sel=[[2, 1, 0]], n_q=[1], n_new=[16]),
+    "decode_many_pages": dict(Hq=16, Hkv=4, D=128, pool=[[1500, 700, 16, 1, 2300]], sel=[[4, 3, 0, 2, 1]],
+                              n_q=[1], n_new=[17]),
     "varlen_batch": dict(Hq=8, Hkv=2, D=128, pool=[[30, 60, 90], [5, 5, 5, 5], [200]],
                          sel=[[2, 0], [0, 1, 2, 3], []], n_q=[70, 3, 129], n_new=[70, 10, 129]),
 }
 
 
 @pytest.mark.parametrize("name", sorted(SMALL))
-@pytest.mark.parametrize("split", [0, 2])
+@pytest.mark.parametrize("split", [0, 2, 5])
 def test_small_shapes(name, split):
     c = SMALL[name]
     wl = synth.make_small(7, 1, c["Hq"], c["Hkv"], c["D"], c["pool"], c["sel"], c["n_q"], c["n_new"], name=name)
