@@ -128,6 +128,12 @@ __device__ __forceinline__ float lg2(float x)
     asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+__device__ __forceinline__ float rcp(float x)
+{
+    float y;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 {
     const __nv_bfloat162 b = __floats2bfloat162_rn(lo, hi);
@@ -414,8 +420,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
             Lh += wl[w * kMaxRep + h] * f;
             weights[h * kMaxSplits + w] = f;                                 // warp weights, reused below
         }
-        cm[h] = M;
-        cl[h] = Lh;
+        cm[h] = (Lh > 0.f) ? M + lg2(Lh) : kNegInf;                          // log2-sum-exp of the CTA's range
+        cl[h] = (Lh > 0.f) ? rcp(Lh) : 0.f;
     }
     int slot_first = 0x7fffffff, slot_end = 0;                                // slots the CTA's range touched
 #pragma unroll 1
@@ -445,22 +451,32 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
     const bool single = p.n_splits == 1;
     const long long row_h0 = static_cast<long long>(ep.q_off) * p.Hq + it.kvh * rep;          // + h: (row, head) index
     const long long rh0 = static_cast<long long>(it.split) * p.n_q_total * p.Hq + row_h0;     // + h: partial index
-    for (int idx = threadIdx.x; idx < rep * D; idx += kThreads) {
-        const int h = idx / D, ch = idx % D;
-        float v = 0.f;
+    const int n_f4 = rep * D / 4;                                             // the rep output rows as float4
+    for (int ff = threadIdx.x; ff < n_f4; ff += kThreads) {
+        const int h = ff / (D / 4);
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll 1
-        for (int w = 0; w < kWarps; ++w) v += obuf[(w * kMaxRep + h) * D + ch] * weights[h * kMaxSplits + w];
-        const float l = cl[h];
-        v = (l > 0.f) ? v / l : 0.f;
-        if (single) static_cast<__nv_bfloat16 *>(p.out)[(row_h0 + h) * D + ch] = __float2bfloat16_rn(v);
-        else p.part_o[(rh0 + h) * D + ch] = v;
+        for (int w = 0; w < kWarps; ++w) {
+            const float f = weights[h * kMaxSplits + w];
+            const float4 v = *reinterpret_cast<const float4 *>(obuf + w * kMaxRep * D + ff * 4);
+            a.x += f * v.x; a.y += f * v.y; a.z += f * v.z; a.w += f * v.w;
+        }
+        const float inv = cl[h];
+        a.x *= inv; a.y *= inv; a.z *= inv; a.w *= inv;
+        if (single) {
+            uint2 o2;
+            o2.x = pack_bf16(a.x, a.y);
+            o2.y = pack_bf16(a.z, a.w);
+            *reinterpret_cast<uint2 *>(static_cast<__nv_bfloat16 *>(p.out) + row_h0 * D + ff * 4) = o2;
+        } else {
+            *reinterpret_cast<float4 *>(p.part_o + rh0 * D + ff * 4) = a;
+        }
     }
     if (single) {
         if (p.mass)
             for (int idx = threadIdx.x; idx < rep * (G + 1); idx += kThreads) {
                 const int h = idx / (G + 1), s = idx % (G + 1);
-                const float l = cl[h];
-                const float lse = (l > 0.f) ? cm[h] + lg2(l) : kNegInf;
+                const float lse = cm[h];
                 float v = 0.f;
                 if (s >= slot_first && s < slot_first + n_local && lse != kNegInf) {
                     const float x = cslot[(s - slot_first) * kMaxRep + h];
@@ -470,10 +486,9 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
             }
         return;
     }
-    if (threadIdx.x < rep) {
-        const float l = cl[threadIdx.x];
-        p.part_lse[rh0 + threadIdx.x] = (l > 0.f) ? cm[threadIdx.x] + lg2(l) : kNegInf;
-    }
+    if (threadIdx.x < rep) p.part_lse[rh0 + threadIdx.x] = cm[threadIdx.x];
+    if (threadIdx.x == 0)
+        p.part_rng[(it.split * static_cast<int>(gridDim.z) + it.ep) * p.Hkv + it.kvh] = make_int2(slot_first, n_local);
     if (p.part_slot)                                                         // only the slots this range touched
         for (int idx = threadIdx.x; idx < rep * n_local; idx += kThreads) {
             const int h = idx / n_local, sl = idx % n_local;
@@ -495,8 +510,26 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
     if (!flags[1]) return;
     __threadfence();
     const long long split_stride = static_cast<long long>(p.n_q_total) * p.Hq;
-    // weights of the splits: one warp per head
-    for (int h = warp; h < rep; h += kWarps) {
+    // Round trip 1, everything that does not depend on anything else: the first partial outputs of every
+    // thread, the splits' slot ranges (lane j of warp w keeps split w + j * kWarps) and the log-sum-exps.
+    constexpr int kBatch = 8;
+    const int groups = max(1, kThreads / n_f4);
+    const int grp = threadIdx.x / n_f4, f = threadIdx.x % n_f4;
+    const bool active = grp < groups;                                        // n_f4 <= kThreads for rep <= 8, D <= 128
+    const float4 *po4 = reinterpret_cast<const float4 *>(p.part_o + row_h0 * D) + f;
+    const long long po_stride4 = split_stride * D / 4;
+    float4 pv[kBatch];
+#pragma unroll
+    for (int j = 0; j < kBatch; ++j) {
+        const int k = grp + j * groups;
+        pv[j] = (active && k < p.n_splits) ? __ldcg(po4 + k * po_stride4) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    int2 my_rng = make_int2(0, 0);
+    {
+        const int k = warp + lane * kWarps;
+        if (k < p.n_splits) my_rng = __ldcg(p.part_rng + (k * static_cast<int>(gridDim.z) + it.ep) * p.Hkv + it.kvh);
+    }
+    for (int h = warp; h < rep; h += kWarps) {                               // weights of the splits: one warp per head
         const float my0 = lane < p.n_splits ? __ldcg(p.part_lse + lane * split_stride + row_h0 + h) : kNegInf;
         const float my1 = lane + 32 < p.n_splits ? __ldcg(p.part_lse + (lane + 32) * split_stride + row_h0 + h) : kNegInf;
         float mxv = fmaxf(my0, my1);
@@ -520,46 +553,11 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
         for (int idx = threadIdx.x; idx < rep * (G + 1); idx += kThreads) tab[idx] = 0.f;
     __syncthreads();
 
-    // output: the rep rows of split k are rep * D contiguous floats; float4 f of split k goes to thread
-    // (k mod groups, f), every load independent of the others
-    const int n_f4 = rep * D / 4;
-    const int groups = max(1, kThreads / n_f4);
-    const int grp = threadIdx.x / n_f4, f = threadIdx.x % n_f4;
-    for (int f0 = 0; f0 < n_f4; f0 += kThreads) {                            // one trip unless rep * D > 1024
-        const int ff = f0 + f;
-        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (grp < groups && ff < n_f4) {
-            const int h = ff / (D / 4);
-#pragma unroll 4
-            for (int k = grp; k < p.n_splits; k += groups) {
-                const float w = weights[h * kMaxSplits + k];
-                const float4 v = __ldcg(reinterpret_cast<const float4 *>(p.part_o + (k * split_stride + row_h0) * D) + ff);
-                a.x += w * v.x; a.y += w * v.y; a.z += w * v.z; a.w += w * v.w;
-            }
-            *reinterpret_cast<float4 *>(red + (grp * n_f4 + f) * 4) = a;
-        }
-        __syncthreads();
-        if (threadIdx.x < n_f4 && ff < n_f4) {
-            float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
-            for (int gi = 0; gi < groups; ++gi) {
-                const float4 v = *reinterpret_cast<const float4 *>(red + (gi * n_f4 + f) * 4);
-                t.x += v.x; t.y += v.y; t.z += v.z; t.w += v.w;
-            }
-            uint2 o2;
-            o2.x = pack_bf16(t.x, t.y);
-            o2.y = pack_bf16(t.z, t.w);
-            *reinterpret_cast<uint2 *>(static_cast<__nv_bfloat16 *>(p.out) + row_h0 * D + ff * 4) = o2;
-        }
-        __syncthreads();
-    }
-    if (!p.mass) return;
-    if (tab_fits) {
-        // every split contributes only the slots its range touched
-        for (int k = warp; k < p.n_splits; k += kWarps) {
-            const int kb = static_cast<int>(static_cast<long long>(total) * k / p.n_splits);
-            const int ke = static_cast<int>(static_cast<long long>(total) * (k + 1) / p.n_splits);
-            if (ke <= kb) continue;
-            const int first = entry_meta(kb) >> 8, cnt = (entry_meta(ke - 1) >> 8) - first + 1;
+    // Round trip 2: the slot log-sums of every split (only the slots its range touched)
+    if (p.mass && tab_fits) {
+        for (int j = 0; warp + j * kWarps < p.n_splits; ++j) {
+            const int k = warp + j * kWarps;
+            const int first = __shfl_sync(0xffffffffu, my_rng.x, j), cnt = __shfl_sync(0xffffffffu, my_rng.y, j);
             for (int idx = lane; idx < cnt * rep; idx += 32) {
                 const int h = idx / cnt, sl = idx % cnt;
                 const float lse = cm[h];
@@ -567,7 +565,40 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
                 if (lse != kNegInf && x != kNegInf) atomicAdd(&tab[h * (G + 1) + first + sl], ex2(x - lse));
             }
         }
-        __syncthreads();
+    }
+    // output: float4 f of split k goes to thread (k mod groups, f)
+    if (active) {
+        const int h = f / (D / 4);
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int j = 0; j < kBatch; ++j) {
+            const int k = grp + j * groups;
+            const float w = (k < p.n_splits) ? weights[h * kMaxSplits + k] : 0.f;
+            a.x += w * pv[j].x; a.y += w * pv[j].y; a.z += w * pv[j].z; a.w += w * pv[j].w;
+        }
+#pragma unroll 1
+        for (int k = grp + kBatch * groups; k < p.n_splits; k += groups) {   // more splits than one batch covers
+            const float w = weights[h * kMaxSplits + k];
+            const float4 v = __ldcg(po4 + k * po_stride4);
+            a.x += w * v.x; a.y += w * v.y; a.z += w * v.z; a.w += w * v.w;
+        }
+        *reinterpret_cast<float4 *>(red + (grp * n_f4 + f) * 4) = a;
+    }
+    __syncthreads();
+    if (threadIdx.x < n_f4) {
+        float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 1
+        for (int gi = 0; gi < groups; ++gi) {
+            const float4 v = *reinterpret_cast<const float4 *>(red + (gi * n_f4 + f) * 4);
+            t.x += v.x; t.y += v.y; t.z += v.z; t.w += v.w;
+        }
+        uint2 o2;
+        o2.x = pack_bf16(t.x, t.y);
+        o2.y = pack_bf16(t.z, t.w);
+        *reinterpret_cast<uint2 *>(static_cast<__nv_bfloat16 *>(p.out) + row_h0 * D + f * 4) = o2;
+    }
+    if (!p.mass) return;
+    if (tab_fits) {
         for (int idx = threadIdx.x; idx < rep * (G + 1); idx += kThreads) {
             const int h = idx / (G + 1), sidx = idx % (G + 1);
             p.mass[(row_h0 + h) * p.mass_stride + sidx] = tab[idx];
@@ -578,12 +609,10 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
             const int h = idx / (G + 1), sidx = idx % (G + 1);
             const float lse = cm[h];
             float v = 0.f;
+#pragma unroll 1
             for (int k = 0; k < p.n_splits; ++k) {
-                const int kb = static_cast<int>(static_cast<long long>(total) * k / p.n_splits);
-                const int ke = static_cast<int>(static_cast<long long>(total) * (k + 1) / p.n_splits);
-                if (ke <= kb) continue;
-                const int first = entry_meta(kb) >> 8, last = entry_meta(ke - 1) >> 8;
-                if (sidx < first || sidx > last) continue;
+                const int2 rng = __ldcg(p.part_rng + (k * static_cast<int>(gridDim.z) + it.ep) * p.Hkv + it.kvh);
+                if (sidx < rng.x || sidx >= rng.x + rng.y) continue;
                 const float x = __ldcg(p.part_slot + (k * split_stride + row_h0 + h) * p.slot_stride + sidx);
                 if (lse != kNegInf && x != kNegInf) v += ex2(x - lse);
             }

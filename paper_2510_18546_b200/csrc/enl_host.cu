@@ -3,7 +3,6 @@
 #include <algorithm>
 #include <cstdio>
 #include <cstring>
-#include <cstdlib>
 #include <new>
 #include <vector>
 
@@ -61,11 +60,9 @@ bool encode_map(CUtensorMap *tm, const void *base, int rank, const cuuint64_t *d
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) return false;
     cuuint32_t estr[5] = {1, 1, 1, 1, 1};
-    static int promo = -1;
-    if (promo < 0) { const char *e = getenv("ENL_L2PROMO"); promo = e ? atoi(e) : 3; }
     return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, static_cast<cuuint32_t>(rank), const_cast<void *>(base), dims,
               strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-              static_cast<CUtensorMapL2promotion>(promo), CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
@@ -423,8 +420,9 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
 
         const int slot_stride = max_slots + 1;
         const int64_t per_rh = d.head_dim + 1 + (has_mass ? slot_stride : 0);      // scratch floats per (split, row, head)
-        auto fits = [&](int ns) {
-            return static_cast<int64_t>(ns) * a->n_q * d.n_q_heads * per_rh * 4 <= d.scratch_bytes;
+        auto fits = [&](int ns) {      // partial O, log-sum-exp and slot log-sums, plus the decode kernel's slot ranges
+            return static_cast<int64_t>(ns) * a->n_q * d.n_q_heads * per_rh * 4 +
+                   static_cast<int64_t>(ns) * B * d.n_kv_heads * 8 + 16 <= d.scratch_bytes;
         };
         // One query token per episode: the streaming decode kernel, whose CTAs cover at most kDecodeMaxPages
         // pages each and always hand their partial results to the merge kernel.
@@ -565,6 +563,10 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
         dp.part_o = c->scratch;
         dp.part_lse = c->scratch + rows * d.head_dim;
         dp.part_slot = has_mass ? c->scratch + rows * (d.head_dim + 1) : nullptr;
+        {
+            const size_t used = rows * (d.head_dim + 1 + (has_mass ? slot_stride : 0));      // floats
+            dp.part_rng = reinterpret_cast<int2 *>(c->scratch + ((used + 1) & ~static_cast<size_t>(1)));
+        }
         dp.counters = c->counters_dev;
         dp.status = c->status_dev;
         dp.n_q_total = a->n_q;

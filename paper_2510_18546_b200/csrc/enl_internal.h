@@ -74,6 +74,7 @@ struct DecodeParams {
     void   *out;            // bf16 [n_q][Hq][D]
     float  *mass;           // fp32 or null
     float  *part_o, *part_lse, *part_slot;      // as in AttnParams; part_slot is null when mass is
+    int2   *part_rng;       // [split][episode][kv head]: first slot and number of slots the split's range touched
     int32_t *counters;      // [episode][kv head], zero between launches: splits that have finished
     int32_t *status;
     int32_t n_q_total;
