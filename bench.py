@@ -132,7 +132,9 @@ def oracle_sample(wl, seconds_target: float = 15.0):
     work, dt, n_calls, n_rows = 0.0, 0.0, 0, 0
     layer, t_dec = 0, wl.decode_steps - 1 if wl.decode_steps else 0
     row_budget = None
-    while dt < seconds_target and layer < wl.n_layers:
+    while dt < seconds_target and (layer < wl.n_layers or (wl.decode_steps and t_dec > 0)):
+        if layer >= wl.n_layers:                    # decode: all layers of this step done, take an earlier step
+            layer, t_dec = 0, t_dec - 1
         k, v = wl.pool_kv(layer, b, "cpu")
         ks = [k[offs[g]:offs[g + 1]] for g in wl.sel_local[b]]
         vs = [v[offs[g]:offs[g + 1]] for g in wl.sel_local[b]]
@@ -162,7 +164,7 @@ def oracle_sample(wl, seconds_target: float = 15.0):
         layer += 1
     if wl.decode_steps:
         value, unit = work / dt / 1e9, "GB/s"
-        what = f"step {t_dec} of layers 0..{n_calls - 1}"
+        what = f"{n_calls} (layer, step) pairs, steps {t_dec}..{wl.decode_steps - 1}, layers in order"
     else:
         value, unit = work / dt / 1e12, "TFLOP/s"
         what = f"layers 0..{n_calls - 1}, {n_rows} query rows in all"
@@ -328,7 +330,8 @@ def main():
     roofline = {"bound": bound, "achieved": achieved, "peak": peak, "unit": unit, "frac": achieved / peak,
                 "traffic": NCU_TRAFFIC_BYTES.get(wl.name), "peak_source": peaks["_source"] +
                 (" (sustained bf16 GEMM)" if bound == "tensor" else " (copy bandwidth)"),
-                "kernel": f"attn_kernel<{wl.head_dim}>" + (" + combine_kernel" if n_splits > 1 else ""),
+                "kernel": (f"decode_kernel<{wl.head_dim}> (split merge fused)" if wl.decode_steps else
+                           f"attn_kernel<{wl.head_dim}>" + (" + combine_kernel" if n_splits > 1 else "")),
                 "launch_ms": attend_ms,
                 "algorithmic_per_launch": per_launch}
 
@@ -390,7 +393,8 @@ def main():
         wl0 = synth.make(args.workload)
         _, _, _, cpu = oracle_sample(wl0)
 
-    launches_per_step = L * (1 + (1 if n_splits > 1 else 0)) + L      # attention (+ merge) + page scatter
+    # attention (+ merge kernel when the prefill kernel splits KV; the decode kernel merges in-kernel) + page scatter
+    launches_per_step = L * (1 + (1 if (n_splits > 1 and not wl.decode_steps) else 0)) + L
     enl.enl_cache_free(cache)
     if rank == 0:
         line = {"metric": metric_name(wl), "value": value, "unit": unit, "n_gpus": world, "steps": args.steps,

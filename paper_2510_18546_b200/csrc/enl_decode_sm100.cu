@@ -30,7 +30,7 @@ namespace {
 
 constexpr int kWarps   = 12;                              // one CTA per SM; 384 threads leave 168 registers each
 constexpr int kThreads = kWarps * 32;
-constexpr int kStages  = 4;                               // TMA stages per warp: 192 KB in flight per SM (D = 128)
+constexpr int kStages  = 2;                               // TMA stages per warp: K and V of one page; 96 KB in flight per SM (D = 128)
 constexpr int kMaxRep  = 8;                               // q heads per kv head (rows 8..15 of the MMA stay zero)
 constexpr int kMaxRun  = kDecodeMaxPages / kWarps + 1;    // pages one warp may own
 constexpr float kRescaleThreshold = 8.0f;                 // log2 units
@@ -84,17 +84,26 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
     return __all_sync(0xffffffffu, ok);
 }
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tm, int x, int y, uint32_t bar)
+// The K/V stream is read once: its lines are marked evict-first so that what is reused from launch to launch
+// (code, plan, partial results) stays in L2.
+__device__ __forceinline__ uint64_t policy_evict_first()
 {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(bar) : "memory");
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
 }
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *tm, int x, int y, int z, uint32_t bar)
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tm, int x, int y, uint32_t bar, uint64_t pol)
 {
     asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-        ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+        ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(bar), "l"(pol) : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *tm, int x, int y, int z, uint32_t bar,
+                                            uint64_t pol)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4}], [%5], %6;"
+        ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(z), "r"(bar), "l"(pol) : "memory");
 }
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4])
 {
@@ -241,6 +250,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
             my_meta = entry_meta(e);
         }
     }
+    const uint64_t pol = policy_evict_first();
     // load i of this warp: K page i/2 (i even) or V page i/2 (i odd); `page` as kept by lane i/2
     auto issue = [&](int i, int page) {
         const int st = i % kStages;
@@ -251,13 +261,13 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
             const CUtensorMap *tm = is_v ? &p.tm_vpool : &p.tm_kpool;
             const int row = (page * p.Hkv + it.kvh) * kPageTokens;
 #pragma unroll
-            for (int hf = 0; hf < kHalves; ++hf) tma_load_2d(dst + hf * (kPageTokens * 128), tm, hf * 64, row, full);
+            for (int hf = 0; hf < kHalves; ++hf) tma_load_2d(dst + hf * (kPageTokens * 128), tm, hf * 64, row, full, pol);
         } else {
             const CUtensorMap *tm = is_v ? &p.tm_vnew : &p.tm_knew;
             const int krow = ep.new_off + (-1 - page) * kPageTokens;         // rows past the tensor's end read as zero
 #pragma unroll
             for (int hf = 0; hf < kHalves; ++hf)
-                tma_load_3d(dst + hf * (kPageTokens * 128), tm, hf * 64, it.kvh, krow, full);
+                tma_load_3d(dst + hf * (kPageTokens * 128), tm, hf * 64, it.kvh, krow, full, pol);
         }
     };
     const int n_loads = 2 * n_w;
@@ -278,6 +288,10 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
             qa[ks][1] = (g < rep) ? *reinterpret_cast<const uint32_t *>(qrow + ks * 16 + 8 + 2 * tq) : 0u;
         }
     }
+    // Touch, while the first pages are on their way, every kernel parameter that is otherwise first read
+    // after the stream: a miss in the constant cache costs about a microsecond, and there it would be exposed.
+    asm volatile("" ::"l"(p.part_o), "l"(p.part_lse), "l"(p.part_slot), "l"(p.part_rng), "l"(p.counters), "l"(p.out),
+                 "l"(p.mass), "r"(p.n_q_total), "r"(p.mass_stride), "r"(p.slot_stride), "r"(p.n_splits), "r"(p.Hq));
     const float scale = p.scale_log2;
     bool ok = true;
     int consumed = 0;                                                        // loads consumed by this warp
