@@ -14,10 +14,14 @@
 // turns those into probabilities.  With KV splits every split writes partial results that a second
 // kernel merges.
 //
-// Roles: warps 0-3 softmax of Q tile 0, warps 4-7 softmax of Q tile 1, warp 8 TMA producer,
-// warp 9 MMA issuer (and TMEM owner), warps 10-11 idle (they complete the third warpgroup so that
-// setmaxnreg can move registers from it to the two softmax warpgroups, which hold a 128-column row of S).  TMEM columns: S0 [0,128) S1 [128,256) O0 [256,384) O1 [384,512);
-// P_i overwrites the first 64 columns of S_i.
+// Roles: 16 softmax warps -- Q tile i = warps 8i..8i+7, and within a tile warps 0-3 take key columns 0..63
+// of every S tile ("half A"), warps 4-7 columns 64..127 ("half B"), so that every row is shared by two
+// threads of two warps with the same TMEM lane quadrant; they exchange the row maximum (and half B's page
+// sums, which half A credits to the slots) through shared memory behind a two-warp mbarrier.  Four
+// softmax warps per scheduler overlap each other's exp2, max, pack and TMEM traffic.  Warp 16 is the TMA
+// producer, warp 17 the MMA issuer (and TMEM owner), warps 18-19 idle: they complete the fifth warpgroup
+// so that setmaxnreg can move registers to the softmax warpgroups.
+// TMEM columns: S0 [0,128) S1 [128,256) O0 [256,384) O1 [384,512); P_i overwrites the first 64 columns of S_i.
 #include <cuda_bf16.h>
 
 #include "enl_internal.h"
@@ -26,11 +30,12 @@
 namespace enl {
 namespace {
 
-constexpr int kThreads      = 384;
-constexpr int kRegsSoftmax  = 224;            // 2 softmax warps + 1 other warp per scheduler: 2*224 + 56 <= 512
-constexpr int kRegsOther    = 56;
-constexpr int kProducerWarp = 8;
-constexpr int kMmaWarp      = 9;
+constexpr int kThreads      = 640;
+constexpr int kSoftmaxWarps = 16;
+constexpr int kRegsSoftmax  = 104;            // the launch gives 640 x 96 registers; what warpgroup 4 releases (4 x 8 per thread) is what the four softmax warpgroups gain
+constexpr int kRegsOther    = 64;
+constexpr int kProducerWarp = 16;
+constexpr int kMmaWarp      = 17;
 constexpr uint32_t kTmemCols = 512;
 constexpr float kRescaleThreshold = 8.0f;     // log2 units: p stays below 2^8 between max updates
 constexpr unsigned long long kWaitLimitNs = 1000ull * 1000ull * 1000ull;
@@ -40,9 +45,14 @@ struct Cfg {
     static constexpr int kHalves    = D / 64;             // 64-channel (128-byte) column blocks
     static constexpr int kHalfBytes = 128 * 128;          // 128 rows x 128 B
     static constexpr int kTileBytes = kHalves * kHalfBytes;
-    static constexpr int kStages    = (D == 128) ? 5 : 8;
+    static constexpr int kStages    = (D == 128) ? 4 : 8;
     static constexpr int kBarOff    = (kQTiles + kStages) * kTileBytes;
-    static constexpr int kSmemBytes = kBarOff + 512 + 1024;   // barriers + alignment slack
+    // exchange area of the softmax thread pairs: row maxima [tile][half][128], half B's page sums
+    // [parity][tile][4][128], 1 / row sum [tile][128]
+    static constexpr int kXmaxOff   = kBarOff + 512;
+    static constexpr int kXsumOff   = kXmaxOff + kQTiles * 2 * 128 * 4;
+    static constexpr int kXinvOff   = kXsumOff + 2 * kQTiles * 4 * 128 * 4;
+    static constexpr int kSmemBytes = kXinvOff + kQTiles * 128 * 4 + 1024;   // + alignment slack
 };
 
 // ---- small PTX wrappers ------------------------------------------------------------------
@@ -78,19 +88,24 @@ __device__ __forceinline__ unsigned long long global_ns()
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-// Bounded wait: gives up after kWaitLimitNs or when another role has raised the abort flag.
+// Bounded wait: gives up about kWaitLimitNs after its 256th failed poll, or when another role has raised the abort flag.
 // The result is made warp-uniform so that warp-collective tcgen05 instructions stay converged.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
                                           int32_t *status)
 {
     bool ok = mbar_try_wait(bar, parity);
     if (!ok) {
-        const unsigned long long t0 = global_ns();
+        // the clock is read only every 256 failed polls (the first reading starts the limit): a poll already
+        // sleeps inside the instruction, and reading the global timer is far slower than a poll
+        unsigned long long t0 = 0;
         uint32_t spins = 0;
         while (!(ok = mbar_try_wait(bar, parity))) {
-            if ((++spins & 63u) == 0u) {
+            if ((++spins & 255u) == 0u) {
                 if (*abort_flag) break;
-                if (global_ns() - t0 > kWaitLimitNs) {
+                const unsigned long long now = global_ns();
+                if (t0 == 0) {
+                    t0 = now;
+                } else if (now - t0 > kWaitLimitNs) {
                     *abort_flag = 1;
                     atomicExch(status, 1);
                     break;
@@ -204,7 +219,7 @@ constexpr float kNegInf = -__builtin_huge_valf();
 
 // Optional phase timestamps of CTA 0 (development builds only; never compiled into the library).
 #ifdef ENL_TRACE
-__device__ long long g_trace[3][96][8];
+__device__ long long g_trace[5][96][8];
 #define ENL_TR(role, tile, slot) do { if (blockIdx.x == 0 && lane == 0 && (tile) < 96) g_trace[role][tile][slot] = clock64(); } while (0)
 #define ENL_PIN(x) asm volatile("" : "+f"(x) :: "memory")
 #else
@@ -234,7 +249,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
     auto bar_s_full   = [&](int i) { return bar0 + 8u * (1 + 2 * C::kStages + i); };
     auto bar_p_full   = [&](int i) { return bar0 + 8u * (3 + 2 * C::kStages + i); };
     auto bar_o_done   = [&](int i) { return bar0 + 8u * (5 + 2 * C::kStages + i); };
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + C::kBarOff + 8 * (7 + 2 * C::kStages));
+    auto bar_pair     = [&](int k) { return bar0 + 8u * (7 + 2 * C::kStages + k); };   // k = tile * 4 + lane quadrant
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + C::kBarOff + 8 * (15 + 2 * C::kStages));
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     // work item
@@ -258,9 +274,10 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
         for (int s = 0; s < C::kStages; ++s) { mbar_init(bar_kv_full(s), 1); mbar_init(bar_kv_empty(s), 1); }
         for (int i = 0; i < kQTiles; ++i) {
             mbar_init(bar_s_full(i), 1);
-            mbar_init(bar_p_full(i), 4);          // one arrival per softmax warp
+            mbar_init(bar_p_full(i), 8);          // one arrival per softmax warp of the tile
             mbar_init(bar_o_done(i), 1);
         }
+        for (int k = 0; k < 4 * kQTiles; ++k) mbar_init(bar_pair(k), 2);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -276,7 +293,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
 
     bool ok = true;
 
-    if (warp >= 8) {
+    if (warp >= kSoftmaxWarps) {
       asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
       if (warp == kProducerWarp) {
         // ================= TMA producer =================
@@ -384,11 +401,11 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                 if (ok && more) ok = wait_full(fk);
                 if (!ok) break;
                 for (int i = 0; i < n_qt; ++i) {
-                    ENL_TR(2, jj, 4 * i);
+                    ENL_TR(4, jj, 4 * i);
                     ok = mbar_wait(bar_p_full(i), static_cast<uint32_t>(jj & 1), abort_flag, p.status);
                     if (!ok) break;
                     tc_fence_after();
-                    ENL_TR(2, jj, 4 * i + 1);
+                    ENL_TR(4, jj, 4 * i + 1);
                     issue_pv(i, fv % C::kStages, jj == 0);
                     if (i == n_qt - 1) commit_to(bar_kv_empty(fv % C::kStages));
                     if (!more) commit_to(bar_o_done(i));
@@ -402,33 +419,63 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
       }
     } else {
       asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
-      if ((warp >> 2) < n_qt) {
-        // ================= softmax / epilogue, one thread per row =================
-        const int i = warp >> 2;
-        const int r = (warp & 3) * 32 + lane;
-        const int t = it.t0 + i * tile_tokens + r / rep;          // episode-relative query token
+      if ((warp >> 3) < n_qt) {
+        // ================= softmax / epilogue: two threads per row, 64 key columns each =================
+        constexpr int kHalfCols = kTileKeys / 2;                   // 64 key columns = 4 pages per thread
+        constexpr int kHalfPages = kPagesPerTile / 2;
+        const int i = warp >> 3;                                   // Q tile
+        const int hb = (warp >> 2) & 1;                            // 0: columns 0..63 (owner of the row's sums), 1: 64..127
+        const int q4 = warp & 3;                                   // TMEM lane quadrant
+        const bool owner = hb == 0;
+        const int r = q4 * 32 + lane;
+        const int t = it.t0 + i * tile_tokens + r / rep;           // episode-relative query token
         const int h = it.kvh * rep + r % rep;
         const bool row_valid = t < ep.n_q;
-        const int c = min(ep.n_new - ep.n_q + t, ep.n_new - 1);  // last visible new key
+        const int c = min(ep.n_new - ep.n_q + t, ep.n_new - 1);    // last visible new key
         const int G = ep.n_slots;
-        const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;
+        const uint32_t lane_sel = static_cast<uint32_t>(q4 * 32) << 16;
         const uint32_t t_s = tmem_base + lane_sel + static_cast<uint32_t>(i * 128);
         const uint32_t t_o = tmem_base + lane_sel + static_cast<uint32_t>(256 + i * 128);
         const bool split_mode = p.n_splits > 1;
         const long long grow = static_cast<long long>(ep.q_off) + t;   // global query row
         const long long rh = (split_mode ? (static_cast<long long>(it.split) * p.n_q_total + grow) : grow) * p.Hq + h;
         float *slot_out = nullptr;
-        if (row_valid) {
+        if (row_valid && owner) {
             if (split_mode) { if (p.part_slot) slot_out = p.part_slot + rh * p.mass_stride; }
             else if (p.mass) slot_out = p.mass + rh * p.mass_stride;
         }
         const float scale = p.scale_log2;
+        float *xmax_own = reinterpret_cast<float *>(smem + C::kXmaxOff) + (i * 2 + hb) * 128 + r;
+        const float *xmax_other = reinterpret_cast<const float *>(smem + C::kXmaxOff) + (i * 2 + (hb ^ 1)) * 128 + r;
+        float *xsum = reinterpret_cast<float *>(smem + C::kXsumOff) + i * (kHalfPages * 128) + r;   // + parity * kQTiles*4*128 + e*128
+        float *xinv = reinterpret_cast<float *>(smem + C::kXinvOff) + i * 128 + r;
+        const uint32_t pbar = bar_pair(i * 4 + q4);
+        uint32_t n_sync = 0;
+        // the two warps that share 32 rows meet here; bounded like every other wait
+        auto pair_sync = [&]() -> bool {
+            __syncwarp();
+            if (lane == 0) mbar_arrive(pbar);
+            const bool done = mbar_wait(pbar, n_sync & 1u, abort_flag, p.status);
+            ++n_sync;
+            return done;
+        };
 
-        float m = kNegInf, l = 0.f, acc = 0.f;
+        float m = kNegInf, l = 0.f, acc = 0.f;                     // l, acc: owner only
         int cur_slot = -1;
+        int pend_slot[kHalfPages];                                 // slots of half B's pages of the previous tile
+        bool pending = false;
+        // a page's sum goes to its slot; a slot that ends parks its log2-sum-exp
+        auto credit = [&](int slot, float v, float m_ref) {
+            if (slot != cur_slot) {
+                if (slot_out && cur_slot >= 0) slot_out[cur_slot] = lg2(acc) + m_ref;
+                acc = 0.f;
+                cur_slot = slot;
+            }
+            acc += v;
+            l += v;
+        };
 
-        // (slot << 8 | valid keys) of the eight pages of a tile; fetched one tile ahead so that the
-        // loads are in flight while this tile is processed
+        // (slot << 8 | valid keys) of the eight pages of a tile; fetched before the wait for the tile's S
         auto load_meta = [&](int j, int (&dst)[kPagesPerTile]) {
             if (j < ep.n_ctiles) {
                 const int4 *e4 = reinterpret_cast<const int4 *>(p.stream_meta + ep.stream_off + j * kPagesPerTile);
@@ -440,52 +487,30 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                 for (int e = 0; e < kPagesPerTile; ++e) dst[e] = (G << 8) | kPageTokens;
             }
         };
-        int meta_next[kPagesPerTile];
-        load_meta(j_beg, meta_next);
-
         for (int jj = 0; jj < n_tiles; ++jj) {
             const int j = j_beg + jj;
             const bool cached = j < ep.n_ctiles;
             int meta[kPagesPerTile];
-#pragma unroll
-            for (int e = 0; e < kPagesPerTile; ++e) meta[e] = meta_next[e];
-            if (jj + 1 < n_tiles) load_meta(j + 1, meta_next);
-            if ((warp & 3) == 0) ENL_TR(i, jj, 0);
+            load_meta(j, meta);
+            if (q4 == 0) ENL_TR(warp >> 2, jj, 0);
             ok = mbar_wait(bar_s_full(i), static_cast<uint32_t>(jj & 1), abort_flag, p.status);
             if (!ok) break;
             tc_fence_after();
-            if ((warp & 3) == 0) ENL_TR(i, jj, 1);
+            if (q4 == 0) ENL_TR(warp >> 2, jj, 1);
 
-            uint32_t su[128];
-#ifdef ENL_TRACE_LD
+            float s[kHalfCols];
             {
-                uint32_t c0[32], c1[32], c2[32], c3[32];
-                tmem_ld32_wait(t_s, c0);
-                if ((warp & 3) == 0) ENL_TR(i, jj, 2);
-                tmem_ld32_wait(t_s + 32, c1);
-                if ((warp & 3) == 0) ENL_TR(i, jj, 6);
-                tmem_ld32_wait(t_s + 64, c2);
-                if ((warp & 3) == 0) ENL_TR(i, jj, 7);
-                tmem_ld32_wait(t_s + 96, c3);
-                if ((warp & 3) == 0) ENL_TR(i, jj, 3);
+                uint32_t su[kHalfCols];
+                tmem_ld64_wait(t_s + static_cast<uint32_t>(hb * kHalfCols), su);
 #pragma unroll
-                for (int x = 0; x < 32; ++x) { su[x] = c0[x]; su[32 + x] = c1[x]; su[64 + x] = c2[x]; su[96 + x] = c3[x]; }
+                for (int x = 0; x < kHalfCols; ++x) s[x] = __uint_as_float(su[x]);
             }
-#define ENL_TR2(a, b, c) do { } while (0)
-#else
-            tmem_ld128_wait(t_s, su);
-            if ((warp & 3) == 0) ENL_TR(i, jj, 2);
-#define ENL_TR2(a, b, c) ENL_TR(a, b, c)
-#endif
-            float s[128];
-#pragma unroll
-            for (int x = 0; x < 128; ++x) s[x] = __uint_as_float(su[x]);
-
+            if (q4 == 0) ENL_TR(warp >> 2, jj, 5);
             // hide page padding (cached tiles) or keys after the causal limit (new-token tiles)
             if (cached) {
 #pragma unroll
-                for (int e = 0; e < kPagesPerTile; ++e) {
-                    const int nv = meta[e] & 0xff;
+                for (int e = 0; e < kHalfPages; ++e) {
+                    const int nv = (hb ? meta[kHalfPages + e] : meta[e]) & 0xff;      // static indices: meta stays in registers
                     if (nv < kPageTokens) {
 #pragma unroll
                         for (int x = 0; x < kPageTokens; ++x)
@@ -493,164 +518,177 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                     }
                 }
             } else {
-                const int lim = c - (j - ep.n_ctiles) * kTileKeys;
-                if (__any_sync(0xffffffffu, lim < kTileKeys - 1)) {
+                const int lim = c - (j - ep.n_ctiles) * kTileKeys - hb * kHalfCols;
+                if (__any_sync(0xffffffffu, lim < kHalfCols - 1)) {
 #pragma unroll
-                    for (int x = 0; x < 128; ++x)
+                    for (int x = 0; x < kHalfCols; ++x)
                         if (x > lim) s[x] = kNegInf;
                 }
             }
-
-#pragma unroll
-            for (int x = 0; x < 128; x += 8) ENL_PIN(s[x]);
-            if ((warp & 3) == 0) ENL_TR2(i, jj, 6);
-            // row maximum: eight independent chains of 3-input max, one per 16-key page
+            // maximum of this thread's 64 columns: four chains of 3-input max, one per page
             float mx;
             {
-                float pm[kPagesPerTile];
+                float pm[kHalfPages];
 #pragma unroll
-                for (int e = 0; e < kPagesPerTile; ++e) {
+                for (int e = 0; e < kHalfPages; ++e) {
                     const int b = e * kPageTokens;
                     float a = fmax3(s[b], s[b + 1], s[b + 2]);
 #pragma unroll
                     for (int x = 3; x < 15; x += 2) a = fmax3(a, s[b + x], s[b + x + 1]);
                     pm[e] = fmaxf(a, s[b + 15]);
                 }
-                mx = fmax3(fmax3(pm[0], pm[1], pm[2]), fmax3(pm[3], pm[4], pm[5]), fmaxf(pm[6], pm[7]));
+                mx = fmaxf(fmaxf(pm[0], pm[1]), fmaxf(pm[2], pm[3]));
             }
-            ENL_PIN(mx);
-            if ((warp & 3) == 0) ENL_TR2(i, jj, 7);
+            // exchange with the thread that holds the row's other 64 columns.  Behind this barrier both have
+            // S in registers, so half B may overwrite columns 32..63 of S with its P.
+            *xmax_own = mx;
+            if (q4 == 0) ENL_TR(warp >> 2, jj, 6);
+            ok = pair_sync();
+            if (!ok) break;
+            mx = fmaxf(mx, *xmax_other);
+            if (q4 == 0) ENL_TR(warp >> 2, jj, 2);
+            // half B's page sums of the previous tile (relative to the maximum that tile used)
+            if (owner && pending) {
+                const float *src = xsum + ((jj - 1) & 1) * (kQTiles * kHalfPages * 128);
+                const float m_ref = (m == kNegInf) ? 0.f : m;
+#pragma unroll
+                for (int e = 0; e < kHalfPages; ++e) credit(pend_slot[e], src[e * 128], m_ref);
+            }
+            if (q4 == 0) ENL_TR(warp >> 2, jj, 7);
             const float m_cand = mx * scale;
             const bool need = m_cand > m + kRescaleThreshold;       // also true when m == -inf < m_cand
-            if (__any_sync(0xffffffffu, need)) {
+            if (__any_sync(0xffffffffu, need)) {                     // same rows, same decision in both halves
                 const float m_new = fmaxf(m, m_cand);
                 const float alpha = (m_new == kNegInf) ? 1.f : ex2(m - m_new);
                 l *= alpha;
                 acc *= alpha;
                 m = m_new;
-                if (jj > 0) {                                        // O_i holds the tiles so far
-#pragma unroll
+                if (jj > 0) {                                        // O_i holds the tiles so far; each half rescales D/2 columns
+#pragma unroll 1
                     for (int k = 0; k < D / 32; ++k) {
-                        uint32_t o[32];
-                        tmem_ld32_wait(t_o + k * 32, o);
+                        uint32_t o[16];
+                        const uint32_t col = static_cast<uint32_t>(hb * (D / 2) + k * 16);
+                        tmem_ld16_wait(t_o + col, o);
 #pragma unroll
-                        for (int x = 0; x < 32; ++x) o[x] = __float_as_uint(__uint_as_float(o[x]) * alpha);
-                        tmem_st32(t_o + k * 32, o);
+                        for (int x = 0; x < 16; ++x) o[x] = __float_as_uint(__uint_as_float(o[x]) * alpha);
+                        tmem_st16(t_o + col, o);
                     }
                 }
             }
-            float m_use = (m == kNegInf) ? 0.f : m;
-            ENL_PIN(m_use);
-            if ((warp & 3) == 0) ENL_TR2(i, jj, 3);
+            const float m_use = (m == kNegInf) ? 0.f : m;
 
+            // p = exp2(s * scale - m) page by page: the page's sum, then its sixteen probabilities as eight bf16 pairs
+            // (even key in the low half) straight into P: this half's keys are columns hb*32 .. hb*32+31 of S_i
             const uint64_t sc2 = pack2(scale, scale), nm2 = pack2(-m_use, -m_use);
-            float bs[kPagesPerTile];                               // sum of p over each page
+            float bs[kHalfPages];
 #pragma unroll
-            for (int e = 0; e < kPagesPerTile; ++e) {
+            for (int e = 0; e < kHalfPages; ++e) {
                 uint64_t pr[kPageTokens / 2];
+                uint32_t pk[kPageTokens / 2];
 #pragma unroll
                 for (int x = 0; x < kPageTokens / 2; ++x) {
                     const int b = e * kPageTokens + 2 * x;
                     float a0, a1;
                     unpack2(fma2(pack2(s[b], s[b + 1]), sc2, nm2), a0, a1);
-                    s[b] = ex2(a0);
-                    s[b + 1] = ex2(a1);
-                    pr[x] = pack2(s[b], s[b + 1]);
+                    a0 = ex2(a0);
+                    a1 = ex2(a1);
+                    pr[x] = pack2(a0, a1);
+                    const __nv_bfloat162 bb = __floats2bfloat162_rn(a0, a1);
+                    pk[x] = *reinterpret_cast<const uint32_t *>(&bb);
                 }
+                tmem_st8(t_s + static_cast<uint32_t>(hb * 32 + e * 8), pk);
                 const uint64_t q0 = add2(add2(pr[0], pr[1]), add2(pr[2], pr[3]));
                 const uint64_t q1 = add2(add2(pr[4], pr[5]), add2(pr[6], pr[7]));
                 float b0, b1;
                 unpack2(add2(q0, q1), b0, b1);
                 bs[e] = b0 + b1;
             }
-            // credit the page sums to their slots; a slot that ends parks its log2-sum-exp
+            if (q4 == 0) ENL_TR(warp >> 2, jj, 3);
+            if (owner) {
 #pragma unroll
-            for (int e = 0; e < kPagesPerTile; ++e) {
-                const int slot = meta[e] >> 8;
-                if (slot != cur_slot) {
-                    if (slot_out && cur_slot >= 0) slot_out[cur_slot] = lg2(acc) + m_use;
-                    acc = 0.f;
-                    cur_slot = slot;
+                for (int e = 0; e < kHalfPages; ++e) {
+                    credit(meta[e] >> 8, bs[e], m_use);
+                    pend_slot[e] = meta[kHalfPages + e] >> 8;
                 }
-                acc += bs[e];
-                l += bs[e];
-            }
-
-            ENL_PIN(l);
-            ENL_PIN(acc);
-            if ((warp & 3) == 0) ENL_TR(i, jj, 4);
-            // P (bf16 pairs, even key in the low half) over the first 64 columns of S_i
+                pending = true;
+            } else {
+                float *dst = xsum + (jj & 1) * (kQTiles * kHalfPages * 128);
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                uint32_t pk[16];
-#pragma unroll
-                for (int x = 0; x < 16; ++x) {
-                    const __nv_bfloat162 b = __floats2bfloat162_rn(s[k * 32 + 2 * x], s[k * 32 + 2 * x + 1]);
-                    pk[x] = *reinterpret_cast<const uint32_t *>(&b);
-                }
-                tmem_st16(t_s + k * 16, pk);
+                for (int e = 0; e < kHalfPages; ++e) dst[e * 128] = bs[e];
             }
             tmem_st_wait();
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_p_full(i));
-            if ((warp & 3) == 0) ENL_TR(i, jj, 5);
+            if (q4 == 0) ENL_TR(warp >> 2, jj, 4);
         }
 
         // ---- per-row results ----
-        const float m_use = (m == kNegInf) ? 0.f : m;
+        float m_use = (m == kNegInf) ? 0.f : m;
+        if (ok) ok = pair_sync();                                   // half B's sums of the last tile are in place
         if (ok) {
-            if (slot_out && cur_slot >= 0) slot_out[cur_slot] = lg2(acc) + m_use;
-            const float lse = (l > 0.f) ? m_use + lg2(l) : kNegInf;
-            if (split_mode) {
-                if (row_valid) {
-                    // slots this split did not walk contribute nothing
-                    int first = G + 1, last = -1;
-                    if (n_tiles > 0) {
-                        first = (j_beg < ep.n_ctiles)
-                                    ? (p.stream_meta[ep.stream_off + j_beg * kPagesPerTile] >> 8) : G;
-                        last = (j_end > ep.n_ctiles)
-                                   ? G : (p.stream_meta[ep.stream_off + j_end * kPagesPerTile - 1] >> 8);
-                    }
-                    if (slot_out)
-                        for (int sl = 0; sl <= G; ++sl)
-                            if (sl < first || sl > last) slot_out[sl] = kNegInf;
-                    p.part_lse[rh] = lse;
-                }
-            } else if (slot_out) {
-                for (int sl = 0; sl <= G; ++sl) slot_out[sl] = ex2(slot_out[sl] - lse);
+            if (owner && pending) {
+                const float *src = xsum + ((n_tiles - 1) & 1) * (kQTiles * kHalfPages * 128);
+#pragma unroll
+                for (int e = 0; e < kHalfPages; ++e) credit(pend_slot[e], src[e * 128], m_use);
             }
-            if (n_tiles > 0) {
-                ok = mbar_wait(bar_o_done(i), 0, abort_flag, p.status);
-                if (ok) {
-                    tc_fence_after();
-                    const float inv = (l > 0.f) ? 1.f / l : 0.f;
+            const float inv = (l > 0.f) ? 1.f / l : 0.f;
+            if (owner) {
+                if (slot_out && cur_slot >= 0) slot_out[cur_slot] = lg2(acc) + m_use;
+                const float lse = (l > 0.f) ? m_use + lg2(l) : kNegInf;
+                if (split_mode) {
+                    if (row_valid) {
+                        // slots this split did not walk contribute nothing
+                        int first = G + 1, last = -1;
+                        if (n_tiles > 0) {
+                            first = (j_beg < ep.n_ctiles)
+                                        ? (p.stream_meta[ep.stream_off + j_beg * kPagesPerTile] >> 8) : G;
+                            last = (j_end > ep.n_ctiles)
+                                       ? G : (p.stream_meta[ep.stream_off + j_end * kPagesPerTile - 1] >> 8);
+                        }
+                        if (slot_out)
+                            for (int sl = 0; sl <= G; ++sl)
+                                if (sl < first || sl > last) slot_out[sl] = kNegInf;
+                        p.part_lse[rh] = lse;
+                    }
+                } else if (slot_out) {
+                    for (int sl = 0; sl <= G; ++sl) slot_out[sl] = ex2(slot_out[sl] - lse);
+                }
+                *xinv = inv;
+            }
+            ok = pair_sync();                                       // 1 / row sum reaches half B
+        }
+        if (ok && n_tiles > 0) {
+            const float inv = *xinv;
+            ok = mbar_wait(bar_o_done(i), 0, abort_flag, p.status);
+            if (ok) {
+                tc_fence_after();
 #pragma unroll
-                    for (int k = 0; k < D / 32; ++k) {
-                        uint32_t o[32];
-                        tmem_ld32_wait(t_o + k * 32, o);
-                        if (row_valid) {
-                            if (split_mode) {
-                                float4 *dst = reinterpret_cast<float4 *>(p.part_o + rh * D + k * 32);
+                for (int k = 0; k < D / 64; ++k) {                  // this half's D/2 output channels
+                    uint32_t o[32];
+                    const int col = hb * (D / 2) + k * 32;
+                    tmem_ld32_wait(t_o + static_cast<uint32_t>(col), o);
+                    if (row_valid) {
+                        if (split_mode) {
+                            float4 *dst = reinterpret_cast<float4 *>(p.part_o + rh * D + col);
 #pragma unroll
-                                for (int x = 0; x < 8; ++x)
-                                    dst[x] = make_float4(__uint_as_float(o[4 * x]) * inv, __uint_as_float(o[4 * x + 1]) * inv,
-                                                         __uint_as_float(o[4 * x + 2]) * inv, __uint_as_float(o[4 * x + 3]) * inv);
-                            } else {
-                                uint4 *dst = reinterpret_cast<uint4 *>(
-                                    static_cast<__nv_bfloat16 *>(p.out) + rh * D + k * 32);
+                            for (int x = 0; x < 8; ++x)
+                                dst[x] = make_float4(__uint_as_float(o[4 * x]) * inv, __uint_as_float(o[4 * x + 1]) * inv,
+                                                     __uint_as_float(o[4 * x + 2]) * inv, __uint_as_float(o[4 * x + 3]) * inv);
+                        } else {
+                            uint4 *dst = reinterpret_cast<uint4 *>(
+                                static_cast<__nv_bfloat16 *>(p.out) + rh * D + col);
 #pragma unroll
-                                for (int x = 0; x < 4; ++x) {
-                                    uint32_t w[4];
+                            for (int x = 0; x < 4; ++x) {
+                                uint32_t w[4];
 #pragma unroll
-                                    for (int y = 0; y < 4; ++y) {
-                                        const __nv_bfloat162 b = __floats2bfloat162_rn(
-                                            __uint_as_float(o[8 * x + 2 * y]) * inv,
-                                            __uint_as_float(o[8 * x + 2 * y + 1]) * inv);
-                                        w[y] = *reinterpret_cast<const uint32_t *>(&b);
-                                    }
-                                    dst[x] = make_uint4(w[0], w[1], w[2], w[3]);
+                                for (int y = 0; y < 4; ++y) {
+                                    const __nv_bfloat162 b = __floats2bfloat162_rn(
+                                        __uint_as_float(o[8 * x + 2 * y]) * inv,
+                                        __uint_as_float(o[8 * x + 2 * y + 1]) * inv);
+                                    w[y] = *reinterpret_cast<const uint32_t *>(&b);
                                 }
+                                dst[x] = make_uint4(w[0], w[1], w[2], w[3]);
                             }
                         }
                     }

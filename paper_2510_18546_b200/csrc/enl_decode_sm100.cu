@@ -69,12 +69,17 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 {
     bool ok = mbar_try_wait(bar, parity);
     if (!ok) {
-        const unsigned long long t0 = global_ns();
+        // the clock is read only every 256 failed polls (the first reading starts the limit): a poll already
+        // sleeps inside the instruction, and reading the global timer is far slower than a poll
+        unsigned long long t0 = 0;
         uint32_t spins = 0;
         while (!(ok = mbar_try_wait(bar, parity))) {
-            if ((++spins & 63u) == 0u) {
+            if ((++spins & 255u) == 0u) {
                 if (*abort_flag) break;
-                if (global_ns() - t0 > kWaitLimitNs) {
+                const unsigned long long now = global_ns();
+                if (t0 == 0) {
+                    t0 = now;
+                } else if (now - t0 > kWaitLimitNs) {
                     *abort_flag = 1;
                     atomicExch(status, 2);
                     break;
