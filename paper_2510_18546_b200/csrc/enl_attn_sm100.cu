@@ -21,7 +21,8 @@
 // softmax warps per scheduler overlap each other's exp2, max, pack and TMEM traffic.  Warp 16 is the TMA
 // producer, warp 17 the MMA issuer (and TMEM owner), warps 18-19 idle: they complete the fifth warpgroup
 // so that setmaxnreg can move registers to the softmax warpgroups.
-// TMEM columns: S0 [0,128) S1 [128,256) O0 [256,384) O1 [384,512); P_i overwrites the first 64 columns of S_i.
+// TMEM columns: S0 [0,128) S1 [128,256) O0 [256,384) O1 [384,512); P_i (bf16) overwrites columns [0,32) and
+// [64,96) of S_i, each softmax half inside its own columns.
 #include <cuda_bf16.h>
 
 #include "enl_internal.h"
@@ -47,11 +48,11 @@ struct Cfg {
     static constexpr int kTileBytes = kHalves * kHalfBytes;
     static constexpr int kStages    = (D == 128) ? 4 : 8;
     static constexpr int kBarOff    = (kQTiles + kStages) * kTileBytes;
-    // exchange area of the softmax thread pairs: row maxima [tile][half][128], half B's page sums
-    // [parity][tile][4][128], 1 / row sum [tile][128]
+    // exchange area of the softmax thread pairs: row maxima [tile][half][128], page sums
+    // [parity][tile][8 pages][128], 1 / row sum [tile][128]
     static constexpr int kXmaxOff   = kBarOff + 512;
     static constexpr int kXsumOff   = kXmaxOff + kQTiles * 2 * 128 * 4;
-    static constexpr int kXinvOff   = kXsumOff + 2 * kQTiles * 4 * 128 * 4;
+    static constexpr int kXinvOff   = kXsumOff + 2 * kQTiles * kPagesPerTile * 128 * 4;
     static constexpr int kSmemBytes = kXinvOff + kQTiles * 128 * 4 + 1024;   // + alignment slack
 };
 
@@ -371,7 +372,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                 if (lane == 0) {
 #pragma unroll
                     for (int kk = 0; kk < kTileKeys / 16; ++kk) {
-                        mma_ts(tmem_o(i), tmem_s(i) + static_cast<uint32_t>(kk * 8),
+                        mma_ts(tmem_o(i), tmem_s(i) + static_cast<uint32_t>((kk >> 2) * 64 + (kk & 3) * 8),   // P of keys 64.. sits in columns 64..
                                smem_desc(stage_addr(st) + static_cast<uint32_t>(kk * 16 * 128), C::kHalfBytes),
                                idesc_pv, (first_tile && kk == 0) ? 0u : 1u);
                     }
@@ -413,6 +414,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                         issue_qk(i, fk % C::kStages);
                         if (i == n_qt - 1) commit_to(bar_kv_empty(fk % C::kStages));
                     }
+                    ENL_TR(4, jj, 4 * i + 2);
                 }
             }
         }
@@ -447,7 +449,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
         const float scale = p.scale_log2;
         float *xmax_own = reinterpret_cast<float *>(smem + C::kXmaxOff) + (i * 2 + hb) * 128 + r;
         const float *xmax_other = reinterpret_cast<const float *>(smem + C::kXmaxOff) + (i * 2 + (hb ^ 1)) * 128 + r;
-        float *xsum = reinterpret_cast<float *>(smem + C::kXsumOff) + i * (kHalfPages * 128) + r;   // + parity * kQTiles*4*128 + e*128
+        float *xsum = reinterpret_cast<float *>(smem + C::kXsumOff) + i * (kPagesPerTile * 128) + r;   // + parity * kQTiles*8*128 + page*128
         float *xinv = reinterpret_cast<float *>(smem + C::kXinvOff) + i * 128 + r;
         const uint32_t pbar = bar_pair(i * 4 + q4);
         uint32_t n_sync = 0;
@@ -462,8 +464,6 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
 
         float m = kNegInf, l = 0.f, acc = 0.f;                     // l, acc: owner only
         int cur_slot = -1;
-        int pend_slot[kHalfPages];                                 // slots of half B's pages of the previous tile
-        bool pending = false;
         // a page's sum goes to its slot; a slot that ends parks its log2-sum-exp
         auto credit = [&](int slot, float v, float m_ref) {
             if (slot != cur_slot) {
@@ -474,30 +474,55 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
             acc += v;
             l += v;
         };
-
-        // (slot << 8 | valid keys) of the eight pages of a tile; fetched before the wait for the tile's S
-        auto load_meta = [&](int j, int (&dst)[kPagesPerTile]) {
-            if (j < ep.n_ctiles) {
-                const int4 *e4 = reinterpret_cast<const int4 *>(p.stream_meta + ep.stream_off + j * kPagesPerTile);
+        // The owner credits the eight page sums of tile j (its own four and half B's four, both parked in shared
+        // memory) only after it has handed P of tile j + 1 to the MMA warp: the slot book-keeping and its
+        // scattered stores then overlap the MMAs instead of delaying them.  `late` = the factor by which the
+        // running sums were rescaled since those page sums were taken.
+        auto credit_tile = [&](int jt, float late, float m_ref) {
+            const float *src = xsum + (jt & 1) * (kQTiles * kPagesPerTile * 128);
+            const int jg = j_beg + jt;
+            if (jg < ep.n_ctiles) {
+                const int4 *e4 = reinterpret_cast<const int4 *>(p.stream_meta + ep.stream_off + jg * kPagesPerTile);
                 const int4 a = __ldg(e4), b = __ldg(e4 + 1);
-                dst[0] = a.x; dst[1] = a.y; dst[2] = a.z; dst[3] = a.w;
-                dst[4] = b.x; dst[5] = b.y; dst[6] = b.z; dst[7] = b.w;
+                credit(a.x >> 8, src[0 * 128] * late, m_ref);
+                credit(a.y >> 8, src[1 * 128] * late, m_ref);
+                credit(a.z >> 8, src[2 * 128] * late, m_ref);
+                credit(a.w >> 8, src[3 * 128] * late, m_ref);
+                credit(b.x >> 8, src[4 * 128] * late, m_ref);
+                credit(b.y >> 8, src[5 * 128] * late, m_ref);
+                credit(b.z >> 8, src[6 * 128] * late, m_ref);
+                credit(b.w >> 8, src[7 * 128] * late, m_ref);
             } else {
+                float v = 0.f;
 #pragma unroll
-                for (int e = 0; e < kPagesPerTile; ++e) dst[e] = (G << 8) | kPageTokens;
+                for (int e = 0; e < kPagesPerTile; ++e) v += src[e * 128];
+                credit(G, v * late, m_ref);
             }
         };
+
         for (int jj = 0; jj < n_tiles; ++jj) {
             const int j = j_beg + jj;
-            const bool cached = j < ep.n_ctiles;
-            int meta[kPagesPerTile];
-            load_meta(j, meta);
+            // valid keys of this thread's four pages, one byte each: page padding (cached tiles) or the causal
+            // limit (new-token tiles)
+            uint32_t nvp;
+            if (j < ep.n_ctiles) {
+                const int4 mv = __ldg(reinterpret_cast<const int4 *>(p.stream_meta + ep.stream_off + j * kPagesPerTile) + hb);
+                nvp = static_cast<uint32_t>(mv.x & 0xff) | (static_cast<uint32_t>(mv.y & 0xff) << 8) |
+                      (static_cast<uint32_t>(mv.z & 0xff) << 16) | (static_cast<uint32_t>(mv.w & 0xff) << 24);
+            } else {
+                const int vis = c - (j - ep.n_ctiles) * kTileKeys - hb * kHalfCols + 1;   // visible keys of this half
+                nvp = 0;
+#pragma unroll
+                for (int e = 0; e < kHalfPages; ++e)
+                    nvp |= static_cast<uint32_t>(min(max(vis - e * kPageTokens, 0), kPageTokens)) << (8 * e);
+            }
             if (q4 == 0) ENL_TR(warp >> 2, jj, 0);
             ok = mbar_wait(bar_s_full(i), static_cast<uint32_t>(jj & 1), abort_flag, p.status);
             if (!ok) break;
             tc_fence_after();
             if (q4 == 0) ENL_TR(warp >> 2, jj, 1);
 
+            // all 64 scores of this thread in one TMEM round trip (a round trip costs about 200 cycles)
             float s[kHalfCols];
             {
                 uint32_t su[kHalfCols];
@@ -505,33 +530,19 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
 #pragma unroll
                 for (int x = 0; x < kHalfCols; ++x) s[x] = __uint_as_float(su[x]);
             }
-            if (q4 == 0) ENL_TR(warp >> 2, jj, 5);
-            // hide page padding (cached tiles) or keys after the causal limit (new-token tiles)
-            if (cached) {
-#pragma unroll
-                for (int e = 0; e < kHalfPages; ++e) {
-                    const int nv = (hb ? meta[kHalfPages + e] : meta[e]) & 0xff;      // static indices: meta stays in registers
-                    if (nv < kPageTokens) {
-#pragma unroll
-                        for (int x = 0; x < kPageTokens; ++x)
-                            if (x >= nv) s[e * kPageTokens + x] = kNegInf;
-                    }
-                }
-            } else {
-                const int lim = c - (j - ep.n_ctiles) * kTileKeys - hb * kHalfCols;
-                if (__any_sync(0xffffffffu, lim < kHalfCols - 1)) {
-#pragma unroll
-                    for (int x = 0; x < kHalfCols; ++x)
-                        if (x > lim) s[x] = kNegInf;
-                }
-            }
-            // maximum of this thread's 64 columns: four chains of 3-input max, one per page
+            // hide page padding / keys after the causal limit, and take the maximum page by page
             float mx;
             {
                 float pm[kHalfPages];
 #pragma unroll
                 for (int e = 0; e < kHalfPages; ++e) {
+                    const int nv = static_cast<int>((nvp >> (8 * e)) & 0xffu);
                     const int b = e * kPageTokens;
+                    if (nv < kPageTokens) {
+#pragma unroll
+                        for (int x = 0; x < kPageTokens; ++x)
+                            if (x >= nv) s[b + x] = kNegInf;
+                    }
                     float a = fmax3(s[b], s[b + 1], s[b + 2]);
 #pragma unroll
                     for (int x = 3; x < 15; x += 2) a = fmax3(a, s[b + x], s[b + x + 1]);
@@ -539,22 +550,14 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                 }
                 mx = fmaxf(fmaxf(pm[0], pm[1]), fmaxf(pm[2], pm[3]));
             }
-            // exchange with the thread that holds the row's other 64 columns.  Behind this barrier both have
-            // S in registers, so half B may overwrite columns 32..63 of S with its P.
+            // exchange with the thread that holds the row's other 64 columns
             *xmax_own = mx;
-            if (q4 == 0) ENL_TR(warp >> 2, jj, 6);
             ok = pair_sync();
             if (!ok) break;
             mx = fmaxf(mx, *xmax_other);
             if (q4 == 0) ENL_TR(warp >> 2, jj, 2);
-            // half B's page sums of the previous tile (relative to the maximum that tile used)
-            if (owner && pending) {
-                const float *src = xsum + ((jj - 1) & 1) * (kQTiles * kHalfPages * 128);
-                const float m_ref = (m == kNegInf) ? 0.f : m;
-#pragma unroll
-                for (int e = 0; e < kHalfPages; ++e) credit(pend_slot[e], src[e * 128], m_ref);
-            }
-            if (q4 == 0) ENL_TR(warp >> 2, jj, 7);
+
+            float late = 1.f;
             const float m_cand = mx * scale;
             const bool need = m_cand > m + kRescaleThreshold;       // also true when m == -inf < m_cand
             if (__any_sync(0xffffffffu, need)) {                     // same rows, same decision in both halves
@@ -562,6 +565,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                 const float alpha = (m_new == kNegInf) ? 1.f : ex2(m - m_new);
                 l *= alpha;
                 acc *= alpha;
+                late = alpha;
                 m = m_new;
                 if (jj > 0) {                                        // O_i holds the tiles so far; each half rescales D/2 columns
 #pragma unroll 1
@@ -577,10 +581,11 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
             }
             const float m_use = (m == kNegInf) ? 0.f : m;
 
-            // p = exp2(s * scale - m) page by page: the page's sum, then its sixteen probabilities as eight bf16 pairs
-            // (even key in the low half) straight into P: this half's keys are columns hb*32 .. hb*32+31 of S_i
+            // p = exp2(s * scale - m) page by page; the page's sum goes to shared memory (the owner credits it to
+            // its slot later), its sixteen probabilities go as eight bf16 pairs (even key in the low half) into P.
+            // Each half keeps its P inside its own 64 columns of S_i (page e at columns hb*64 + 8e .. +7).
             const uint64_t sc2 = pack2(scale, scale), nm2 = pack2(-m_use, -m_use);
-            float bs[kHalfPages];
+            float *sum_dst = xsum + (jj & 1) * (kQTiles * kPagesPerTile * 128) + hb * (kHalfPages * 128);
 #pragma unroll
             for (int e = 0; e < kHalfPages; ++e) {
                 uint64_t pr[kPageTokens / 2];
@@ -596,42 +601,27 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                     const __nv_bfloat162 bb = __floats2bfloat162_rn(a0, a1);
                     pk[x] = *reinterpret_cast<const uint32_t *>(&bb);
                 }
-                tmem_st8(t_s + static_cast<uint32_t>(hb * 32 + e * 8), pk);
+                tmem_st8(t_s + static_cast<uint32_t>(hb * kHalfCols + e * 8), pk);
                 const uint64_t q0 = add2(add2(pr[0], pr[1]), add2(pr[2], pr[3]));
                 const uint64_t q1 = add2(add2(pr[4], pr[5]), add2(pr[6], pr[7]));
                 float b0, b1;
                 unpack2(add2(q0, q1), b0, b1);
-                bs[e] = b0 + b1;
+                sum_dst[e * 128] = b0 + b1;
             }
             if (q4 == 0) ENL_TR(warp >> 2, jj, 3);
-            if (owner) {
-#pragma unroll
-                for (int e = 0; e < kHalfPages; ++e) {
-                    credit(meta[e] >> 8, bs[e], m_use);
-                    pend_slot[e] = meta[kHalfPages + e] >> 8;
-                }
-                pending = true;
-            } else {
-                float *dst = xsum + (jj & 1) * (kQTiles * kHalfPages * 128);
-#pragma unroll
-                for (int e = 0; e < kHalfPages; ++e) dst[e * 128] = bs[e];
-            }
             tmem_st_wait();
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_p_full(i));
             if (q4 == 0) ENL_TR(warp >> 2, jj, 4);
+            if (owner && jj > 0) credit_tile(jj - 1, late, m_use);
         }
 
         // ---- per-row results ----
         float m_use = (m == kNegInf) ? 0.f : m;
         if (ok) ok = pair_sync();                                   // half B's sums of the last tile are in place
         if (ok) {
-            if (owner && pending) {
-                const float *src = xsum + ((n_tiles - 1) & 1) * (kQTiles * kHalfPages * 128);
-#pragma unroll
-                for (int e = 0; e < kHalfPages; ++e) credit(pend_slot[e], src[e * 128], m_use);
-            }
+            if (owner && n_tiles > 0) credit_tile(n_tiles - 1, 1.f, m_use);
             const float inv = (l > 0.f) ? 1.f / l : 0.f;
             if (owner) {
                 if (slot_out && cur_slot >= 0) slot_out[cur_slot] = lg2(acc) + m_use;
