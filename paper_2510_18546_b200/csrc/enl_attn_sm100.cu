@@ -39,6 +39,7 @@ constexpr int kProducerWarp = 16;
 constexpr int kMmaWarp      = 17;
 constexpr uint32_t kTmemCols = 512;
 constexpr float kRescaleThreshold = 8.0f;     // log2 units: p stays below 2^8 between max updates
+constexpr float kMaxJump = 100.0f;            // log2 units: most a tile's scores may exceed the maximum of all earlier tiles
 constexpr unsigned long long kWaitLimitNs = 1000ull * 1000ull * 1000ull;
 
 template <int D>
@@ -48,11 +49,11 @@ struct Cfg {
     static constexpr int kTileBytes = kHalves * kHalfBytes;
     static constexpr int kStages    = (D == 128) ? 4 : 8;
     static constexpr int kBarOff    = (kQTiles + kStages) * kTileBytes;
-    // exchange area of the softmax thread pairs: row maxima [tile][half][128], page sums
-    // [parity][tile][8 pages][128], 1 / row sum [tile][128]
+    // exchange area of the softmax thread pairs: row maxima [parity][tile][half][128], page sums
+    // [tile mod 3][tile][8 pages][128], 1 / row sum [tile][128]
     static constexpr int kXmaxOff   = kBarOff + 512;
-    static constexpr int kXsumOff   = kXmaxOff + kQTiles * 2 * 128 * 4;
-    static constexpr int kXinvOff   = kXsumOff + 2 * kQTiles * kPagesPerTile * 128 * 4;
+    static constexpr int kXsumOff   = kXmaxOff + 2 * kQTiles * 2 * 128 * 4;
+    static constexpr int kXinvOff   = kXsumOff + 3 * kQTiles * kPagesPerTile * 128 * 4;
     static constexpr int kSmemBytes = kXinvOff + kQTiles * 128 * 4 + 1024;   // + alignment slack
 };
 
@@ -447,9 +448,10 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
             else if (p.mass) slot_out = p.mass + rh * p.mass_stride;
         }
         const float scale = p.scale_log2;
-        float *xmax_own = reinterpret_cast<float *>(smem + C::kXmaxOff) + (i * 2 + hb) * 128 + r;
+        float *xmax_own = reinterpret_cast<float *>(smem + C::kXmaxOff) + (i * 2 + hb) * 128 + r;          // + parity * kQTiles*2*128
         const float *xmax_other = reinterpret_cast<const float *>(smem + C::kXmaxOff) + (i * 2 + (hb ^ 1)) * 128 + r;
-        float *xsum = reinterpret_cast<float *>(smem + C::kXsumOff) + i * (kPagesPerTile * 128) + r;   // + parity * kQTiles*8*128 + page*128
+        constexpr int kXmaxPar = kQTiles * 2 * 128;
+        float *xsum = reinterpret_cast<float *>(smem + C::kXsumOff) + i * (kPagesPerTile * 128) + r;   // + (tile mod 3) * kQTiles*8*128 + page*128
         float *xinv = reinterpret_cast<float *>(smem + C::kXinvOff) + i * 128 + r;
         const uint32_t pbar = bar_pair(i * 4 + q4);
         uint32_t n_sync = 0;
@@ -463,6 +465,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
         };
 
         float m = kNegInf, l = 0.f, acc = 0.f;                     // l, acc: owner only
+        float mx_prev = kNegInf;                                   // this thread's maximum of the previous tile (unscaled)
         int cur_slot = -1;
         // a page's sum goes to its slot; a slot that ends parks its log2-sum-exp
         auto credit = [&](int slot, float v, float m_ref) {
@@ -479,7 +482,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
         // scattered stores then overlap the MMAs instead of delaying them.  `late` = the factor by which the
         // running sums were rescaled since those page sums were taken.
         auto credit_tile = [&](int jt, float late, float m_ref) {
-            const float *src = xsum + (jt & 1) * (kQTiles * kPagesPerTile * 128);
+            const float *src = xsum + (jt % 3) * (kQTiles * kPagesPerTile * 128);
             const int jg = j_beg + jt;
             if (jg < ep.n_ctiles) {
                 const int4 *e4 = reinterpret_cast<const int4 *>(p.stream_meta + ep.stream_off + jg * kPagesPerTile);
@@ -550,15 +553,28 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                 }
                 mx = fmaxf(fmaxf(pm[0], pm[1]), fmaxf(pm[2], pm[3]));
             }
-            // exchange with the thread that holds the row's other 64 columns
-            *xmax_own = mx;
-            ok = pair_sync();
-            if (!ok) break;
-            mx = fmaxf(mx, *xmax_other);
+            // The reference maximum needs the other half's columns too.  Waiting for them every tile would put a
+            // two-warp barrier on the critical path, so the exchange lags by one tile: this tile's exponentials
+            // use the maximum over all EARLIER tiles (both halves know it: the partner's maximum of the previous
+            // tile has been in shared memory since before that tile's P was handed over), and this tile's
+            // maximum only moves the reference for the next one.  A probability may then exceed 1 by the factor
+            // 2^(jump of this tile over everything before it), harmless in floating point up to kMaxJump.  The
+            // first tile, and any tile that starts without a reference, exchange synchronously.
+            const bool sync_tile = (jj == 0) || __any_sync(0xffffffffu, m == kNegInf);   // same rows, same m in both halves
+            xmax_own[(jj & 1) * kXmaxPar] = mx;
+            float mx_ref;
+            if (sync_tile) {
+                ok = pair_sync();
+                if (!ok) break;
+                mx_ref = fmaxf(mx, xmax_other[(jj & 1) * kXmaxPar]);
+            } else {
+                mx_ref = fmaxf(mx_prev, xmax_other[((jj - 1) & 1) * kXmaxPar]);
+            }
+            mx_prev = mx;
             if (q4 == 0) ENL_TR(warp >> 2, jj, 2);
 
             float late = 1.f;
-            const float m_cand = mx * scale;
+            const float m_cand = mx_ref * scale;
             const bool need = m_cand > m + kRescaleThreshold;       // also true when m == -inf < m_cand
             if (__any_sync(0xffffffffu, need)) {                     // same rows, same decision in both halves
                 const float m_new = fmaxf(m, m_cand);
@@ -580,12 +596,19 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                 }
             }
             const float m_use = (m == kNegInf) ? 0.f : m;
+            if (!sync_tile && __any_sync(0xffffffffu, mx * scale > m_use + kMaxJump)) {
+                // beyond what the lagging reference can carry: keep the result finite and report it
+                if (mx * scale > m_use + kMaxJump) atomicExch(p.status, 3);
+                const float cap = (m_use + kMaxJump) / scale;
+#pragma unroll
+                for (int x = 0; x < kHalfCols; ++x) s[x] = fminf(s[x], cap);
+            }
 
             // p = exp2(s * scale - m) page by page; the page's sum goes to shared memory (the owner credits it to
             // its slot later), its sixteen probabilities go as eight bf16 pairs (even key in the low half) into P.
             // Each half keeps its P inside its own 64 columns of S_i (page e at columns hb*64 + 8e .. +7).
             const uint64_t sc2 = pack2(scale, scale), nm2 = pack2(-m_use, -m_use);
-            float *sum_dst = xsum + (jj & 1) * (kQTiles * kPagesPerTile * 128) + hb * (kHalfPages * 128);
+            float *sum_dst = xsum + (jj % 3) * (kQTiles * kPagesPerTile * 128) + hb * (kHalfPages * 128);
 #pragma unroll
             for (int e = 0; e < kHalfPages; ++e) {
                 uint64_t pr[kPageTokens / 2];
