@@ -48,14 +48,17 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
+// One poll: the thread may stay suspended inside the instruction for up to the hinted time, and is woken when
+// the phase completes; a longer hint means fewer polling instructions competing with the warps that work.
+constexpr uint32_t kSuspendHintNs = 20000;
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        : "=r"(ok) : "r"(bar), "r"(parity), "r"(kSuspendHintNs) : "memory");
     return ok != 0;
 }
 __device__ __forceinline__ unsigned long long global_ns()
@@ -69,12 +72,12 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 {
     bool ok = mbar_try_wait(bar, parity);
     if (!ok) {
-        // the clock is read only every 256 failed polls (the first reading starts the limit): a poll already
-        // sleeps inside the instruction, and reading the global timer is far slower than a poll
+        // the clock is read only every 16 failed polls (the first reading starts the limit): a poll already
+        // sleeps inside the instruction
         unsigned long long t0 = 0;
         uint32_t spins = 0;
         while (!(ok = mbar_try_wait(bar, parity))) {
-            if ((++spins & 255u) == 0u) {
+            if ((++spins & 15u) == 0u) {
                 if (*abort_flag) break;
                 const unsigned long long now = global_ns();
                 if (t0 == 0) {
