@@ -295,6 +295,10 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // everything above touched only shared memory, TMEM and the gather plan; from here on the caller's tensors,
+    // the pool and the scratch are read and written, so the previous kernel of the stream must have finished
+    pdl_trigger();
+    pdl_wait();
 
     bool ok = true;
 
@@ -749,13 +753,14 @@ cudaError_t prepare_attention(int head_dim)
 cudaError_t launch_attention(const AttnParams &p, int head_dim, int n_items, cudaStream_t st)
 {
     if (n_items <= 0) return cudaSuccess;
+    cudaError_t e;
     if (head_dim == 128)
-        attn_kernel<128><<<n_items, kThreads, Cfg<128>::kSmemBytes, st>>>(p);
+        e = launch_pdl(attn_kernel<128>, dim3(n_items), dim3(kThreads), Cfg<128>::kSmemBytes, st, p);
     else if (head_dim == 64)
-        attn_kernel<64><<<n_items, kThreads, Cfg<64>::kSmemBytes, st>>>(p);
+        e = launch_pdl(attn_kernel<64>, dim3(n_items), dim3(kThreads), Cfg<64>::kSmemBytes, st, p);
     else
         return cudaErrorInvalidValue;
-    return cudaGetLastError();
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace enl

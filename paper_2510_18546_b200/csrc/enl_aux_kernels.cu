@@ -46,6 +46,8 @@ __global__ void combine_kernel(const CombineParams p)
     const int lane = threadIdx.x & 31;
     const long long rh = blockIdx.x * static_cast<long long>(blockDim.x >> 5) + (threadIdx.x >> 5);
     const long long split_stride = static_cast<long long>(p.n_q_total) * p.Hq;
+    pdl_trigger();
+    pdl_wait();                                             // the partial results come from the previous kernel
     if (rh >= split_stride) return;
     const int row = static_cast<int>(rh / p.Hq);
     const float ninf = -__builtin_huge_valf();
@@ -121,9 +123,9 @@ cudaError_t launch_combine(const CombineParams &p, cudaStream_t st)
     if (pairs <= 0) return cudaSuccess;
     const int warps = 8;
     const int blocks = static_cast<int>((pairs + warps - 1) / warps);
-    if (p.D == 128) combine_kernel<128><<<blocks, warps * 32, 0, st>>>(p);
-    else combine_kernel<64><<<blocks, warps * 32, 0, st>>>(p);
-    return cudaGetLastError();
+    const cudaError_t e = (p.D == 128) ? launch_pdl(combine_kernel<128>, dim3(blocks), dim3(warps * 32), 0, st, p)
+                                       : launch_pdl(combine_kernel<64>, dim3(blocks), dim3(warps * 32), 0, st, p);
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace enl

@@ -244,6 +244,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     __syncthreads();
+    pdl_trigger();
 
     // lane j keeps the page id and the meta word of entry j of this warp's run (n_w <= 32): one coalesced
     // load up front, so that no global load sits between a stage becoming free and its refill
@@ -258,6 +259,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
             my_meta = entry_meta(e);
         }
     }
+    // so far only shared memory and the gather plan were touched; the caller's tensors and the pool come next
+    pdl_wait();
     const uint64_t pol = policy_evict_first();
     // load i of this warp: K page i/2 (i even) or V page i/2 (i odd); `page` as kept by lane i/2
     auto issue = [&](int i, int page) {
@@ -663,13 +666,14 @@ cudaError_t launch_decode(const DecodeParams &p, int head_dim, int batch, cudaSt
 {
     if (batch <= 0 || p.n_splits <= 0) return cudaSuccess;
     const dim3 grid(p.n_splits, p.Hkv, batch);
+    cudaError_t e;
     if (head_dim == 128)
-        decode_kernel<128><<<grid, kThreads, DecCfg<128>::kSmemBytes, st>>>(p);
+        e = launch_pdl(decode_kernel<128>, grid, dim3(kThreads), DecCfg<128>::kSmemBytes, st, p);
     else if (head_dim == 64)
-        decode_kernel<64><<<grid, kThreads, DecCfg<64>::kSmemBytes, st>>>(p);
+        e = launch_pdl(decode_kernel<64>, grid, dim3(kThreads), DecCfg<64>::kSmemBytes, st, p);
     else
         return cudaErrorInvalidValue;
-    return cudaGetLastError();
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace enl

@@ -96,6 +96,29 @@ struct CombineParams {
     int32_t n_splits;
 };
 
+// Programmatic dependent launch: a kernel launched this way may start (set-up only) while the previous kernel
+// of the stream is still draining; it must execute pdl_wait() before it touches anything a predecessor may have
+// written, and pdl_trigger() as early as it likes so that its own successor can be set up the same way.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+template <typename Kernel, typename Params>
+inline cudaError_t launch_pdl(Kernel kernel, dim3 grid, dim3 block, size_t smem, cudaStream_t st, const Params &prm)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, prm);
+}
+#endif
+
 // launchers (defined in the .cu files of the kernels)
 cudaError_t launch_attention(const AttnParams &p, int head_dim, int n_items, cudaStream_t st);
 cudaError_t launch_combine(const CombineParams &p, cudaStream_t st);
