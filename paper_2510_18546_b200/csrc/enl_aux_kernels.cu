@@ -52,6 +52,64 @@ __global__ void combine_kernel(const CombineParams p)
     const int row = static_cast<int>(rh / p.Hq);
     const float ninf = -__builtin_huge_valf();
 
+    // Few splits (the usual case): every load of the warp -- log-sum-exps, partial outputs, the first 32 slot
+    // log-sums -- is issued before anything is computed, so the warp pays one memory round trip, not five.
+    if (p.n_splits <= 4) {
+        const float *slot0 = p.part_slot ? p.part_slot + rh * p.slot_stride + lane : nullptr;
+        const int G = p.mass ? p.row_slots[row] : -1;
+        float lv[4], sv[4], ov[4][V];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const bool on = k < p.n_splits;
+            lv[k] = on ? __ldcg(p.part_lse + k * split_stride + rh) : ninf;
+            sv[k] = (on && p.mass && lane <= G) ? __ldcg(slot0 + k * split_stride * p.slot_stride) : ninf;
+            const float *src = p.part_o + ((on ? k : 0) * split_stride + rh) * D + lane * V;
+            if constexpr (V == 4) {
+                const float4 t = __ldcg(reinterpret_cast<const float4 *>(src));
+                ov[k][0] = t.x; ov[k][1] = t.y; ov[k][2] = t.z; ov[k][3] = t.w;
+            } else {
+                const float2 t = __ldcg(reinterpret_cast<const float2 *>(src));
+                ov[k][0] = t.x; ov[k][1] = t.y;
+            }
+        }
+        const float mxv = fmaxf(fmaxf(lv[0], lv[1]), fmaxf(lv[2], lv[3]));
+        float sum = 0.f;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) sum += (lv[k] != ninf) ? ex2f(lv[k] - mxv) : 0.f;
+        const float lse = mxv + log2f(sum);
+        const float lse_s = (lse > ninf) ? lse : 0.f;
+        float acc[V];
+#pragma unroll
+        for (int x = 0; x < V; ++x) acc[x] = 0.f;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const float w = (lv[k] != ninf) ? ex2f(lv[k] - lse) : 0.f;
+#pragma unroll
+            for (int x = 0; x < V; ++x) acc[x] += w * ov[k][x];
+        }
+        __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(p.out) + rh * D + lane * V;
+#pragma unroll
+        for (int x = 0; x < V; x += 2)
+            *reinterpret_cast<__nv_bfloat162 *>(dst + x) = __floats2bfloat162_rn(acc[x], acc[x + 1]);
+        if (p.mass) {
+            if (lane <= G) {
+                float w = 0.f;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) w += ex2f(sv[k] - lse_s);       // exp2(-inf) = 0: absent slots drop out
+                p.mass[rh * p.mass_stride + lane] = w;
+            }
+            for (int s = lane + 32; s <= G; s += 32) {                      // more than 32 slots: the rest, as below
+                float w = 0.f;
+                for (int k = 0; k < p.n_splits; ++k) {
+                    const float v = __ldcg(p.part_slot + (k * split_stride + rh) * p.slot_stride + s);
+                    if (v != ninf) w += ex2f(v - lse);
+                }
+                p.mass[rh * p.mass_stride + s] = w;
+            }
+        }
+        return;
+    }
+
     // every lane needs every split's log-sum-exp: lane k loads split k (and k + 32), then shuffles
     float my0 = lane < p.n_splits ? p.part_lse[lane * split_stride + rh] : ninf;
     float my1 = lane + 32 < p.n_splits ? p.part_lse[(lane + 32) * split_stride + rh] : ninf;
