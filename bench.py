@@ -132,13 +132,27 @@ def oracle_sample(wl, seconds_target: float = 15.0):
     work, dt, n_calls, n_rows = 0.0, 0.0, 0, 0
     layer, t_dec = 0, wl.decode_steps - 1 if wl.decode_steps else 0
     row_budget = None
-    while dt < seconds_target and (layer < wl.n_layers or (wl.decode_steps and t_dec > 0)):
-        if layer >= wl.n_layers:                    # decode: all layers of this step done, take an earlier step
-            layer, t_dec = 0, t_dec - 1
-        k, v = wl.pool_kv(layer, b, "cpu")
-        ks = [k[offs[g]:offs[g + 1]] for g in wl.sel_local[b]]
-        vs = [v[offs[g]:offs[g + 1]] for g in wl.sel_local[b]]
-        q, kn, vn = wl.new_qkv(layer, "cpu")
+    dec_layers = min(4, wl.n_layers)            # decode: a few layers' pools are drawn once, then step after step
+    drawn = {}
+
+    def draw(layer):
+        if layer not in drawn:
+            k, v = wl.pool_kv(layer, b, "cpu")
+            drawn[layer] = ([k[offs[g]:offs[g + 1]] for g in wl.sel_local[b]],
+                            [v[offs[g]:offs[g + 1]] for g in wl.sel_local[b]], wl.new_qkv(layer, "cpu"))
+        return drawn[layer]
+
+    while dt < seconds_target:
+        if wl.decode_steps:
+            if layer >= dec_layers:
+                layer, t_dec = 0, t_dec - 1
+            if t_dec < 0:
+                break
+        elif layer >= wl.n_layers:
+            break
+        ks, vs, (q, kn, vn) = draw(layer)
+        if not wl.decode_steps:
+            drawn.pop(layer)                     # prefill: one pass per layer, do not keep the pool
         if wl.decode_steps:
             q, kn, vn = q[t_dec:t_dec + 1], kn[:t_dec + 1], vn[:t_dec + 1]
             rows = [0]
@@ -164,7 +178,7 @@ def oracle_sample(wl, seconds_target: float = 15.0):
         layer += 1
     if wl.decode_steps:
         value, unit = work / dt / 1e9, "GB/s"
-        what = f"{n_calls} (layer, step) pairs, steps {t_dec}..{wl.decode_steps - 1}, layers in order"
+        what = f"{n_calls} (layer, step) pairs: layers 0..{dec_layers - 1} of steps {max(t_dec, 0)}..{wl.decode_steps - 1}"
     else:
         value, unit = work / dt / 1e12, "TFLOP/s"
         what = f"layers 0..{n_calls - 1}, {n_rows} query rows in all"
@@ -343,7 +357,13 @@ def main():
         hv = [x.cpu().pin_memory() for x in vns]
         ho = [torch.empty_like(o, device="cpu").pin_memory() for o in outs]
         hm = [torch.empty_like(m, device="cpu").pin_memory() for m in masses]
-        dq, dk, dv = torch.empty_like(qs[0]), torch.empty_like(kns[0]), torch.empty_like(vns[0])
+        # Two sets of device input buffers and two copy streams: the upload of layer l + 1 and the download of
+        # layer l - 1 run while layer l computes (PCIe is full duplex); events order them against the stream the
+        # library launches on.
+        dbuf = [(torch.empty_like(qs[0]), torch.empty_like(kns[0]), torch.empty_like(vns[0])) for _ in range(2)]
+        main = torch.cuda.current_stream(dev)
+        s_up, s_dn = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+        ev_free = [None, None]
 
         def e2e_step(i):
             t = (i % wl.decode_steps) if wl.decode_steps else None
@@ -361,14 +381,29 @@ def main():
                     bi += hq[layer][t:t + 1].nbytes + 2 * hk[layer][t:t + 1].nbytes
                     attend(layer, qs[layer], kns[layer], vns[layer], outs[layer], masses[layer], t)
                 else:
-                    dq.copy_(hq[layer], non_blocking=True)
-                    dk.copy_(hk[layer], non_blocking=True)
-                    dv.copy_(hv[layer], non_blocking=True)
+                    dq, dk, dv = dbuf[layer & 1]
+                    with torch.cuda.stream(s_up):
+                        if ev_free[layer & 1] is not None:
+                            s_up.wait_event(ev_free[layer & 1])      # the attend that last read this buffer set
+                        dq.copy_(hq[layer], non_blocking=True)
+                        dk.copy_(hk[layer], non_blocking=True)
+                        dv.copy_(hv[layer], non_blocking=True)
+                        ev_up = torch.cuda.Event()
+                        ev_up.record(s_up)
+                    main.wait_event(ev_up)
                     bi += hq[layer].nbytes + hk[layer].nbytes + hv[layer].nbytes
                     attend(layer, dq, dk, dv, outs[layer], masses[layer], t)
-                ho[layer].copy_(outs[layer], non_blocking=True)
-                hm[layer].copy_(masses[layer], non_blocking=True)
+                ev_done = torch.cuda.Event()
+                ev_done.record(main)
+                ev_free[layer & 1] = ev_done
+                with torch.cuda.stream(s_dn):
+                    s_dn.wait_event(ev_done)
+                    ho[layer].copy_(outs[layer], non_blocking=True)
+                    hm[layer].copy_(masses[layer], non_blocking=True)
                 bo += ho[layer].nbytes + hm[layer].nbytes
+            ev_last = torch.cuda.Event()
+            ev_last.record(s_dn)
+            main.wait_event(ev_last)                                 # the step ends when its results are on the host
             return bi, bo
 
         for i in range(3):

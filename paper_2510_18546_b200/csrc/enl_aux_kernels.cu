@@ -15,6 +15,8 @@ __global__ void page_scatter_kernel(uint4 *__restrict__ kpool, uint4 *__restrict
                                     int Hkv, int chunks_per_row)
 {
     const long long total = static_cast<long long>(n_tokens) * Hkv * chunks_per_row;
+    pdl_trigger();
+    pdl_wait();                                             // an attention kernel may still be reading these pages
     for (long long id = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; id < total;
          id += static_cast<long long>(gridDim.x) * blockDim.x) {
         const int ch = static_cast<int>(id % chunks_per_row);
@@ -169,10 +171,19 @@ cudaError_t launch_page_scatter(void *kpool_layer, void *vpool_layer, const void
     const int threads = 256;
     long long blocks = (total + threads - 1) / threads;
     if (blocks > 148 * 8) blocks = 148 * 8;
-    page_scatter_kernel<<<static_cast<int>(blocks), threads, 0, st>>>(
-        static_cast<uint4 *>(kpool_layer), static_cast<uint4 *>(vpool_layer), static_cast<const uint4 *>(k),
-        static_cast<const uint4 *>(v), run, first_pos, n_tokens, Hkv, cpr);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(blocks));
+    cfg.blockDim = dim3(threads);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, page_scatter_kernel, static_cast<uint4 *>(kpool_layer),
+                                             static_cast<uint4 *>(vpool_layer), static_cast<const uint4 *>(k),
+                                             static_cast<const uint4 *>(v), run, first_pos, n_tokens, Hkv, cpr);
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 cudaError_t launch_combine(const CombineParams &p, cudaStream_t st)
