@@ -584,7 +584,9 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
             const float m_cand = mx_ref * scale;
             const bool need = m_cand > m + kRescaleThreshold;       // also true when m == -inf < m_cand
             if (__any_sync(0xffffffffu, need)) {                     // same rows, same decision in both halves
-                const float m_new = fmaxf(m, m_cand);
+                // the reference moves by at most kMaxJump per tile, so that the rescale factor cannot underflow
+                // (only a row that has already been reported as out of range is ever held back by this)
+                const float m_new = (m == kNegInf) ? m_cand : fminf(fmaxf(m, m_cand), m + kMaxJump);
                 const float alpha = (m_new == kNegInf) ? 1.f : ex2(m - m_new);
                 l *= alpha;
                 acc *= alpha;
@@ -603,7 +605,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                 }
             }
             const float m_use = (m == kNegInf) ? 0.f : m;
-            if (!sync_tile && __any_sync(0xffffffffu, mx * scale > m_use + kMaxJump)) {
+            if (__any_sync(0xffffffffu, mx * scale > m_use + kMaxJump)) {
                 // beyond what the lagging reference can carry: keep the result finite and report it
                 if (mx * scale > m_use + kMaxJump) atomicExch(p.status, 3);
                 const float cap = (m_use + kMaxJump) / scale;

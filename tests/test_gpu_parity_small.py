@@ -113,3 +113,47 @@ def test_append_keeps_existing_rows():
         assert list(sel_off) == [0, 66, 96]
         qo, mo, _ = s.oracle(0, 0, q, kn, vn)
         check_close(out, qo, mass, mo, what="append")
+
+
+def _crafted_jump(k_second: float):
+    """Two 128-token groups: zero keys in the first, constant keys in the second, so that every score of the
+    second KV tile exceeds every score of the first by q.k/sqrt(D) = 16 * k_second * 128 / sqrt(128)."""
+    dev = torch.device("cuda:0")
+    Hq, Hkv, D, n = 8, 2, 128, 40
+    g = torch.Generator(device=dev).manual_seed(5)
+    k0 = torch.zeros(128, Hkv, D, dtype=torch.bfloat16, device=dev)
+    k1 = torch.full((128, Hkv, D), k_second, dtype=torch.bfloat16, device=dev)
+    v0 = torch.randn(128, Hkv, D, generator=g, device=dev).to(torch.bfloat16)
+    v1 = torch.randn(128, Hkv, D, generator=g, device=dev).to(torch.bfloat16)
+    q = torch.full((n, Hq, D), 16.0, dtype=torch.bfloat16, device=dev)
+    kn = torch.zeros(n, Hkv, D, dtype=torch.bfloat16, device=dev)
+    vn = torch.randn(n, Hkv, D, generator=g, device=dev).to(torch.bfloat16)
+    cache = enl.enl_cache_create(1, Hq, Hkv, D, 2, 256, device=0, max_q_tokens=64)
+    try:
+        enl.enl_group_store(cache, 0, 0, k0, v0)
+        enl.enl_group_store(cache, 1, 0, k1, v1)
+        out = torch.empty_like(q)
+        mass = torch.zeros(n, Hq, 3, dtype=torch.float32, device=dev)
+        enl.enl_attend(cache, 0, [0, 1], q, kn, vn, out, mass)
+        torch.cuda.synchronize()
+        status = enl.enl_cache_status(cache)
+    finally:
+        enl.enl_cache_free(cache)
+    from oracle import enl_oracle as orc
+    ro, rm = orc.attend_slots(Hq, Hkv, D, [k0.cpu(), k1.cpu()], [v0.cpu(), v1.cpu()], q.cpu(), kn.cpu(), vn.cpu())
+    return status, out, mass, ro, rm
+
+
+def test_lagging_reference_carries_a_large_jump():
+    """The second key tile beats the first by 65 log2 units: far beyond the lazy-rescale threshold, still exact."""
+    status, out, mass, ro, rm = _crafted_jump(0.25)         # 16 * 0.25 * 128 / sqrt(128) * log2(e) = 65.3
+    assert status == enl.ENL_OK
+    check_close(out, ro, mass, rm, what="jump 65")
+    assert mass[:, :, 0].abs().max().item() < 1e-6 and (mass[:, :, 1] - 1).abs().max().item() < 1e-3
+
+
+def test_jump_beyond_the_range_is_reported():
+    """130 log2 units in one tile is more than the lagging reference carries: finite output, ENL_E_RANGE."""
+    status, out, mass, ro, rm = _crafted_jump(0.5)
+    assert status == enl.ENL_E_RANGE
+    assert torch.isfinite(out.float()).all() and torch.isfinite(mass).all()
