@@ -169,6 +169,55 @@ int enl_plan_inspect(const enl_cache_t *c, int32_t cap_entries, int32_t *stream_
                      int32_t *ep_stream_off, int32_t *ep_cached_tiles, int32_t *n_splits,
                      int32_t *n_items);
 
+/* ---- clustering reduce: what consumes the group mass ------------------------------------------ */
+
+#define ENL_CLUSTER_MAX_LAYERS   16
+#define ENL_CLUSTER_MAX_OBJECTS  480
+
+typedef struct {
+    int32_t n_layers;                  /* scored layers (the paper: about 1/10 of the model)          */
+    const float *const *mass;          /* HOST array of n_layers DEVICE pointers: the group_mass of   */
+                                       /*   the scoring enl_attend of each layer,                     */
+                                       /*   [n_q][n_q_heads][mass_stride] fp32                        */
+    int32_t n_q, n_q_heads, mass_stride;
+    int32_t n_groups;                  /* slots 0 .. n_groups-1 are the existing groups (the slot of  */
+                                       /*   the new tokens, if present, lies beyond and is ignored)   */
+    int32_t n_obj;                     /* newly detected objects                                      */
+    const int32_t *obj_off;            /* HOST [n_obj+1]: object o owns query rows obj_off[o] ..      */
+                                       /*   obj_off[o+1]-1 (its tokens in the new-token prompt)       */
+    float threshold;
+    float *avg;                        /* device fp32 [n_obj][n_groups]: mean mass over the object's  */
+                                       /*   rows, all q heads and all scored layers                   */
+    int32_t *assign;                   /* device int32 [n_obj]: the group with the largest average if */
+                                       /*   it exceeds threshold (lowest index on ties), else -1 =    */
+                                       /*   "open a new group"                                        */
+} enl_cluster_args_t;
+
+/*
+ * Sec. 3.3 "Attention-based Memory Clustering": "if the average attention between a newly detected
+ * object and an existing group exceeds a specific threshold, we cluster this object into the group";
+ * the paper leaves open over what the average runs and which group wins when several exceed it: here
+ * the mean over the object's token rows, q heads and scored layers of the probability mass on the
+ * group, and the group with the largest mean.  An object with an empty span gets average 0.
+ * Everything is enqueued on the stream; allocates nothing.  Errors: ENL_E_INVAL (null pointer, spans
+ * not ascending or beyond n_q, mass_stride < n_groups), ENL_E_LIMIT (more than ENL_CLUSTER_MAX_LAYERS
+ * layers or ENL_CLUSTER_MAX_OBJECTS objects per call), ENL_E_CUDA.
+ */
+int enl_cluster_assign(const enl_cluster_args_t *args, void *cuda_stream);
+
+/* ---- retrieval knapsack: what produces the select list ----------------------------------------- */
+
+/*
+ * Sec. 3.4, Eq. 1-2: choose x_i in {0,1} maximising sum (P_i - threshold) x_i subject to
+ * sum M_i x_i <= M.  Host-only integer dynamic programme: M_i are rounded UP and M rounded DOWN to
+ * multiples of `quantum` bytes (so the budget is never exceeded), groups with P_i <= threshold are
+ * never taken; of two choices with the same value the one found first (fewer late groups) is kept.  Writes the chosen group indices in ascending
+ * order to sel_out (capacity n) and returns their count, or ENL_E_INVAL / ENL_E_NOMEM (the table
+ * needs n * (M / quantum + 1) bytes).
+ */
+int enl_select_knapsack(int32_t n, const float *prob, float threshold, const int64_t *mem_bytes,
+                        int64_t budget_bytes, int64_t quantum, int32_t *sel_out);
+
 /* ---- an entry point that allocates nothing ------------------------------------------------ */
 
 #define ENL_STATIC_MAX_SEGMENTS  255                 /* cached segments per call                      */

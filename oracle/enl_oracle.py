@@ -186,3 +186,52 @@ class OracleCache:
                                    k_new[cu_new[b]:cu_new[b + 1]], v_new[cu_new[b]:cu_new[b + 1]],
                                    rows=rows))
         return res
+
+
+# ---- clustering reduce and retrieval knapsack (the consumers / producers around the attention) ----
+
+def cluster_assign(masses: Sequence[np.ndarray], obj_off: Sequence[int], n_groups: int, threshold: float):
+    """Sec. 3.3: average attention between each new object and each existing group, and the decision.
+
+    ``masses``: one ``[n_q, Hq, >= n_groups]`` array per scored layer (the per-slot mass of the scoring
+    attend); object o owns query rows ``obj_off[o]:obj_off[o+1]``.  The average runs over the object's
+    rows, all q heads and all layers (float64).  Returns ``(avg [n_obj, n_groups], assign [n_obj])`` with
+    ``assign = argmax`` (lowest index on ties) where the largest average exceeds the threshold, else -1."""
+    n_obj = len(obj_off) - 1
+    avg = np.zeros((n_obj, n_groups), dtype=np.float64)
+    assign = np.full(n_obj, -1, dtype=np.int64)
+    for o in range(n_obj):
+        r0, r1 = int(obj_off[o]), int(obj_off[o + 1])
+        total = np.zeros(n_groups, dtype=np.float64)
+        count = 0
+        for m in masses:
+            blk = np.asarray(m, dtype=np.float64)[r0:r1, :, :n_groups]
+            total += blk.sum(axis=(0, 1))
+            count += blk.shape[0] * blk.shape[1]
+        if count:
+            avg[o] = total / count
+        g = int(np.argmax(avg[o]))
+        if avg[o, g] > threshold:
+            assign[o] = g
+    return avg, assign
+
+
+def knapsack_bruteforce(prob: Sequence[float], threshold: float, mem_bytes: Sequence[int], budget_bytes: int,
+                        quantum: int):
+    """Sec. 3.4, Eq. 1-2 by enumeration: max sum (P_i - threshold) x_i  s.t.  sum M_i x_i <= M, x_i in {0,1},
+    with M_i rounded up and M rounded down to multiples of ``quantum``.  Returns ``(best value, best subsets)``:
+    every subset (as a sorted tuple) that reaches the best value within 1e-12.  Small n only."""
+    n = len(prob)
+    w = [-(-int(m) // int(quantum)) for m in mem_bytes]
+    cap = int(budget_bytes) // int(quantum)
+    best, arg = 0.0, [()]
+    for mask in range(1, 1 << n):
+        idx = tuple(i for i in range(n) if mask >> i & 1)
+        if sum(w[i] for i in idx) > cap:
+            continue
+        v = float(sum(float(np.float32(prob[i])) - float(np.float32(threshold)) for i in idx))
+        if v > best + 1e-12:
+            best, arg = v, [idx]
+        elif abs(v - best) <= 1e-12:
+            arg.append(idx)
+    return best, arg

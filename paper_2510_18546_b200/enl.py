@@ -23,7 +23,8 @@ ENL_OK, ENL_E_INVAL, ENL_E_NOGROUP, ENL_E_NOMEM, ENL_E_CUDA, ENL_E_TIMEOUT, ENL_
 ENL_STATIC_MAX_SEGMENTS, ENL_STATIC_MAX_KEYS, ENL_STATIC_SCRATCH_BYTES = 255, 65536, 4 << 20
 
 EXPORTS = ("enl_cache_create", "enl_group_store", "enl_attend", "enl_cache_free", "enl_strerror",
-           "enl_group_len", "enl_cache_status", "enl_plan_inspect", "enl_attend_static")
+           "enl_group_len", "enl_cache_status", "enl_plan_inspect", "enl_attend_static", "enl_cluster_assign",
+           "enl_select_knapsack")
 
 
 class CacheDesc(ctypes.Structure):
@@ -48,6 +49,13 @@ class StaticArgs(ctypes.Structure):
                 ("n_seg", ctypes.c_int32), ("seg_len", ctypes.c_void_p), ("n_new", ctypes.c_int32),
                 ("q", ctypes.c_void_p), ("k", ctypes.c_void_p), ("v", ctypes.c_void_p), ("out", ctypes.c_void_p),
                 ("group_mass", ctypes.c_void_p)]
+
+
+class ClusterArgs(ctypes.Structure):
+    _fields_ = [("n_layers", ctypes.c_int32), ("mass", ctypes.c_void_p), ("n_q", ctypes.c_int32),
+                ("n_q_heads", ctypes.c_int32), ("mass_stride", ctypes.c_int32), ("n_groups", ctypes.c_int32),
+                ("n_obj", ctypes.c_int32), ("obj_off", ctypes.c_void_p), ("threshold", ctypes.c_float),
+                ("avg", ctypes.c_void_p), ("assign", ctypes.c_void_p)]
 
 
 class EnlError(RuntimeError):
@@ -85,6 +93,11 @@ def lib() -> ctypes.CDLL:
         L.enl_plan_inspect.restype = ctypes.c_int
         L.enl_attend_static.argtypes = [ctypes.POINTER(StaticArgs), ctypes.c_void_p]
         L.enl_attend_static.restype = ctypes.c_int
+        L.enl_cluster_assign.argtypes = [ctypes.POINTER(ClusterArgs), ctypes.c_void_p]
+        L.enl_cluster_assign.restype = ctypes.c_int
+        L.enl_select_knapsack.argtypes = [ctypes.c_int32, ctypes.c_void_p, ctypes.c_float, ctypes.c_void_p,
+                                          ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p]
+        L.enl_select_knapsack.restype = ctypes.c_int
         _lib = L
     return _lib
 
@@ -168,6 +181,35 @@ def enl_attend_static(seg_len: Sequence[int], n_new: int, q, k, v, out, group_ma
     rc = lib().enl_attend_static(ctypes.byref(a), stream or None)
     if rc != ENL_OK:
         raise EnlError(rc, "enl_attend_static")
+
+
+def enl_cluster_assign(masses: Sequence, obj_off: Sequence[int], n_groups: int, threshold: float, avg, assign,
+                       stream: int = 0) -> None:
+    """``masses``: one fp32 CUDA tensor ``[n_q, Hq, stride]`` per scored layer (the group_mass of the scoring
+    attend); ``avg``: fp32 ``[n_obj, n_groups]``, ``assign``: int32 ``[n_obj]`` CUDA tensors (outputs)."""
+    ptrs = (ctypes.c_void_p * len(masses))(*[int(m.data_ptr()) for m in masses])
+    off = _i32(obj_off)
+    a = ClusterArgs()
+    a.n_layers, a.mass = len(masses), ctypes.cast(ptrs, ctypes.c_void_p)
+    a.n_q, a.n_q_heads, a.mass_stride = int(masses[0].shape[0]), int(masses[0].shape[1]), int(masses[0].shape[2])
+    a.n_groups, a.n_obj, a.obj_off, a.threshold = int(n_groups), len(off) - 1, _np_ptr(off), float(threshold)
+    a.avg, a.assign = _ptr(avg), _ptr(assign)
+    rc = lib().enl_cluster_assign(ctypes.byref(a), stream or None)
+    if rc != ENL_OK:
+        raise EnlError(rc, "enl_cluster_assign")
+
+
+def enl_select_knapsack(prob: Sequence[float], threshold: float, mem_bytes: Sequence[int], budget_bytes: int,
+                        quantum: int = 1 << 20) -> np.ndarray:
+    """Host-only.  Returns the selected group indices (ascending, int32)."""
+    pr = np.ascontiguousarray(np.asarray(prob, dtype=np.float32))
+    mb = np.ascontiguousarray(np.asarray(mem_bytes, dtype=np.int64))
+    out = np.zeros(max(len(pr), 1), np.int32)
+    rc = lib().enl_select_knapsack(len(pr), _np_ptr(pr), float(threshold), _np_ptr(mb), int(budget_bytes),
+                                   int(quantum), _np_ptr(out))
+    if rc < 0:
+        raise EnlError(rc, "enl_select_knapsack")
+    return out[:rc].copy()
 
 
 def enl_cache_free(cache: int) -> None:
