@@ -685,6 +685,71 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
             ok = mbar_wait(bar_o_done(i), 0, abort_flag, p.status);
             if (ok) {
                 tc_fence_after();
+                if constexpr (D == 128) {
+                    // Row-per-thread stores would touch 32 different rows per instruction.  Each warp stages its
+                    // 32 rows x 128 bytes in the (now idle) shared memory of its Q tile, 16-byte chunks swizzled by
+                    // row, and writes them out four whole 128-byte row pieces per instruction.
+                    uint8_t *stg = smem + i * C::kTileBytes + (hb * 4 + q4) * 4096;
+                    auto row_index = [&](int rr, bool &valid) -> long long {     // (row, head) index of staged row rr
+                        const int r2 = q4 * 32 + rr;
+                        const int t2 = it.t0 + i * tile_tokens + r2 / rep;
+                        valid = t2 < ep.n_q;
+                        const long long g2 = static_cast<long long>(ep.q_off) + t2;
+                        return (split_mode ? (static_cast<long long>(it.split) * p.n_q_total + g2) : g2) * p.Hq +
+                               it.kvh * rep + r2 % rep;
+                    };
+                    if (split_mode) {
+#pragma unroll 1
+                        for (int k = 0; k < 2; ++k) {               // 32 fp32 channels per pass
+                            uint32_t o[32];
+                            const int col = hb * (D / 2) + k * 32;
+                            tmem_ld32_wait(t_o + static_cast<uint32_t>(col), o);
+#pragma unroll
+                            for (int cch = 0; cch < 8; ++cch)
+                                *reinterpret_cast<float4 *>(stg + lane * 128 + ((cch ^ (lane & 7)) << 4)) =
+                                    make_float4(__uint_as_float(o[4 * cch]) * inv, __uint_as_float(o[4 * cch + 1]) * inv,
+                                                __uint_as_float(o[4 * cch + 2]) * inv, __uint_as_float(o[4 * cch + 3]) * inv);
+                            __syncwarp();
+#pragma unroll 1
+                            for (int itr = 0; itr < 8; ++itr) {
+                                const int rr = itr * 4 + (lane >> 3), cch = lane & 7;
+                                bool valid;
+                                const long long rh2 = row_index(rr, valid);
+                                const float4 v = *reinterpret_cast<const float4 *>(stg + rr * 128 + ((cch ^ (rr & 7)) << 4));
+                                if (valid) *reinterpret_cast<float4 *>(p.part_o + rh2 * D + col + cch * 4) = v;
+                            }
+                            __syncwarp();
+                        }
+                    } else {
+#pragma unroll
+                        for (int k = 0; k < 2; ++k) {               // 64 bf16 channels = 128 bytes per row
+                            uint32_t o[32];
+                            tmem_ld32_wait(t_o + static_cast<uint32_t>(hb * (D / 2) + k * 32), o);
+#pragma unroll
+                            for (int cch = 0; cch < 4; ++cch) {
+                                uint32_t w[4];
+#pragma unroll
+                                for (int y = 0; y < 4; ++y) {
+                                    const __nv_bfloat162 b = __floats2bfloat162_rn(
+                                        __uint_as_float(o[8 * cch + 2 * y]) * inv, __uint_as_float(o[8 * cch + 2 * y + 1]) * inv);
+                                    w[y] = *reinterpret_cast<const uint32_t *>(&b);
+                                }
+                                *reinterpret_cast<uint4 *>(stg + lane * 128 + (((k * 4 + cch) ^ (lane & 7)) << 4)) =
+                                    make_uint4(w[0], w[1], w[2], w[3]);
+                            }
+                        }
+                        __syncwarp();
+#pragma unroll 1
+                        for (int itr = 0; itr < 8; ++itr) {
+                            const int rr = itr * 4 + (lane >> 3), cch = lane & 7;
+                            bool valid;
+                            const long long rh2 = row_index(rr, valid);
+                            const uint4 v = *reinterpret_cast<const uint4 *>(stg + rr * 128 + ((cch ^ (rr & 7)) << 4));
+                            if (valid)
+                                *reinterpret_cast<uint4 *>(static_cast<__nv_bfloat16 *>(p.out) + rh2 * D + hb * (D / 2) + cch * 8) = v;
+                        }
+                    }
+                } else {
 #pragma unroll
                 for (int k = 0; k < D / 64; ++k) {                  // this half's D/2 output channels
                     uint32_t o[32];
@@ -714,6 +779,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                             }
                         }
                     }
+                }
                 }
             }
         }
