@@ -448,6 +448,29 @@ def main():
                    "objects": len(obj_off) - 1, "groups": n_groups, "layers": L,
                    "note": "enl_cluster_assign over the masses of the scoring layers; masses (%.0f MB) exceed L2" % (c_bytes / 1e6)}
 
+    # the slow tier (Sec. 3.2): push the step's selected groups out to pinned host memory, time loading them back
+    tier = None
+    if wl.name == "planner" and not args.no_e2e:
+        enl.enl_tier_enable(cache, wl.pool_tokens)
+        ids = [int(x) for x in sel]
+        t_ms, moved = [], 0
+        for _ in range(3):
+            for gid in ids:
+                enl.enl_group_evict(cache, gid, stream=stream)
+            torch.cuda.synchronize(dev)
+            ta, tb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            ta.record()
+            st_ = enl.enl_step_prepare(cache, ids, stream=stream)
+            tb.record()
+            torch.cuda.synchronize(dev)
+            t_ms.append(ta.elapsed_time(tb))
+            moved = st_["bytes_h2d"]
+        again = enl.enl_step_prepare(cache, ids, stream=stream)
+        tier = {"load_ms": float(np.median(t_ms)), "bytes_h2d": int(moved), "gbs": moved / (np.median(t_ms) * 1e-3) / 1e9,
+                "groups": len(ids), "layers": L, "hit_rate_when_repeated": again["n_hit"] / max(len(ids), 1),
+                "note": "enl_step_prepare after evicting the step's selected groups: one kernel copies their pages "
+                        "of all layers from the pinned host pool"}
+
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         wl0 = synth.make(args.workload)
@@ -468,7 +491,7 @@ def main():
                            "l2": "inputs larger than L2: every layer of a step reads its own pages and tensors"},
                 "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e,
                 "gpu_launches": launches_per_step * args.steps, "clocks": clk.summary(),
-                "status": "ok" if status == 0 else enl.strerror(status), "cluster_reduce": cluster,
+                "status": "ok" if status == 0 else enl.strerror(status), "cluster_reduce": cluster, "slow_tier": tier,
                 "fraction_of_nominal": achieved / (8000.0 if bound == "hbm" else 2250.0)}
         print(json.dumps(line), flush=True)
 

@@ -57,8 +57,9 @@ enum {                                            /* return codes               
     ENL_E_CUDA     = -4,   /* a CUDA call failed, or a GPU operation on a bookkeeping cache    */
     ENL_E_TIMEOUT  = -5,   /* a bounded wait inside a kernel expired (see enl_cache_status)    */
     ENL_E_LIMIT    = -6,   /* a size beyond the fixed maxima of enl_attend_static              */
-    ENL_E_RANGE    = -7    /* scores of one 128-key tile exceeded the maximum of all earlier    */
+    ENL_E_RANGE    = -7,   /* scores of one 128-key tile exceeded the maximum of all earlier    */
                            /*   keys by more than 2^100 (see enl_cache_status)                  */
+    ENL_E_EVICTED  = -8    /* the group's K/V is in the slow tier only (see enl_step_prepare)   */
 };
 
 typedef struct {
@@ -168,6 +169,39 @@ int enl_plan_inspect(const enl_cache_t *c, int32_t cap_entries, int32_t *stream_
                      int32_t *stream_meta, int32_t *n_entries, int32_t cap_batch,
                      int32_t *ep_stream_off, int32_t *ep_cached_tiles, int32_t *n_splits,
                      int32_t *n_items);
+
+/* ---- slow tier: all groups live in host memory, the selected ones are loaded once per step ------ */
+
+typedef struct {
+    int32_t n_hit;                     /* selected groups that were already in device memory          */
+    int32_t n_miss;                    /* selected groups loaded from the slow tier by this call      */
+    int32_t n_evicted;                 /* groups pushed out of device memory to make room             */
+    int64_t bytes_h2d, bytes_d2h;      /* page bytes moved, all layers, K and V                       */
+} enl_prepare_stats_t;
+
+/*
+ * Sec. 3.2: "we store all the KV cache in the slow memory and only load the selected groups into the
+ * device memory", once per planning step rather than once per decoded token.
+ * enl_tier_enable gives the cache a slow tier: a pinned host pool (same page format) for
+ * host_tokens tokens summed over groups (plus one page of slack per group).  From then on a group is in
+ * device memory, in the slow tier, or in both.
+ * enl_group_evict copies a group's pages to the slow tier (all layers; skipped when the copy there is
+ * current) and releases its device pages.
+ * enl_step_prepare makes every group of the select list device-resident before the step's attends:
+ * a resident group is a hit, any other is loaded from the slow tier once, for all layers; when the
+ * device pool is short, the least recently selected groups outside the list are evicted first.  The
+ * cache hit rate of the step (Sec. 3.4, last paragraph) is n_hit / n_sel.
+ * All copies are enqueued on the stream (kernels that read or write the pinned pool directly).
+ * enl_attend / enl_group_store on a group that is only in the slow tier return ENL_E_EVICTED.
+ * Errors: ENL_E_INVAL, ENL_E_NOGROUP, ENL_E_NOMEM (host pool or device pool too small for the
+ * request; residency is unchanged then), ENL_E_CUDA.
+ */
+int enl_tier_enable(enl_cache_t *c, int64_t host_tokens);
+int enl_group_evict(enl_cache_t *c, int32_t group_id, void *cuda_stream);
+int enl_step_prepare(enl_cache_t *c, const int32_t *sel_ids, int32_t n_sel, void *cuda_stream,
+                     enl_prepare_stats_t *stats);
+/* 1 if the group's pages are in device memory, 0 if only in the slow tier, ENL_E_* on a bad id. */
+int enl_group_resident(const enl_cache_t *c, int32_t group_id);
 
 /* ---- clustering reduce: what consumes the group mass ------------------------------------------ */
 

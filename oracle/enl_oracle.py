@@ -235,3 +235,55 @@ def knapsack_bruteforce(prob: Sequence[float], threshold: float, mem_bytes: Sequ
         elif abs(v - best) <= 1e-12:
             arg.append(idx)
     return best, arg
+
+
+class TierModel:
+    """Residency book-keeping of the slow tier (Sec. 3.2 / 3.4): which groups are in device memory, under a
+    device budget in pages, with least-recently-selected eviction.  Plain Python; the reference for the hit /
+    miss / eviction counts of enl_step_prepare."""
+
+    def __init__(self, device_pages: int, page_tokens: int = 16):
+        self.free = int(device_pages)
+        self.page_tokens = page_tokens
+        self.pages: Dict[int, int] = {}          # group -> pages
+        self.resident: Dict[int, bool] = {}
+        self.last_use: Dict[int, int] = {}
+        self.tick = 0
+
+    def store(self, gid: int, n_tokens: int) -> None:
+        need = -(-n_tokens // self.page_tokens)
+        have = self.pages.get(gid, 0)
+        assert self.resident.get(gid, True)
+        self.free -= need - have
+        assert self.free >= 0
+        self.pages[gid] = need
+        self.resident[gid] = True
+        self.last_use.setdefault(gid, 0)
+
+    def evict(self, gid: int) -> None:
+        if self.resident[gid]:
+            self.free += self.pages[gid]
+            self.resident[gid] = False
+
+    def prepare(self, sel: Sequence[int]):
+        self.tick += 1
+        uniq = list(dict.fromkeys(int(g) for g in sel))
+        hits = [g for g in uniq if self.resident[g]]
+        misses = [g for g in uniq if not self.resident[g]]
+        need = sum(self.pages[g] for g in misses)
+        evicted = []
+        if self.free < need:
+            cand = sorted((g for g in self.pages if self.resident[g] and self.pages[g] > 0 and g not in uniq),
+                          key=lambda g: (self.last_use[g], g))
+            for g in cand:
+                if self.free >= need:
+                    break
+                self.evict(g)
+                evicted.append(g)
+            assert self.free >= need
+        for g in misses:
+            self.free -= self.pages[g]
+            self.resident[g] = True
+        for g in uniq:
+            self.last_use[g] = self.tick
+        return hits, misses, evicted

@@ -159,7 +159,30 @@ __global__ void combine_kernel(const CombineParams p)
     }
 }
 
+// grid (pairs, layers, 2): one CTA moves one page of K or V of one layer, 16 bytes per thread and trip
+__global__ void page_copy_kernel(const uint8_t *src_k, const uint8_t *src_v, uint8_t *dst_k, uint8_t *dst_v,
+                                 size_t src_layer_bytes, size_t dst_layer_bytes, const int2 *pairs, int page_bytes)
+{
+    pdl_trigger();
+    pdl_wait();
+    const int2 pr = pairs[blockIdx.x];
+    const uint8_t *s = (blockIdx.z ? src_v : src_k) + src_layer_bytes * blockIdx.y + static_cast<size_t>(pr.x) * page_bytes;
+    uint8_t *d = (blockIdx.z ? dst_v : dst_k) + dst_layer_bytes * blockIdx.y + static_cast<size_t>(pr.y) * page_bytes;
+    for (int i = threadIdx.x * 16; i < page_bytes; i += blockDim.x * 16)
+        *reinterpret_cast<uint4 *>(d + i) = *reinterpret_cast<const uint4 *>(s + i);
+}
+
 }  // namespace
+
+cudaError_t launch_page_copy(const uint8_t *src_k, const uint8_t *src_v, uint8_t *dst_k, uint8_t *dst_v,
+                             size_t src_layer_bytes, size_t dst_layer_bytes, const int2 *pairs, int n_pairs,
+                             int n_layers, int page_bytes, cudaStream_t st)
+{
+    if (n_pairs <= 0) return cudaSuccess;
+    page_copy_kernel<<<dim3(n_pairs, n_layers, 2), 256, 0, st>>>(src_k, src_v, dst_k, dst_v, src_layer_bytes,
+                                                                dst_layer_bytes, pairs, page_bytes);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_page_scatter(void *kpool_layer, void *vpool_layer, const void *k, const void *v,
                                 const PageRun &run, int first_pos, int n_tokens, int Hkv, int D,

@@ -16,6 +16,11 @@ namespace {
 struct Group {
     std::vector<int32_t> pages;       // shared by all layers: positions 16*i .. 16*i+15 live in pages[i]
     std::vector<int32_t> len;         // per layer, -1 = never stored
+    // slow tier (Sec. 3.2): pages in the pinned host pool, and which copy is current
+    std::vector<int32_t> host_pages;
+    bool resident = true;             // the device pages hold the group
+    bool host_current = false;        // the host pages hold what the device pages held when last written back
+    uint64_t last_use = 0;            // tick of the last enl_step_prepare that selected the group
 };
 
 struct DeviceGuard {
@@ -96,6 +101,17 @@ struct enl_cache {
     std::vector<int32_t> seen;              // duplicate detection stamps
     int32_t stamp = 0;
 
+    // slow tier
+    bool tier = false;
+    int64_t n_host_pages = 0;
+    size_t host_layer_bytes = 0;
+    uint8_t *host_k = nullptr, *host_v = nullptr;           // pinned, [layer][page][kv head][16][D]
+    std::vector<int32_t> free_host_pages;
+    int2 *pairs_host = nullptr, *pairs_dev = nullptr;        // page moves of one enqueue (pinned staging + device copy)
+    int32_t cap_pairs = 0;
+    cudaEvent_t pairs_copied = nullptr;
+    uint64_t tick = 0;
+
     float *scratch = nullptr;
     int32_t *status_dev = nullptr;
     int32_t *counters_dev = nullptr;        // decode: finished splits per (episode, kv head)
@@ -123,8 +139,14 @@ void destroy(enl_cache *c)
         if (c->status_dev) cudaFree(c->status_dev);
         if (c->counters_dev) cudaFree(c->counters_dev);
         if (c->plan_copied) cudaEventDestroy(c->plan_copied);
+        if (c->host_k) cudaFreeHost(c->host_k);
+        if (c->host_v) cudaFreeHost(c->host_v);
+        if (c->pairs_host) cudaFreeHost(c->pairs_host);
+        if (c->pairs_dev) cudaFree(c->pairs_dev);
+        if (c->pairs_copied) cudaEventDestroy(c->pairs_copied);
     } else {
         delete[] c->plan_host;
+        delete[] c->pairs_host;
     }
     delete c;
 }
@@ -144,6 +166,7 @@ extern "C" const char *enl_strerror(int code)
         case ENL_E_TIMEOUT: return "a bounded wait inside a kernel expired";
         case ENL_E_LIMIT: return "size beyond the fixed maxima of the entry point that allocates nothing";
         case ENL_E_RANGE: return "scores rose by more than 2^100 within one key tile; probabilities were clamped";
+        case ENL_E_EVICTED: return "the group is in the slow tier only; enl_step_prepare loads it";
         default: return "unknown error";
     }
 }
@@ -281,6 +304,7 @@ extern "C" int enl_group_store(enl_cache_t *c, int32_t group_id, int32_t layer, 
         if ((reinterpret_cast<uintptr_t>(k_dev) | reinterpret_cast<uintptr_t>(v_dev)) & 15) return ENL_E_INVAL;
     }
     Group &g = c->groups[group_id];
+    if (!g.resident) return ENL_E_EVICTED;
     const int32_t old_len = g.len.empty() ? -1 : g.len[layer];
     const int64_t new_len64 = (mode == ENL_APPEND && old_len > 0) ? static_cast<int64_t>(old_len) + n_tokens : n_tokens;
     if (new_len64 > 0x3fffffff) return ENL_E_INVAL;
@@ -297,6 +321,7 @@ extern "C" int enl_group_store(enl_cache_t *c, int32_t group_id, int32_t layer, 
         c->free_pages.pop_back();
     }
     g.len[layer] = new_len;
+    g.host_current = false;                                  // the device copy is newer now
     int keep = 0;
     for (int l = 0; l < c->d.n_layers; ++l) keep = std::max(keep, ceil_div(std::max(g.len[l], 0), kPageTokens));
     while (static_cast<int>(g.pages.size()) > keep) {       // pages no layer needs any more
@@ -373,6 +398,7 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
             if (gid < 0 || gid >= d.max_groups) return ENL_E_NOGROUP;
             const Group &g = c->groups[gid];
             if (g.len.empty() || g.len[a->layer] < 0) return ENL_E_NOGROUP;
+            if (!g.resident) return ENL_E_EVICTED;
             if (c->seen[gid] == c->stamp) return ENL_E_INVAL;
             c->seen[gid] = c->stamp;
             sel_len[s] = g.len[a->layer];
@@ -639,6 +665,224 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
         cp.n_splits = p.n_splits;
         if (launch_combine(cp, st) != cudaSuccess) { cudaGetLastError(); return ENL_E_CUDA; }
     }
+    return ENL_OK;
+}
+
+
+// ---- slow tier (Sec. 3.2) -------------------------------------------------------------------------
+
+namespace {
+
+int page_bytes_of(const enl_cache *c) { return c->d.n_kv_heads * kPageTokens * c->d.head_dim * 2; }
+
+// Enqueues the page moves collected in c->pairs_host[0 .. n): direction to_host or to_device.
+int enqueue_moves(enl_cache *c, int n, bool to_host, cudaStream_t st)
+{
+    if (!c->gpu || n == 0) return ENL_OK;
+    // the pinned staging list is free again as soon as this upload has run (the event), the device list when the
+    // copy kernel behind it has (stream order)
+    if (cudaMemcpyAsync(c->pairs_dev, c->pairs_host, sizeof(int2) * n, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaEventRecord(c->pairs_copied, st) != cudaSuccess) {
+        cudaGetLastError();
+        return ENL_E_CUDA;
+    }
+    const cudaError_t e = to_host
+        ? launch_page_copy(c->kpool, c->vpool, c->host_k, c->host_v, c->layer_bytes, c->host_layer_bytes, c->pairs_dev, n,
+                           c->d.n_layers, page_bytes_of(c), st)
+        : launch_page_copy(c->host_k, c->host_v, c->kpool, c->vpool, c->host_layer_bytes, c->layer_bytes, c->pairs_dev, n,
+                           c->d.n_layers, page_bytes_of(c), st);
+    if (e != cudaSuccess) { cudaGetLastError(); return ENL_E_CUDA; }
+    return ENL_OK;
+}
+
+// The staging list is reused by the next enqueue: wait until the previous upload of it has been consumed.
+bool staging_free(enl_cache *c)
+{
+    return !c->gpu || cudaEventSynchronize(c->pairs_copied) == cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" int enl_tier_enable(enl_cache_t *c, int64_t host_tokens)
+{
+    if (!c || host_tokens <= 0 || c->tier) return ENL_E_INVAL;
+    const int64_t n_host = (host_tokens + kPageTokens - 1) / kPageTokens + c->d.max_groups;
+    if (n_host > 0x7fffffffll) return ENL_E_INVAL;
+    c->n_host_pages = n_host;
+    c->host_layer_bytes = static_cast<size_t>(n_host) * page_bytes_of(c);
+    c->cap_pairs = static_cast<int32_t>(std::max<int64_t>(c->n_pages, 16));
+    if (c->gpu) {
+        DeviceGuard g(c->d.device);
+        const size_t bytes = c->host_layer_bytes * c->d.n_layers;
+        const bool okm = cudaMallocHost(&c->host_k, bytes) == cudaSuccess && cudaMallocHost(&c->host_v, bytes) == cudaSuccess &&
+                         cudaMallocHost(&c->pairs_host, sizeof(int2) * c->cap_pairs) == cudaSuccess &&
+                         cudaMalloc(&c->pairs_dev, sizeof(int2) * c->cap_pairs) == cudaSuccess &&
+                         cudaEventCreateWithFlags(&c->pairs_copied, cudaEventDisableTiming) == cudaSuccess &&
+                         cudaEventRecord(c->pairs_copied, 0) == cudaSuccess;
+        if (!okm) {
+            cudaGetLastError();
+            if (c->host_k) cudaFreeHost(c->host_k);
+            if (c->host_v) cudaFreeHost(c->host_v);
+            if (c->pairs_host) cudaFreeHost(c->pairs_host);
+            if (c->pairs_dev) cudaFree(c->pairs_dev);
+            if (c->pairs_copied) cudaEventDestroy(c->pairs_copied);
+            c->host_k = c->host_v = nullptr;
+            c->pairs_host = c->pairs_dev = nullptr;
+            c->pairs_copied = nullptr;
+            return ENL_E_NOMEM;
+        }
+    } else {
+        c->pairs_host = new (std::nothrow) int2[c->cap_pairs];
+        if (!c->pairs_host) return ENL_E_NOMEM;
+    }
+    c->free_host_pages.reserve(n_host);
+    for (int64_t pg = n_host - 1; pg >= 0; --pg) c->free_host_pages.push_back(static_cast<int32_t>(pg));
+    c->tier = true;
+    return ENL_OK;
+}
+
+extern "C" int enl_group_resident(const enl_cache_t *c, int32_t group_id)
+{
+    if (!c) return ENL_E_INVAL;
+    if (group_id < 0 || group_id >= c->d.max_groups) return ENL_E_NOGROUP;
+    return c->groups[group_id].resident ? 1 : 0;
+}
+
+namespace {
+
+// Writes group g back (if its host copy is stale) and releases its device pages.  `n` = moves already
+// collected in the staging list; returns the new count, or a negative error with nothing changed.
+int evict_one(enl_cache *c, Group &g, int n, int64_t *bytes_d2h)
+{
+    const int np = static_cast<int>(g.pages.size());
+    if (!g.host_current) {
+        const int have = static_cast<int>(g.host_pages.size());
+        if (np > have && static_cast<size_t>(np - have) > c->free_host_pages.size()) return ENL_E_NOMEM;
+        if (n + np > c->cap_pairs) return ENL_E_NOMEM;
+        for (int i = have; i < np; ++i) { g.host_pages.push_back(c->free_host_pages.back()); c->free_host_pages.pop_back(); }
+        while (static_cast<int>(g.host_pages.size()) > np) { c->free_host_pages.push_back(g.host_pages.back()); g.host_pages.pop_back(); }
+        for (int i = 0; i < np; ++i) c->pairs_host[n++] = make_int2(g.pages[i], g.host_pages[i]);
+        *bytes_d2h += static_cast<int64_t>(np) * page_bytes_of(c) * 2 * c->d.n_layers;
+        g.host_current = true;
+    }
+    for (int i = np - 1; i >= 0; --i) c->free_pages.push_back(g.pages[i]);
+    g.pages.clear();
+    g.resident = false;
+    return n;
+}
+
+}  // namespace
+
+extern "C" int enl_group_evict(enl_cache_t *c, int32_t group_id, void *cuda_stream)
+{
+    if (!c || !c->tier) return ENL_E_INVAL;
+    if (group_id < 0 || group_id >= c->d.max_groups) return ENL_E_NOGROUP;
+    Group &g = c->groups[group_id];
+    if (g.len.empty()) return ENL_E_NOGROUP;
+    if (!g.resident) return ENL_OK;
+    DeviceGuard dg(c->gpu ? c->d.device : -1);
+    if (!staging_free(c)) { cudaGetLastError(); return ENL_E_CUDA; }
+    int64_t d2h = 0;
+    const int n = evict_one(c, g, 0, &d2h);
+    if (n < 0) return n;
+    ++c->epoch;
+    return enqueue_moves(c, n, true, static_cast<cudaStream_t>(cuda_stream));
+}
+
+extern "C" int enl_step_prepare(enl_cache_t *c, const int32_t *sel_ids, int32_t n_sel, void *cuda_stream,
+                                enl_prepare_stats_t *stats)
+{
+    if (!c || !c->tier || n_sel < 0 || (n_sel > 0 && !sel_ids)) return ENL_E_INVAL;
+    enl_prepare_stats_t stt = {0, 0, 0, 0, 0};
+    // validate, count what has to come in
+    int64_t need_pages = 0;
+    for (int s = 0; s < n_sel; ++s) {
+        const int32_t gid = sel_ids[s];
+        if (gid < 0 || gid >= c->d.max_groups) return ENL_E_NOGROUP;
+        const Group &g = c->groups[gid];
+        if (g.len.empty()) return ENL_E_NOGROUP;
+    }
+    ++c->tick;
+    if (++c->stamp == 0x7fffffff) { std::fill(c->seen.begin(), c->seen.end(), 0); c->stamp = 1; }
+    std::vector<int32_t> misses;
+    for (int s = 0; s < n_sel; ++s) {
+        const int32_t gid = sel_ids[s];
+        if (c->seen[gid] == c->stamp) continue;                       // listed twice (several episodes): once is enough
+        c->seen[gid] = c->stamp;
+        Group &g = c->groups[gid];
+        if (g.resident) { ++stt.n_hit; continue; }
+        ++stt.n_miss;
+        misses.push_back(gid);
+        need_pages += static_cast<int64_t>(g.host_pages.size());
+    }
+    // room in the device pool: evict the least recently selected groups that this step does not use
+    std::vector<int32_t> victims;
+    int64_t free_after = static_cast<int64_t>(c->free_pages.size());
+    if (free_after < need_pages) {
+        std::vector<int32_t> cand;
+        for (int32_t gid = 0; gid < c->d.max_groups; ++gid) {
+            const Group &g = c->groups[gid];
+            if (!g.len.empty() && g.resident && !g.pages.empty() && c->seen[gid] != c->stamp) cand.push_back(gid);
+        }
+        std::sort(cand.begin(), cand.end(), [&](int32_t x, int32_t y) {
+            const Group &gx = c->groups[x], &gy = c->groups[y];
+            return gx.last_use != gy.last_use ? gx.last_use < gy.last_use : x < y;
+        });
+        for (int32_t gid : cand) {
+            if (free_after >= need_pages) break;
+            victims.push_back(gid);
+            free_after += static_cast<int64_t>(c->groups[gid].pages.size());
+        }
+        if (free_after < need_pages) { --c->tick; return ENL_E_NOMEM; }
+    }
+    // host pages and staging room for the write-backs, checked before anything changes
+    {
+        int64_t host_need = 0, moves = 0;
+        for (int32_t gid : victims) {
+            const Group &g = c->groups[gid];
+            if (!g.host_current) {
+                host_need += std::max<int64_t>(0, static_cast<int64_t>(g.pages.size()) - static_cast<int64_t>(g.host_pages.size()));
+                moves += static_cast<int64_t>(g.pages.size());
+            }
+        }
+        if (host_need > static_cast<int64_t>(c->free_host_pages.size()) || moves > c->cap_pairs || need_pages > c->cap_pairs) {
+            --c->tick;
+            return ENL_E_NOMEM;
+        }
+    }
+    DeviceGuard dg(c->gpu ? c->d.device : -1);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (!victims.empty() || !misses.empty()) ++c->epoch;
+    if (!victims.empty()) {
+        if (!staging_free(c)) { cudaGetLastError(); return ENL_E_CUDA; }
+        int n = 0;
+        for (int32_t gid : victims) {
+            n = evict_one(c, c->groups[gid], n, &stt.bytes_d2h);
+            if (n < 0) return n;                                       // cannot happen: sizes were checked above
+            ++stt.n_evicted;
+        }
+        const int rc = enqueue_moves(c, n, true, st);
+        if (rc != ENL_OK) return rc;
+    }
+    if (!misses.empty()) {
+        if (!staging_free(c)) { cudaGetLastError(); return ENL_E_CUDA; }
+        int n = 0;
+        for (int32_t gid : misses) {
+            Group &g = c->groups[gid];
+            const int np = static_cast<int>(g.host_pages.size());
+            for (int i = 0; i < np; ++i) {
+                g.pages.push_back(c->free_pages.back());
+                c->free_pages.pop_back();
+                c->pairs_host[n++] = make_int2(g.host_pages[i], g.pages[i]);
+            }
+            g.resident = true;                                         // host copy stays current until the next store
+            stt.bytes_h2d += static_cast<int64_t>(np) * page_bytes_of(c) * 2 * c->d.n_layers;
+        }
+        const int rc = enqueue_moves(c, n, false, st);
+        if (rc != ENL_OK) return rc;
+    }
+    for (int s = 0; s < n_sel; ++s) c->groups[sel_ids[s]].last_use = c->tick;
+    if (stats) *stats = stt;
     return ENL_OK;
 }
 

@@ -134,6 +134,11 @@ struct PageRun {
 cudaError_t launch_page_scatter(void *kpool_layer, void *vpool_layer, const void *k, const void *v,
                                 const PageRun &run, int first_pos, int n_tokens,
                                 int Hkv, int D, cudaStream_t st);
+// Copies whole pages (all kv heads) between two pools of the page format, every layer, K and V: pairs[i] =
+// {source page, destination page}; the pools may be device memory or pinned host memory.
+cudaError_t launch_page_copy(const uint8_t *src_k, const uint8_t *src_v, uint8_t *dst_k, uint8_t *dst_v,
+                             size_t src_layer_bytes, size_t dst_layer_bytes, const int2 *pairs, int n_pairs,
+                             int n_layers, int page_bytes, cudaStream_t st);
 size_t attention_smem_bytes(int head_dim);
 // Opts the attention kernel into its dynamic shared memory size on the current device.
 cudaError_t prepare_attention(int head_dim);

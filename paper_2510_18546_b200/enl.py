@@ -19,12 +19,12 @@ ENL_BF16 = 1
 ENL_DEVICE_NONE = -1
 ENL_REPLACE, ENL_APPEND = 0, 1
 ENL_PLAN_ONLY = 1
-ENL_OK, ENL_E_INVAL, ENL_E_NOGROUP, ENL_E_NOMEM, ENL_E_CUDA, ENL_E_TIMEOUT, ENL_E_LIMIT, ENL_E_RANGE = 0, -1, -2, -3, -4, -5, -6, -7
+ENL_OK, ENL_E_INVAL, ENL_E_NOGROUP, ENL_E_NOMEM, ENL_E_CUDA, ENL_E_TIMEOUT, ENL_E_LIMIT, ENL_E_RANGE, ENL_E_EVICTED = 0, -1, -2, -3, -4, -5, -6, -7, -8
 ENL_STATIC_MAX_SEGMENTS, ENL_STATIC_MAX_KEYS, ENL_STATIC_SCRATCH_BYTES = 255, 65536, 4 << 20
 
 EXPORTS = ("enl_cache_create", "enl_group_store", "enl_attend", "enl_cache_free", "enl_strerror",
            "enl_group_len", "enl_cache_status", "enl_plan_inspect", "enl_attend_static", "enl_cluster_assign",
-           "enl_select_knapsack")
+           "enl_select_knapsack", "enl_tier_enable", "enl_group_evict", "enl_step_prepare", "enl_group_resident")
 
 
 class CacheDesc(ctypes.Structure):
@@ -56,6 +56,11 @@ class ClusterArgs(ctypes.Structure):
                 ("n_q_heads", ctypes.c_int32), ("mass_stride", ctypes.c_int32), ("n_groups", ctypes.c_int32),
                 ("n_obj", ctypes.c_int32), ("obj_off", ctypes.c_void_p), ("threshold", ctypes.c_float),
                 ("avg", ctypes.c_void_p), ("assign", ctypes.c_void_p)]
+
+
+class PrepareStats(ctypes.Structure):
+    _fields_ = [("n_hit", ctypes.c_int32), ("n_miss", ctypes.c_int32), ("n_evicted", ctypes.c_int32),
+                ("bytes_h2d", ctypes.c_int64), ("bytes_d2h", ctypes.c_int64)]
 
 
 class EnlError(RuntimeError):
@@ -98,6 +103,15 @@ def lib() -> ctypes.CDLL:
         L.enl_select_knapsack.argtypes = [ctypes.c_int32, ctypes.c_void_p, ctypes.c_float, ctypes.c_void_p,
                                           ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p]
         L.enl_select_knapsack.restype = ctypes.c_int
+        L.enl_tier_enable.argtypes = [ctypes.c_void_p, ctypes.c_int64]
+        L.enl_tier_enable.restype = ctypes.c_int
+        L.enl_group_evict.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p]
+        L.enl_group_evict.restype = ctypes.c_int
+        L.enl_step_prepare.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p,
+                                       ctypes.POINTER(PrepareStats)]
+        L.enl_step_prepare.restype = ctypes.c_int
+        L.enl_group_resident.argtypes = [ctypes.c_void_p, ctypes.c_int32]
+        L.enl_group_resident.restype = ctypes.c_int
         _lib = L
     return _lib
 
@@ -210,6 +224,32 @@ def enl_select_knapsack(prob: Sequence[float], threshold: float, mem_bytes: Sequ
     if rc < 0:
         raise EnlError(rc, "enl_select_knapsack")
     return out[:rc].copy()
+
+
+def enl_tier_enable(cache: int, host_tokens: int) -> None:
+    rc = lib().enl_tier_enable(cache, int(host_tokens))
+    if rc != ENL_OK:
+        raise EnlError(rc, "enl_tier_enable")
+
+
+def enl_group_evict(cache: int, group_id: int, stream: int = 0) -> None:
+    rc = lib().enl_group_evict(cache, int(group_id), stream or None)
+    if rc != ENL_OK:
+        raise EnlError(rc, "enl_group_evict")
+
+
+def enl_step_prepare(cache: int, sel_ids: Sequence[int], stream: int = 0) -> dict:
+    """Makes the selected groups device-resident; returns hits, misses, evictions and bytes moved."""
+    sel = _i32(sel_ids)
+    st = PrepareStats()
+    rc = lib().enl_step_prepare(cache, _np_ptr(sel) if len(sel) else None, len(sel), stream or None, ctypes.byref(st))
+    if rc != ENL_OK:
+        raise EnlError(rc, "enl_step_prepare")
+    return dict(n_hit=st.n_hit, n_miss=st.n_miss, n_evicted=st.n_evicted, bytes_h2d=st.bytes_h2d, bytes_d2h=st.bytes_d2h)
+
+
+def enl_group_resident(cache: int, group_id: int) -> int:
+    return int(lib().enl_group_resident(cache, int(group_id)))
 
 
 def enl_cache_free(cache: int) -> None:
