@@ -34,8 +34,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_read.sum + dram__bytes_write.sum per attention launch from the ncu capture summarised in
 # profiles/ (same kernel, same workload shape); None until a capture exists for the workload.
 NCU_TRAFFIC_BYTES = {
-    "planner": 15.46e6 + 0.07e6,      # attn_kernel<128>, profiles/attn_kernel_planner.md (the split merge is not in it)
-    "decode": 140.6e6 + 4.3e6,        # decode_kernel<128>, profiles/decode_kernel_decode.md
+    "planner": 15.41e6 + 0.03e6,      # attn_kernel<128>, profiles/attn_kernel_planner.md (the split merge is not in it)
+    "decode": 140.6e6 + 3.3e6,        # decode_kernel<128>, profiles/decode_kernel_decode.md
 }
 
 
