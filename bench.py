@@ -348,7 +348,8 @@ def main():
                 "traffic": NCU_TRAFFIC_BYTES.get(wl.name), "peak_source": peaks["_source"] +
                 (" (sustained bf16 GEMM)" if bound == "tensor" else " (copy bandwidth)"),
                 "kernel": (f"decode_kernel<{wl.head_dim}> (split merge fused)" if wl.decode_steps else
-                           f"attn_kernel<{wl.head_dim}>" + (" + combine_kernel" if n_splits > 1 else "")),
+                           f"attn_kernel<{wl.head_dim}>" + (" + combine_kernel" if plan["merge_kind"] == 1 else
+                                                            " (split merge by CTA pairs)" if plan["merge_kind"] == 2 else "")),
                 "launch_ms": attend_ms,
                 "algorithmic_per_launch": per_launch}
 
@@ -476,8 +477,8 @@ def main():
         wl0 = synth.make(args.workload)
         _, _, _, cpu = oracle_sample(wl0)
 
-    # attention (+ merge kernel when the prefill kernel splits KV; the decode kernel merges in-kernel) + page scatter
-    launches_per_step = L * (1 + (1 if (n_splits > 1 and not wl.decode_steps) else 0)) + L
+    # attention (+ merge kernel when the splits go through the scratch buffer) + page scatter
+    launches_per_step = L * (1 + (1 if plan["merge_kind"] == 1 else 0)) + L
     enl.enl_cache_free(cache)
     if rank == 0:
         line = {"metric": metric_name(wl), "value": value, "unit": unit, "n_gpus": world, "steps": args.steps,

@@ -164,11 +164,14 @@ int enl_cache_status(enl_cache_t *c);
  *   stream_pages[i], stream_meta[i] : page id and (slot << 8 | valid tokens) of KV-stream entry i
  *   ep_stream_off[b], ep_cached_tiles[b] : first entry and number of 128-key tiles of episode b
  *   n_splits : KV splits chosen;  n_items : CTAs of the attention launch
+ *   merge_kind : how the splits are merged: 0 no splits, 1 partial results in the scratch buffer and a
+ *                second (merge) kernel, 2 inside the attention kernel by pairs of CTAs (two splits,
+ *                head_dim 128), 3 inside the one-token decode kernel
  */
 int enl_plan_inspect(const enl_cache_t *c, int32_t cap_entries, int32_t *stream_pages,
                      int32_t *stream_meta, int32_t *n_entries, int32_t cap_batch,
                      int32_t *ep_stream_off, int32_t *ep_cached_tiles, int32_t *n_splits,
-                     int32_t *n_items);
+                     int32_t *n_items, int32_t *merge_kind);
 
 /* ---- slow tier: all groups live in host memory, the selected ones are loaded once per step ------ */
 

@@ -54,7 +54,9 @@ struct Cfg {
     static constexpr int kXmaxOff   = kBarOff + 512;
     static constexpr int kXsumOff   = kXmaxOff + 2 * kQTiles * 2 * 128 * 4;
     static constexpr int kXinvOff   = kXsumOff + 3 * kQTiles * kPagesPerTile * 128 * 4;
-    static constexpr int kSmemBytes = kXinvOff + kQTiles * 128 * 4 + 1024;   // + alignment slack
+    // pair merge: what the other CTA of the cluster knows about this CTA's rows, [tile][128] x (m, l, shared-slot log-sum, -)
+    static constexpr int kXpeerOff  = kXinvOff + kQTiles * 128 * 4;
+    static constexpr int kSmemBytes = kXpeerOff + kQTiles * 128 * 16 + 1024;   // + alignment slack
 };
 
 // ---- small PTX wrappers ------------------------------------------------------------------
@@ -87,6 +89,52 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
         : "=r"(ok) : "r"(bar), "r"(parity), "r"(kSuspendHintNs) : "memory");
     return ok != 0;
 }
+// The same poll with acquire semantics at cluster scope: data another CTA of the cluster wrote before its
+// release.cluster arrival is visible afterwards.  No suspend hint: a thread suspended with the long hint was seen
+// to sleep through an arrival that came from the other CTA.
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Distributed shared memory of a two-CTA cluster: address of the peer's copy of a local shared-memory location,
+// a 16-byte store to it, and an arrival (release, cluster scope) on one of its barriers.
+__device__ __forceinline__ uint32_t cluster_rank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t peer_addr(uint32_t local, uint32_t rank)
+{
+    uint32_t a;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(a) : "r"(local), "r"(rank));
+    return a;
+}
+__device__ __forceinline__ void peer_store4(uint32_t addr, float a, float b, float c, float d)
+{
+    asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+__device__ __forceinline__ void peer_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// bulk copy from this CTA's shared memory into the peer's; the bytes are counted on a barrier of the peer
+__device__ __forceinline__ void peer_bulk_copy(uint32_t dst_peer, uint32_t src_local, uint32_t bytes, uint32_t bar_peer)
+{
+    asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst_peer), "r"(src_local), "r"(bytes), "r"(bar_peer) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
 __device__ __forceinline__ unsigned long long global_ns()
 {
     unsigned long long t;
@@ -95,16 +143,18 @@ __device__ __forceinline__ unsigned long long global_ns()
 }
 // Bounded wait: gives up about kWaitLimitNs after its 16th failed poll, or when another role has raised the abort flag.
 // The result is made warp-uniform so that warp-collective tcgen05 instructions stay converged.
+template <bool kCluster = false>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
                                           int32_t *status)
 {
-    bool ok = mbar_try_wait(bar, parity);
+    auto poll = [&]() { return kCluster ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity); };
+    bool ok = poll();
     if (!ok) {
         // the clock is read only every 16 failed polls (the first reading starts the limit): a poll already
         // sleeps inside the instruction
         unsigned long long t0 = 0;
         uint32_t spins = 0;
-        while (!(ok = mbar_try_wait(bar, parity))) {
+        while (!(ok = poll())) {
             if ((++spins & 15u) == 0u) {
                 if (*abort_flag) break;
                 const unsigned long long now = global_ns();
@@ -256,6 +306,12 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
     auto bar_o_done   = [&](int i) { return bar0 + 8u * (5 + 2 * C::kStages + i); };
     auto bar_pair     = [&](int k) { return bar0 + 8u * (7 + 2 * C::kStages + k); };   // k = tile * 4 + lane quadrant
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + C::kBarOff + 8 * (15 + 2 * C::kStages));
+    // pair merge (cluster of two): the peer's row sums have arrived / the peer's partial output has arrived /
+    // the peer's K/V ring is idle and may be written
+    const uint32_t bar_peer_ml = bar0 + 8u * (16 + 2 * C::kStages);
+    const uint32_t bar_peer_o = bar0 + 8u * (17 + 2 * C::kStages);
+    const uint32_t bar_peer_free = bar0 + 8u * (18 + 2 * C::kStages);
+    const uint32_t bar_peer_ack = bar0 + 8u * (19 + 2 * C::kStages);   // the peer has received what this CTA staged for it
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     // work item
@@ -283,6 +339,11 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
             mbar_init(bar_o_done(i), 1);
         }
         for (int k = 0; k < 4 * kQTiles; ++k) mbar_init(bar_pair(k), 2);
+        mbar_init(bar_peer_ml, static_cast<uint32_t>(n_qt * 128));   // one arrival per row owner of the peer
+        mbar_init(bar_peer_o, 1);                                    // this thread's arrival below + 64 KB from the peer
+        mbar_init(bar_peer_free, 1);
+        mbar_init(bar_peer_ack, 1);
+        if (p.pair_merge) mbar_expect_tx(bar_peer_o, 8u * 8192u);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -295,6 +356,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    const bool pair = p.pair_merge != 0;
+    if (pair) cluster_sync_all();                // the peer's barriers exist before anything is sent to them
     // everything above touched only shared memory, TMEM and the gather plan; from here on the caller's tensors,
     // the pool and the scratch are read and written, so the previous kernel of the stream must have finished
     pdl_trigger();
@@ -425,6 +488,12 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                     ENL_TR(4, jj, 4 * i + 2);
                 }
             }
+            // pair merge: once every MMA of this CTA has completed, its K/V ring is idle and the peer may write
+            // into it (only a CTA that finishes a Q tile receives anything)
+            if (ok && pair && it.split < n_qt) {
+                for (int i = 0; i < n_qt && ok; ++i) ok = mbar_wait(bar_o_done(i), 0, abort_flag, p.status);
+                if (ok && lane == 0) peer_arrive(peer_addr(bar_peer_free, cluster_rank() ^ 1u));
+            }
         }
       }
     } else {
@@ -446,7 +515,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
         const uint32_t lane_sel = static_cast<uint32_t>(q4 * 32) << 16;
         const uint32_t t_s = tmem_base + lane_sel + static_cast<uint32_t>(i * 128);
         const uint32_t t_o = tmem_base + lane_sel + static_cast<uint32_t>(256 + i * 128);
-        const bool split_mode = p.n_splits > 1;
+        const bool split_mode = p.n_splits > 1 && !pair;
         const long long grow = static_cast<long long>(ep.q_off) + t;   // global query row
         const long long rh = (split_mode ? (static_cast<long long>(it.split) * p.n_q_total + grow) : grow) * p.Hq + h;
         float *slot_out = nullptr;
@@ -471,13 +540,24 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
             return done;
         };
 
+        // Pair merge: the slot in which the two splits meet is walked by both.  Split 0 writes it (adding what
+        // split 1 sends); split 1 keeps its part in `bnd` instead of storing it.
+        int shared_slot = -1, skip_slot = -1;
+        float bnd = kNegInf;
+        if (pair) {
+            const int jb = (it.split == 0) ? j_end : j_beg;         // first tile of split 1
+            const int last0 = (jb > ep.n_ctiles) ? G : (__ldg(p.stream_meta + ep.stream_off + jb * kPagesPerTile - 1) >> 8);
+            const int first1 = (jb < ep.n_ctiles) ? (__ldg(p.stream_meta + ep.stream_off + jb * kPagesPerTile) >> 8) : G;
+            if (last0 == first1) { shared_slot = last0; if (it.split == 1) skip_slot = last0; }
+        }
         float m = kNegInf, l = 0.f, acc = 0.f;                     // l, acc: owner only
         float mx_prev = kNegInf;                                   // this thread's maximum of the previous tile (unscaled)
         int cur_slot = -1;
         // a page's sum goes to its slot; a slot that ends parks its log2-sum-exp
         auto credit = [&](int slot, float v, float m_ref) {
             if (slot != cur_slot) {
-                if (slot_out && cur_slot >= 0) slot_out[cur_slot] = lg2(acc) + m_ref;
+                if (cur_slot == skip_slot) bnd = lg2(acc) + m_ref;
+                else if (slot_out && cur_slot >= 0) slot_out[cur_slot] = lg2(acc) + m_ref;
                 acc = 0.f;
                 cur_slot = slot;
             }
@@ -655,10 +735,27 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
         if (ok) {
             if (owner && n_tiles > 0) credit_tile(n_tiles - 1, 1.f, m_use);
             const float inv = (l > 0.f) ? 1.f / l : 0.f;
+            float pair_lse = kNegInf, pair_bnd = kNegInf;
             if (owner) {
-                if (slot_out && cur_slot >= 0) slot_out[cur_slot] = lg2(acc) + m_use;
+                if (cur_slot == skip_slot && cur_slot >= 0) bnd = lg2(acc) + m_use;
+                else if (slot_out && cur_slot >= 0) slot_out[cur_slot] = lg2(acc) + m_use;
                 const float lse = (l > 0.f) ? m_use + lg2(l) : kNegInf;
-                if (split_mode) {
+                if (pair) {
+                    // the two CTAs of the cluster tell each other (reference, sum, shared-slot part) of every row
+                    const uint32_t peer = cluster_rank() ^ 1u;
+                    const uint32_t mine = sbase + static_cast<uint32_t>(C::kXpeerOff + (i * 128 + r) * 16);
+                    peer_store4(peer_addr(mine, peer), m_use, l, bnd, 0.f);
+                    peer_arrive(peer_addr(bar_peer_ml, peer));
+                    ok = mbar_wait<true>(bar_peer_ml, 0, abort_flag, p.status);
+                    const float4 pe = *reinterpret_cast<const float4 *>(smem + C::kXpeerOff + (i * 128 + r) * 16);
+                    const bool va = l > 0.f, vb = pe.y > 0.f;
+                    const float M = fmaxf(va ? m_use : kNegInf, vb ? pe.x : kNegInf);
+                    const float fa = va ? ex2(m_use - M) : 0.f;
+                    const float L = (va ? l * fa : 0.f) + (vb ? pe.y * ex2(pe.x - M) : 0.f);
+                    pair_lse = (L > 0.f) ? M + lg2(L) : kNegInf;
+                    pair_bnd = pe.z;
+                    *xinv = (L > 0.f) ? fa / L : 0.f;                // weight of this CTA's unnormalised O
+                } else if (split_mode) {
                     if (row_valid) {
                         // slots this split did not walk contribute nothing
                         int first = G + 1, last = -1;
@@ -673,19 +770,126 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                                 if (sl < first || sl > last) slot_out[sl] = kNegInf;
                         p.part_lse[rh] = lse;
                     }
-                } else if (slot_out) {
-                    for (int sl = 0; sl <= G; ++sl) slot_out[sl] = ex2(slot_out[sl] - lse);
                 }
-                *xinv = inv;
+                if (!pair) *xinv = inv;
+                // the row's final log-sum-exp (and the other split's part of the shared slot) for both halves: the
+                // maximum exchange area is idle after the loop
+                xmax_own[0] = pair ? pair_lse : lse;
+                xmax_own[kXmaxPar] = pair_bnd;
             }
-            ok = pair_sync();                                       // 1 / row sum reaches half B
+            if (ok) ok = pair_sync();                               // 1 / row sum (pair merge: the weight) reaches half B
         }
+        // Masses: parked log-sums -> shares of the row's total, eight slots at a time (eight loads in flight; one
+        // load, one exponential and one store per trip would pay a memory round trip per slot).  Without a peer the
+        // owner does them while half B already writes its output channels and the last MMAs drain.  In a pair both
+        // halves share them, after the output: the other CTA waits for that.  (Both orders were timed.)
+        auto finish_masses = [&]() {
+            if (!(row_valid && p.mass && !split_mode) || (!pair && !owner)) return;
+            float *slots = p.mass + rh * p.mass_stride;
+            const float *xref = owner ? xmax_own : xmax_other;      // written by the owner before the last pair sync
+            const float ref = xref[0], extra = xref[kXmaxPar];
+            int first = 0, last = G;
+            if (pair) {                                             // the slots this CTA walked
+                first = (j_beg < ep.n_ctiles) ? (p.stream_meta[ep.stream_off + j_beg * kPagesPerTile] >> 8) : G;
+                last = (j_end > ep.n_ctiles) ? G : (p.stream_meta[ep.stream_off + j_end * kPagesPerTile - 1] >> 8);
+            }
+            for (int s0 = first + (pair ? 8 * hb : 0); s0 <= last; s0 += (pair ? 16 : 8)) {
+                float v[8];
+#pragma unroll
+                for (int x = 0; x < 8; ++x) v[x] = (s0 + x <= last) ? slots[s0 + x] : kNegInf;
+#pragma unroll
+                for (int x = 0; x < 8; ++x) {
+                    const int sl = s0 + x;
+                    if (sl <= last && sl != skip_slot) {            // the shared slot is written by split 0 alone
+                        float w = (ref != kNegInf) ? ex2(v[x] - ref) : 0.f;
+                        if (sl == shared_slot && ref != kNegInf) w += ex2(extra - ref);
+                        slots[sl] = w;
+                    }
+                }
+            }
+        };
+        const bool masses_first = !pair;
+        if (ok && masses_first) finish_masses();
+        bool exported = false;
         if (ok && n_tiles > 0) {
             const float inv = *xinv;
             ok = mbar_wait(bar_o_done(i), 0, abort_flag, p.status);
             if (ok) {
                 tc_fence_after();
                 if constexpr (D == 128) {
+                  if (pair) {
+                    // This CTA finishes Q tile `it.split` and hands the other tile's weighted partial output to the
+                    // peer, which finishes that one.  Partials travel row-per-thread into the peer's idle K/V ring
+                    // (8 KB per warp, 16-byte chunks swizzled by row); thread (warp, lane) of the receiver reads what
+                    // thread (warp, lane) of the sender wrote.
+                    const uint32_t peer = cluster_rank() ^ 1u;
+                    const uint32_t ring_off = static_cast<uint32_t>(kQTiles * C::kTileBytes + (hb * 4 + q4) * 8192 + lane * 256);
+                    constexpr uint32_t kExportStageOff = 65536;     // upper half of the ring (D = 128: 4 stages x 32 KB)
+                    if (i == it.split) {
+                        uint8_t *stg = smem + i * C::kTileBytes + (hb * 4 + q4) * 4096;
+#pragma unroll 1
+                        for (int k = 0; k < 2 && ok; ++k) {         // 32 channels per pass
+                            uint32_t o[32];
+                            tmem_ld32_wait(t_o + static_cast<uint32_t>(hb * (D / 2) + k * 32), o);
+                            if (k == 0) {
+                                ok = mbar_wait<true>(bar_peer_o, 0, abort_flag, p.status);
+                                // the peer may retire once its staging area has been read out: tell it
+                                if (ok && hb == 0 && q4 == 0 && lane == 0) peer_arrive(peer_addr(bar_peer_ack, peer));
+                            }
+                            if (!ok) break;
+#pragma unroll
+                            for (int cch = 0; cch < 4; ++cch) {
+                                const float4 a = *reinterpret_cast<const float4 *>(smem + ring_off + (((k * 8 + 2 * cch) ^ (lane & 7)) << 4));
+                                const float4 b = *reinterpret_cast<const float4 *>(smem + ring_off + (((k * 8 + 2 * cch + 1) ^ (lane & 7)) << 4));
+                                const __nv_bfloat162 b0 = __floats2bfloat162_rn(fmaf(__uint_as_float(o[8 * cch + 0]), inv, a.x), fmaf(__uint_as_float(o[8 * cch + 1]), inv, a.y));
+                                const __nv_bfloat162 b1 = __floats2bfloat162_rn(fmaf(__uint_as_float(o[8 * cch + 2]), inv, a.z), fmaf(__uint_as_float(o[8 * cch + 3]), inv, a.w));
+                                const __nv_bfloat162 b2 = __floats2bfloat162_rn(fmaf(__uint_as_float(o[8 * cch + 4]), inv, b.x), fmaf(__uint_as_float(o[8 * cch + 5]), inv, b.y));
+                                const __nv_bfloat162 b3 = __floats2bfloat162_rn(fmaf(__uint_as_float(o[8 * cch + 6]), inv, b.z), fmaf(__uint_as_float(o[8 * cch + 7]), inv, b.w));
+                                *reinterpret_cast<uint4 *>(stg + lane * 128 + (((k * 4 + cch) ^ (lane & 7)) << 4)) =
+                                    make_uint4(*reinterpret_cast<const uint32_t *>(&b0), *reinterpret_cast<const uint32_t *>(&b1),
+                                               *reinterpret_cast<const uint32_t *>(&b2), *reinterpret_cast<const uint32_t *>(&b3));
+                            }
+                        }
+                        __syncwarp();
+                        if (ok) {
+#pragma unroll 1
+                            for (int itr = 0; itr < 8; ++itr) {
+                                const int rr = itr * 4 + (lane >> 3), cch = lane & 7;
+                                const int r2 = q4 * 32 + rr;
+                                const int t2 = it.t0 + i * tile_tokens + r2 / rep;
+                                const long long rh2 = (static_cast<long long>(ep.q_off) + t2) * p.Hq + it.kvh * rep + r2 % rep;
+                                const uint4 v = *reinterpret_cast<const uint4 *>(stg + rr * 128 + ((cch ^ (rr & 7)) << 4));
+                                if (t2 < ep.n_q)
+                                    *reinterpret_cast<uint4 *>(static_cast<__nv_bfloat16 *>(p.out) + rh2 * D + hb * (D / 2) + cch * 8) = v;
+                            }
+                        }
+                    } else {
+                        // staged in the upper half of this CTA's own ring (idle once both tiles' MMAs are done), then
+                        // one bulk copy per warp into the lower half of the peer's ring, counted in bytes on its barrier
+                        if (n_qt == 2) ok = mbar_wait(bar_o_done(i ^ 1), 0, abort_flag, p.status);
+                        if (ok) {
+                            uint8_t *stage = smem + ring_off + kExportStageOff;
+#pragma unroll 1
+                            for (int k = 0; k < 2; ++k) {
+                                uint32_t o[32];
+                                tmem_ld32_wait(t_o + static_cast<uint32_t>(hb * (D / 2) + k * 32), o);
+#pragma unroll
+                                for (int cch = 0; cch < 8; ++cch)
+                                    *reinterpret_cast<float4 *>(stage + (((k * 8 + cch) ^ (lane & 7)) << 4)) =
+                                        make_float4(__uint_as_float(o[4 * cch]) * inv, __uint_as_float(o[4 * cch + 1]) * inv,
+                                                    __uint_as_float(o[4 * cch + 2]) * inv, __uint_as_float(o[4 * cch + 3]) * inv);
+                            }
+                            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                            __syncwarp();
+                            ok = mbar_wait<true>(bar_peer_free, 0, abort_flag, p.status);
+                            if (ok && lane == 0)
+                                peer_bulk_copy(peer_addr(sbase + ring_off - lane * 256, peer),
+                                               sbase + ring_off - lane * 256 + kExportStageOff, 8192,
+                                               peer_addr(bar_peer_o, peer));
+                            exported = ok;
+                        }
+                    }
+                  } else {
                     // Row-per-thread stores would touch 32 different rows per instruction.  Each warp stages its
                     // 32 rows x 128 bytes in the (now idle) shared memory of its Q tile, 16-byte chunks swizzled by
                     // row, and writes them out four whole 128-byte row pieces per instruction.
@@ -749,6 +953,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                                 *reinterpret_cast<uint4 *>(static_cast<__nv_bfloat16 *>(p.out) + rh2 * D + hb * (D / 2) + cch * 8) = v;
                         }
                     }
+                  }
                 } else {
 #pragma unroll
                 for (int k = 0; k < D / 64; ++k) {                  // this half's D/2 output channels
@@ -783,6 +988,9 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                 }
             }
         }
+        if (ok && !masses_first) finish_masses();
+        // what this CTA staged for its peer must have been fetched before the CTA may retire
+        if (exported) ok = mbar_wait<true>(bar_peer_ack, 0, abort_flag, p.status);
       }
     }
 
@@ -822,8 +1030,9 @@ cudaError_t launch_attention(const AttnParams &p, int head_dim, int n_items, cud
 {
     if (n_items <= 0) return cudaSuccess;
     cudaError_t e;
+    if (p.pair_merge && (head_dim != 128 || p.n_splits != 2 || (n_items & 1))) return cudaErrorInvalidValue;
     if (head_dim == 128)
-        e = launch_pdl(attn_kernel<128>, dim3(n_items), dim3(kThreads), Cfg<128>::kSmemBytes, st, p);
+        e = launch_pdl(attn_kernel<128>, dim3(n_items), dim3(kThreads), Cfg<128>::kSmemBytes, st, p, p.pair_merge ? 2u : 1u);
     else if (head_dim == 64)
         e = launch_pdl(attn_kernel<64>, dim3(n_items), dim3(kThreads), Cfg<64>::kSmemBytes, st, p);
     else

@@ -96,6 +96,7 @@ struct enl_cache {
     int32_t plan_split_hint = 0;
     bool plan_has_mass = false;
     bool plan_decode = false;               // the plan is for the one-token decode kernel
+    bool plan_pair = false;                 // two splits whose CTAs merge inside the attention kernel (cluster of two)
     std::vector<int32_t> key_sel, key_cu, key_len;   // what the current plan was built from
     int32_t plan_entries = 0, plan_items = 0, plan_splits = 1, plan_batch = 0, plan_max_slots = 0;
     std::vector<int32_t> seen;              // duplicate detection stamps
@@ -542,6 +543,10 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
         c->plan_split_hint = a->split_hint;
         c->plan_has_mass = has_mass;
         c->plan_decode = decode;
+        // Two splits of a head_dim-128 call are launched as clusters of two CTAs, which exchange their partial
+        // results through distributed shared memory: no scratch round trip and no merge kernel.  Every CTA must
+        // have at least one tile, and the items of a pair must be neighbours (they are: same tile count, stable sort).
+        c->plan_pair = !decode && n_splits == 2 && d.head_dim == 128 && min_tiles >= 2;
         c->key_sel.assign(a->sel_ids, a->sel_ids + a->n_sel);
         c->key_cu = cu_key;
         c->key_len = sel_len;
@@ -640,8 +645,10 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
     p.rep = c->rep;
     p.mass_stride = a->mass_stride;
     p.n_splits = c->plan_splits;
+    p.pair_merge = c->plan_pair ? 1 : 0;
     p.scale_log2 = 1.4426950408889634f / sqrtf(static_cast<float>(d.head_dim));
-    if (p.n_splits > 1) {
+    const bool scratch_merge = p.n_splits > 1 && !c->plan_pair;
+    if (scratch_merge) {
         const size_t rows = static_cast<size_t>(p.n_splits) * a->n_q * d.n_q_heads;
         p.part_o = c->scratch;
         p.part_lse = c->scratch + rows * d.head_dim;
@@ -649,7 +656,7 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
         p.mass_stride = slot_stride;                 // the partial slot buffer is packed
     }
     if (launch_attention(p, d.head_dim, c->plan_items, st) != cudaSuccess) { cudaGetLastError(); return ENL_E_CUDA; }
-    if (p.n_splits > 1) {
+    if (scratch_merge) {
         CombineParams cp;
         cp.part_o = p.part_o;
         cp.part_lse = p.part_lse;
@@ -888,13 +895,14 @@ extern "C" int enl_step_prepare(enl_cache_t *c, const int32_t *sel_ids, int32_t 
 
 extern "C" int enl_plan_inspect(const enl_cache_t *cc, int32_t cap_entries, int32_t *stream_pages, int32_t *stream_meta,
                                 int32_t *n_entries, int32_t cap_batch, int32_t *ep_stream_off,
-                                int32_t *ep_cached_tiles, int32_t *n_splits, int32_t *n_items)
+                                int32_t *ep_cached_tiles, int32_t *n_splits, int32_t *n_items, int32_t *merge_kind)
 {
     enl_cache *c = const_cast<enl_cache *>(cc);
     if (!c || !c->plan_valid) return ENL_E_INVAL;
     if (n_entries) *n_entries = c->plan_entries;
     if (n_splits) *n_splits = c->plan_splits;
     if (n_items) *n_items = c->plan_items;
+    if (merge_kind) *merge_kind = c->plan_decode ? 3 : c->plan_pair ? 2 : c->plan_splits > 1 ? 1 : 0;
     const int32_t *s = c->h_stream(), *m = c->h_meta();
     for (int i = 0; i < c->plan_entries && i < cap_entries; ++i) {
         if (stream_pages) stream_pages[i] = s[i];

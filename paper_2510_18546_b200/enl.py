@@ -94,7 +94,7 @@ def lib() -> ctypes.CDLL:
         L.enl_cache_status.restype = ctypes.c_int
         L.enl_plan_inspect.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p,
                                        ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p,
-                                       ctypes.c_void_p, ctypes.c_void_p]
+                                       ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
         L.enl_plan_inspect.restype = ctypes.c_int
         L.enl_attend_static.argtypes = [ctypes.POINTER(StaticArgs), ctypes.c_void_p]
         L.enl_attend_static.restype = ctypes.c_int
@@ -265,16 +265,17 @@ def enl_cache_status(cache: int) -> int:
 
 
 def enl_plan_inspect(cache: int, cap_entries: int = 1 << 16, cap_batch: int = 256):
-    """Host copy of the last gather plan: dict with stream pages/meta, per-episode offsets, splits, items."""
+    """Host copy of the last gather plan: dict with stream pages/meta, per-episode offsets, splits, items and
+    how the splits are merged (0 none, 1 merge kernel, 2 CTA pairs inside the attention kernel, 3 decode kernel)."""
     pages = np.zeros(cap_entries, np.int32)
     meta = np.zeros(cap_entries, np.int32)
     off = np.zeros(cap_batch, np.int32)
     tiles = np.zeros(cap_batch, np.int32)
-    ne, ns, ni = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32()
+    ne, ns, ni, mk = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32()
     rc = lib().enl_plan_inspect(cache, cap_entries, _np_ptr(pages), _np_ptr(meta), ctypes.byref(ne), cap_batch,
-                                _np_ptr(off), _np_ptr(tiles), ctypes.byref(ns), ctypes.byref(ni))
+                                _np_ptr(off), _np_ptr(tiles), ctypes.byref(ns), ctypes.byref(ni), ctypes.byref(mk))
     if rc != ENL_OK:
         raise EnlError(rc, "enl_plan_inspect")
     n = min(ne.value, cap_entries)
     return dict(pages=pages[:n], meta=meta[:n], n_entries=ne.value, ep_stream_off=off, ep_cached_tiles=tiles,
-                n_splits=ns.value, n_items=ni.value)
+                n_splits=ns.value, n_items=ni.value, merge_kind=mk.value)

@@ -210,3 +210,33 @@ def test_plan_is_reused_until_a_store_changes_the_cache():
         assert p3["n_entries"] == 8 and [m & 0xff for m in p3["meta"][:6]] == [16, 16, 16, 2, 16, 5]
     finally:
         enl.enl_cache_free(c)
+
+
+def test_merge_kind_follows_splits_shape_and_tile_count():
+    """Two splits of a head_dim-128 call go to CTA pairs (kind 2) only when every CTA has a tile of its own;
+    other split counts use the scratch buffer and the merge kernel (1); one query token per episode is the decode
+    kernel's business (3)."""
+    c = host_cache()
+    try:
+        for g, n in enumerate([300, 40, 7]):
+            enl.enl_group_store(c, g, 0, None, None, n_tokens=n)
+        plan(c, 0, [0, 1], 64, 64, split_hint=1)
+        assert enl.enl_plan_inspect(c)["merge_kind"] == 0
+        plan(c, 0, [0, 1], 64, 64, split_hint=2)
+        p = enl.enl_plan_inspect(c)
+        assert p["merge_kind"] == 2 and p["n_splits"] == 2 and p["n_items"] % 2 == 0
+        plan(c, 0, [0, 1], 64, 64, split_hint=3)
+        assert enl.enl_plan_inspect(c)["merge_kind"] == 1
+        plan(c, 0, [], 64, 64, split_hint=2)                    # one tile in all: a second CTA would have nothing to do
+        assert enl.enl_plan_inspect(c)["merge_kind"] == 1
+        plan(c, 0, [0, 1], 1, 9)
+        assert enl.enl_plan_inspect(c)["merge_kind"] == 3
+    finally:
+        enl.enl_cache_free(c)
+    c = host_cache(head_dim=64)
+    try:
+        enl.enl_group_store(c, 0, 0, None, None, n_tokens=300)
+        plan(c, 0, [0], 64, 64, split_hint=2)
+        assert enl.enl_plan_inspect(c)["merge_kind"] == 1
+    finally:
+        enl.enl_cache_free(c)

@@ -10,12 +10,14 @@ from tests.helpers import Session, check_close
 pytestmark = pytest.mark.gpu
 
 
-def run_case(wl, split_hint=0, layer=0):
+def run_case(wl, split_hint=0, layer=0, expect_merge=None):
     with Session(wl, [layer]) as s:
         q, kn, vn = wl.new_qkv(layer, s.device)
         out, mass, sel_off = s.attend(0, q, kn, vn, split_hint=split_hint)
         torch.cuda.synchronize()
         assert enl.enl_cache_status(s.cache) == enl.ENL_OK
+        if expect_merge is not None:
+            assert enl.enl_plan_inspect(s.cache)["merge_kind"] == expect_merge
         cs, cq, cn = wl.cu()
         so = 0
         for b in range(wl.batch):
@@ -68,6 +70,39 @@ def test_small_shapes(name, split):
     c = SMALL[name]
     wl = synth.make_small(7, 1, c["Hq"], c["Hkv"], c["D"], c["pool"], c["sel"], c["n_q"], c["n_new"], name=name)
     run_case(wl, split_hint=split)
+
+
+# Two KV splits of a head_dim-128 call are merged by pairs of CTAs inside the attention kernel.  The slot in which
+# the splits meet is credited by both: inside a group, on a group boundary, inside the new tokens.
+PAIR = {
+    "meet_inside_slot": dict(Hq=8, Hkv=2, D=128, pool=[[300, 40]], sel=[[0, 1]], n_q=[64], n_new=[64]),
+    "meet_on_boundary": dict(Hq=8, Hkv=2, D=128, pool=[[128, 128, 5]], sel=[[0, 1]], n_q=[30], n_new=[30]),
+    "meet_in_new_tokens": dict(Hq=8, Hkv=2, D=128, pool=[[100]], sel=[[0]], n_q=[400], n_new=[400]),
+    "one_q_tile_zero_len_group": dict(Hq=8, Hkv=2, D=128, pool=[[128, 0, 130]], sel=[[0, 1, 2]], n_q=[20], n_new=[20]),
+    "rep1_many_rows": dict(Hq=2, Hkv=2, D=128, pool=[[70, 90, 11]], sel=[[2, 1, 0]], n_q=[300], n_new=[333]),
+    "batch_of_three": dict(Hq=8, Hkv=2, D=128, pool=[[30, 60, 90], [5, 5, 250], [200]],
+                           sel=[[2, 0], [0, 1, 2], [0]], n_q=[70, 3, 129], n_new=[70, 10, 129]),
+}
+
+
+@pytest.mark.parametrize("name", sorted(PAIR))
+def test_pair_merge(name):
+    c = PAIR[name]
+    wl = synth.make_small(11, 1, c["Hq"], c["Hkv"], c["D"], c["pool"], c["sel"], c["n_q"], c["n_new"], name=name)
+    run_case(wl, split_hint=2, expect_merge=2)
+
+
+def test_split_merge_kinds():
+    c = SMALL["ragged_d128"]
+    wl = synth.make_small(7, 1, c["Hq"], c["Hkv"], c["D"], c["pool"], c["sel"], c["n_q"], c["n_new"], name="kinds")
+    run_case(wl, split_hint=1, expect_merge=0)
+    run_case(wl, split_hint=3, expect_merge=1)
+    c = SMALL["empty_select"]                       # one tile only: nothing for a second CTA of a pair to do
+    wl = synth.make_small(7, 1, c["Hq"], c["Hkv"], c["D"], c["pool"], c["sel"], c["n_q"], c["n_new"], name="kinds1")
+    run_case(wl, split_hint=2, expect_merge=1)
+    c = SMALL["decode_grown"]
+    wl = synth.make_small(7, 1, c["Hq"], c["Hkv"], c["D"], c["pool"], c["sel"], c["n_q"], c["n_new"], name="kinds2")
+    run_case(wl, split_hint=0, expect_merge=3)
 
 
 def test_zero_length_group_has_zero_mass():
