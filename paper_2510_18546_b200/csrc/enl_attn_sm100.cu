@@ -103,7 +103,7 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t par
     return ok != 0;
 }
 // Distributed shared memory of a two-CTA cluster: address of the peer's copy of a local shared-memory location,
-// a 16-byte store to it, and an arrival (release, cluster scope) on one of its barriers.
+// stores to it, and arrivals on its barriers.
 __device__ __forceinline__ uint32_t cluster_rank()
 {
     uint32_t r;
@@ -116,9 +116,17 @@ __device__ __forceinline__ uint32_t peer_addr(uint32_t local, uint32_t rank)
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(a) : "r"(local), "r"(rank));
     return a;
 }
-__device__ __forceinline__ void peer_store4(uint32_t addr, float a, float b, float c, float d)
+// 16-byte store into the peer's shared memory whose completion is counted (in bytes) on a barrier of the peer: the
+// sender needs no release fence, which would also wait for its earlier global stores
+__device__ __forceinline__ void peer_push4(uint32_t addr, float a, float b, float c, float d, uint32_t bar_peer)
 {
-    asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.f32 [%0], {%1, %2, %3, %4}, [%5];"
+                 ::"r"(addr), "f"(a), "f"(b), "f"(c), "f"(d), "r"(bar_peer) : "memory");
+}
+// an arrival that publishes nothing (a plain "go ahead")
+__device__ __forceinline__ void peer_arrive_relaxed(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ void peer_arrive(uint32_t bar)
 {
@@ -339,11 +347,14 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
             mbar_init(bar_o_done(i), 1);
         }
         for (int k = 0; k < 4 * kQTiles; ++k) mbar_init(bar_pair(k), 2);
-        mbar_init(bar_peer_ml, static_cast<uint32_t>(n_qt * 128));   // one arrival per row owner of the peer
+        mbar_init(bar_peer_ml, 1);                                   // this thread's arrival below + 16 bytes per row from the peer
         mbar_init(bar_peer_o, 1);                                    // this thread's arrival below + 64 KB from the peer
         mbar_init(bar_peer_free, 1);
         mbar_init(bar_peer_ack, 1);
-        if (p.pair_merge) mbar_expect_tx(bar_peer_o, 8u * 8192u);
+        if (p.pair_merge) {
+            mbar_expect_tx(bar_peer_ml, static_cast<uint32_t>(n_qt * 128 * 16));
+            mbar_expect_tx(bar_peer_o, 8u * 8192u);
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -525,7 +536,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
         }
         const float scale = p.scale_log2;
         float *xmax_own = reinterpret_cast<float *>(smem + C::kXmaxOff) + (i * 2 + hb) * 128 + r;          // + parity * kQTiles*2*128
-        const float *xmax_other = reinterpret_cast<const float *>(smem + C::kXmaxOff) + (i * 2 + (hb ^ 1)) * 128 + r;
+        float *xmax_other = reinterpret_cast<float *>(smem + C::kXmaxOff) + (i * 2 + (hb ^ 1)) * 128 + r;
         constexpr int kXmaxPar = kQTiles * 2 * 128;
         float *xsum = reinterpret_cast<float *>(smem + C::kXsumOff) + i * (kPagesPerTile * 128) + r;   // + (tile mod 3) * kQTiles*8*128 + page*128
         float *xinv = reinterpret_cast<float *>(smem + C::kXinvOff) + i * 128 + r;
@@ -731,21 +742,61 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
 
         // ---- per-row results ----
         float m_use = (m == kNegInf) ? 0.f : m;
+        bool exported = false;
+        float w_peer = 0.f;
         if (ok) ok = pair_sync();                                   // half B's sums of the last tile are in place
         if (ok) {
             if (owner && n_tiles > 0) credit_tile(n_tiles - 1, 1.f, m_use);
             const float inv = (l > 0.f) ? 1.f / l : 0.f;
             float pair_lse = kNegInf, pair_bnd = kNegInf;
+            const float lse = (l > 0.f) ? m_use + lg2(l) : kNegInf;
             if (owner) {
                 if (cur_slot == skip_slot && cur_slot >= 0) bnd = lg2(acc) + m_use;
                 else if (slot_out && cur_slot >= 0) slot_out[cur_slot] = lg2(acc) + m_use;
-                const float lse = (l > 0.f) ? m_use + lg2(l) : kNegInf;
                 if (pair) {
                     // the two CTAs of the cluster tell each other (reference, sum, shared-slot part) of every row
                     const uint32_t peer = cluster_rank() ^ 1u;
                     const uint32_t mine = sbase + static_cast<uint32_t>(C::kXpeerOff + (i * 128 + r) * 16);
-                    peer_store4(peer_addr(mine, peer), m_use, l, bnd, 0.f);
-                    peer_arrive(peer_addr(bar_peer_ml, peer));
+                    peer_push4(peer_addr(mine, peer), m_use, l, bnd, 0.f, peer_addr(bar_peer_ml, peer));
+                }
+            }
+            if constexpr (D == 128) {
+              if (pair && i != it.split && n_tiles > 0) {
+                // This CTA finishes Q tile `it.split`; the accumulator of the other tile goes to the peer, which
+                // finishes that one.  It goes as it is (relative to this CTA's own reference; the peer learns the
+                // weight from the row sums above), so that nothing but the last MMA stands before it: staged
+                // row-per-thread in the upper half of this CTA's ring (idle once both tiles' MMAs are done; 8 KB per
+                // warp, 16-byte chunks swizzled by row), then one bulk copy per warp into the lower half of the
+                // peer's ring, counted in bytes on the peer's barrier.
+                const uint32_t peer = cluster_rank() ^ 1u;
+                const uint32_t warp_off = static_cast<uint32_t>(kQTiles * C::kTileBytes + (hb * 4 + q4) * 8192);
+                constexpr uint32_t kExportStageOff = 65536;         // upper half of the ring (4 stages x 32 KB)
+                ok = mbar_wait(bar_o_done(i), 0, abort_flag, p.status);
+                if (ok && n_qt == 2) ok = mbar_wait(bar_o_done(i ^ 1), 0, abort_flag, p.status);
+                if (ok) {
+                    tc_fence_after();
+                    uint8_t *stage = smem + warp_off + kExportStageOff + lane * 256;
+#pragma unroll 1
+                    for (int k = 0; k < 2; ++k) {
+                        uint32_t o[32];
+                        tmem_ld32_wait(t_o + static_cast<uint32_t>(hb * (D / 2) + k * 32), o);
+#pragma unroll
+                        for (int cch = 0; cch < 8; ++cch)
+                            *reinterpret_cast<uint4 *>(stage + (((k * 8 + cch) ^ (lane & 7)) << 4)) =
+                                make_uint4(o[4 * cch], o[4 * cch + 1], o[4 * cch + 2], o[4 * cch + 3]);
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    ok = mbar_wait<true>(bar_peer_free, 0, abort_flag, p.status);
+                    if (ok && lane == 0)
+                        peer_bulk_copy(peer_addr(sbase + warp_off, peer), sbase + warp_off + kExportStageOff, 8192,
+                                       peer_addr(bar_peer_o, peer));
+                    exported = ok;
+                }
+              }
+            }
+            if (owner && ok) {
+                if (pair) {
                     ok = mbar_wait<true>(bar_peer_ml, 0, abort_flag, p.status);
                     const float4 pe = *reinterpret_cast<const float4 *>(smem + C::kXpeerOff + (i * 128 + r) * 16);
                     const bool va = l > 0.f, vb = pe.y > 0.f;
@@ -755,6 +806,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                     pair_lse = (L > 0.f) ? M + lg2(L) : kNegInf;
                     pair_bnd = pe.z;
                     *xinv = (L > 0.f) ? fa / L : 0.f;                // weight of this CTA's unnormalised O
+                    w_peer = (L > 0.f && vb) ? ex2(pe.x - M) / L : 0.f;   // and of the peer's
+                    xmax_other[0] = w_peer;                          // for half B (its slot of the exchange area is idle)
                 } else if (split_mode) {
                     if (row_valid) {
                         // slots this split did not walk contribute nothing
@@ -810,21 +863,18 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
         };
         const bool masses_first = !pair;
         if (ok && masses_first) finish_masses();
-        bool exported = false;
-        if (ok && n_tiles > 0) {
+        if (pair && !owner) w_peer = xmax_own[0];
+        if (ok && n_tiles > 0 && !(pair && i != it.split)) {
             const float inv = *xinv;
             ok = mbar_wait(bar_o_done(i), 0, abort_flag, p.status);
             if (ok) {
                 tc_fence_after();
                 if constexpr (D == 128) {
                   if (pair) {
-                    // This CTA finishes Q tile `it.split` and hands the other tile's weighted partial output to the
-                    // peer, which finishes that one.  Partials travel row-per-thread into the peer's idle K/V ring
-                    // (8 KB per warp, 16-byte chunks swizzled by row); thread (warp, lane) of the receiver reads what
-                    // thread (warp, lane) of the sender wrote.
+                    // This CTA finishes Q tile `it.split`: its own accumulator and what the peer sent (see the export
+                    // above), each with its weight.  Thread (warp, lane) reads what thread (warp, lane) of the peer wrote.
                     const uint32_t peer = cluster_rank() ^ 1u;
                     const uint32_t ring_off = static_cast<uint32_t>(kQTiles * C::kTileBytes + (hb * 4 + q4) * 8192 + lane * 256);
-                    constexpr uint32_t kExportStageOff = 65536;     // upper half of the ring (D = 128: 4 stages x 32 KB)
                     if (i == it.split) {
                         uint8_t *stg = smem + i * C::kTileBytes + (hb * 4 + q4) * 4096;
 #pragma unroll 1
@@ -834,17 +884,18 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                             if (k == 0) {
                                 ok = mbar_wait<true>(bar_peer_o, 0, abort_flag, p.status);
                                 // the peer may retire once its staging area has been read out: tell it
-                                if (ok && hb == 0 && q4 == 0 && lane == 0) peer_arrive(peer_addr(bar_peer_ack, peer));
+                                if (ok && hb == 0 && q4 == 0 && lane == 0) peer_arrive_relaxed(peer_addr(bar_peer_ack, peer));
                             }
                             if (!ok) break;
 #pragma unroll
                             for (int cch = 0; cch < 4; ++cch) {
                                 const float4 a = *reinterpret_cast<const float4 *>(smem + ring_off + (((k * 8 + 2 * cch) ^ (lane & 7)) << 4));
                                 const float4 b = *reinterpret_cast<const float4 *>(smem + ring_off + (((k * 8 + 2 * cch + 1) ^ (lane & 7)) << 4));
-                                const __nv_bfloat162 b0 = __floats2bfloat162_rn(fmaf(__uint_as_float(o[8 * cch + 0]), inv, a.x), fmaf(__uint_as_float(o[8 * cch + 1]), inv, a.y));
-                                const __nv_bfloat162 b1 = __floats2bfloat162_rn(fmaf(__uint_as_float(o[8 * cch + 2]), inv, a.z), fmaf(__uint_as_float(o[8 * cch + 3]), inv, a.w));
-                                const __nv_bfloat162 b2 = __floats2bfloat162_rn(fmaf(__uint_as_float(o[8 * cch + 4]), inv, b.x), fmaf(__uint_as_float(o[8 * cch + 5]), inv, b.y));
-                                const __nv_bfloat162 b3 = __floats2bfloat162_rn(fmaf(__uint_as_float(o[8 * cch + 6]), inv, b.z), fmaf(__uint_as_float(o[8 * cch + 7]), inv, b.w));
+                                auto mix = [&](uint32_t own, float theirs) { return fmaf(__uint_as_float(own), inv, theirs * w_peer); };
+                                const __nv_bfloat162 b0 = __floats2bfloat162_rn(mix(o[8 * cch + 0], a.x), mix(o[8 * cch + 1], a.y));
+                                const __nv_bfloat162 b1 = __floats2bfloat162_rn(mix(o[8 * cch + 2], a.z), mix(o[8 * cch + 3], a.w));
+                                const __nv_bfloat162 b2 = __floats2bfloat162_rn(mix(o[8 * cch + 4], b.x), mix(o[8 * cch + 5], b.y));
+                                const __nv_bfloat162 b3 = __floats2bfloat162_rn(mix(o[8 * cch + 6], b.z), mix(o[8 * cch + 7], b.w));
                                 *reinterpret_cast<uint4 *>(stg + lane * 128 + (((k * 4 + cch) ^ (lane & 7)) << 4)) =
                                     make_uint4(*reinterpret_cast<const uint32_t *>(&b0), *reinterpret_cast<const uint32_t *>(&b1),
                                                *reinterpret_cast<const uint32_t *>(&b2), *reinterpret_cast<const uint32_t *>(&b3));
@@ -862,31 +913,6 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                                 if (t2 < ep.n_q)
                                     *reinterpret_cast<uint4 *>(static_cast<__nv_bfloat16 *>(p.out) + rh2 * D + hb * (D / 2) + cch * 8) = v;
                             }
-                        }
-                    } else {
-                        // staged in the upper half of this CTA's own ring (idle once both tiles' MMAs are done), then
-                        // one bulk copy per warp into the lower half of the peer's ring, counted in bytes on its barrier
-                        if (n_qt == 2) ok = mbar_wait(bar_o_done(i ^ 1), 0, abort_flag, p.status);
-                        if (ok) {
-                            uint8_t *stage = smem + ring_off + kExportStageOff;
-#pragma unroll 1
-                            for (int k = 0; k < 2; ++k) {
-                                uint32_t o[32];
-                                tmem_ld32_wait(t_o + static_cast<uint32_t>(hb * (D / 2) + k * 32), o);
-#pragma unroll
-                                for (int cch = 0; cch < 8; ++cch)
-                                    *reinterpret_cast<float4 *>(stage + (((k * 8 + cch) ^ (lane & 7)) << 4)) =
-                                        make_float4(__uint_as_float(o[4 * cch]) * inv, __uint_as_float(o[4 * cch + 1]) * inv,
-                                                    __uint_as_float(o[4 * cch + 2]) * inv, __uint_as_float(o[4 * cch + 3]) * inv);
-                            }
-                            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                            __syncwarp();
-                            ok = mbar_wait<true>(bar_peer_free, 0, abort_flag, p.status);
-                            if (ok && lane == 0)
-                                peer_bulk_copy(peer_addr(sbase + ring_off - lane * 256, peer),
-                                               sbase + ring_off - lane * 256 + kExportStageOff, 8192,
-                                               peer_addr(bar_peer_o, peer));
-                            exported = ok;
                         }
                     }
                   } else {
