@@ -92,6 +92,22 @@ def test_pair_merge(name):
     run_case(wl, split_hint=2, expect_merge=2)
 
 
+def test_pair_merge_without_mass_and_twice_in_a_row():
+    """No mass buffer: the slot book-keeping of the pair has nowhere to write.  The second call reuses the plan and
+    the barriers' fresh state of a new launch."""
+    c = PAIR["meet_inside_slot"]
+    wl = synth.make_small(12, 1, c["Hq"], c["Hkv"], c["D"], c["pool"], c["sel"], c["n_q"], c["n_new"], name="pair_nomass")
+    with Session(wl, [0]) as s:
+        q, kn, vn = wl.new_qkv(0, s.device)
+        qo, _, _ = s.oracle(0, 0, q, kn, vn)
+        for _ in range(2):
+            out, mass, _ = s.attend(0, q, kn, vn, split_hint=2, want_mass=False)
+            torch.cuda.synchronize()
+            assert mass is None and enl.enl_cache_status(s.cache) == enl.ENL_OK
+            assert enl.enl_plan_inspect(s.cache)["merge_kind"] == 2
+            check_close(out, qo, None, None, what="pair merge without mass")
+
+
 def test_split_merge_kinds():
     c = SMALL["ragged_d128"]
     wl = synth.make_small(7, 1, c["Hq"], c["Hkv"], c["D"], c["pool"], c["sel"], c["n_q"], c["n_new"], name="kinds")
