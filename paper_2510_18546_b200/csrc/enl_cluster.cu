@@ -12,8 +12,9 @@ namespace {
 
 constexpr int kMaxLayers = ENL_CLUSTER_MAX_LAYERS;
 constexpr int kMaxObjects = ENL_CLUSTER_MAX_OBJECTS;
-constexpr int kWarps = 16;
-constexpr int kGroupsPerCta = 128;            // 32 lanes x float4
+constexpr int kWarps = 8;
+constexpr int kGroupsPerCta = 32;             // one group per lane
+constexpr int kUnroll = 16;                   // (row, head) pairs, i.e. loads, in flight per warp
 
 struct ClusterParams {
     const float *mass[kMaxLayers];
@@ -24,50 +25,42 @@ struct ClusterParams {
     int32_t *assign;
 };
 
-// grid (objects, ceil(n_groups / 128)); warp w takes (row, head) pairs w, w + 16, ... of the object's span,
-// lane l sums groups l, l + 32, l + 64, l + 96 of the CTA's 128-group chunk: every warp load is one coalesced
-// 128-byte line whatever the row stride, and four pairs (sixteen loads) are in flight per warp.
+// grid (objects, ceil(n_groups / 32)); warp w takes (row, head) pairs w, w + 8, ... of the object's span, lane l
+// sums group l of the CTA's 32-group chunk: every warp load is one coalesced 128-byte line whatever the row
+// stride, and sixteen of them are in flight per warp.  Many small CTAs (eight resident per SM) rather than few
+// large ones: with equal-sized CTAs a second, partly filled wave would cost up to half the time.
 __global__ void __launch_bounds__(kWarps * 32) cluster_avg_kernel(const __grid_constant__ ClusterParams p)
 {
     __shared__ float part[kWarps][kGroupsPerCta];
     const int obj = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int g0 = blockIdx.y * kGroupsPerCta + lane;
+    const int g = blockIdx.y * kGroupsPerCta + lane;
     const int r0 = p.obj_off[obj], r1 = p.obj_off[obj + 1];
     const long long pairs = static_cast<long long>(r1 - r0) * p.Hq;
     enl::pdl_trigger();
     enl::pdl_wait();                                   // the masses come from the attention kernels before
-    bool on[4];
-#pragma unroll
-    for (int k = 0; k < 4; ++k) on[k] = g0 + 32 * k < p.n_groups;
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    const bool on = g < p.n_groups;
+    float acc = 0.f;
     for (int l = 0; l < p.n_layers; ++l) {
-        const float *base = p.mass[l] + static_cast<long long>(r0) * p.Hq * p.mass_stride + g0;
+        const float *base = p.mass[l] + static_cast<long long>(r0) * p.Hq * p.mass_stride + g;
         long long i = warp;
-        for (; i + 3 * kWarps < pairs; i += 4 * kWarps) {
-            float v[4][4];
+        for (; i + (kUnroll - 1) * kWarps < pairs; i += kUnroll * kWarps) {
+            float v[kUnroll];
 #pragma unroll
-            for (int u = 0; u < 4; ++u)
+            for (int u = 0; u < kUnroll; ++u) v[u] = on ? __ldcs(base + (i + u * kWarps) * p.mass_stride) : 0.f;
+            // summed in the order of the pairs, as a plain loop would
 #pragma unroll
-                for (int k = 0; k < 4; ++k) v[u][k] = on[k] ? __ldcs(base + (i + u * kWarps) * p.mass_stride + 32 * k) : 0.f;
-#pragma unroll
-            for (int u = 0; u < 4; ++u)
-#pragma unroll
-                for (int k = 0; k < 4; ++k) acc[k] += v[u][k];
+            for (int u = 0; u < kUnroll; ++u) acc += v[u];
         }
         for (; i < pairs; i += kWarps)
-#pragma unroll
-            for (int k = 0; k < 4; ++k)
-                if (on[k]) acc[k] += __ldcs(base + i * p.mass_stride + 32 * k);
+            if (on) acc += __ldcs(base + i * p.mass_stride);
     }
-#pragma unroll
-    for (int k = 0; k < 4; ++k) part[warp][lane + 32 * k] = acc[k];
+    part[warp][lane] = acc;
     __syncthreads();
-    for (int gl = threadIdx.x; gl < kGroupsPerCta; gl += kWarps * 32) {
+    if (warp == 0) {
         float t = 0.f;
-        for (int w = 0; w < kWarps; ++w) t += part[w][gl];
-        const int g = blockIdx.y * kGroupsPerCta + gl;
+        for (int w = 0; w < kWarps; ++w) t += part[w][lane];
         const float inv = (pairs > 0) ? 1.f / (static_cast<float>(pairs) * static_cast<float>(p.n_layers)) : 0.f;
-        if (g < p.n_groups) p.avg[static_cast<long long>(obj) * p.n_groups + g] = t * inv;
+        if (on) p.avg[static_cast<long long>(obj) * p.n_groups + g] = t * inv;
     }
 }
 
