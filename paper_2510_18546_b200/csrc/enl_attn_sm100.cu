@@ -535,6 +535,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
             else if (p.mass) slot_out = p.mass + rh * p.mass_stride;
         }
         const float scale = p.scale_log2;
+        const float inv_scale = 1.f / scale;
         float *xmax_own = reinterpret_cast<float *>(smem + C::kXmaxOff) + (i * 2 + hb) * 128 + r;          // + parity * kQTiles*2*128
         float *xmax_other = reinterpret_cast<float *>(smem + C::kXmaxOff) + (i * 2 + (hb ^ 1)) * 128 + r;
         constexpr int kXmaxPar = kQTiles * 2 * 128;
@@ -623,52 +624,49 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
             tc_fence_after();
             if (q4 == 0) ENL_TR(warp >> 2, jj, 1);
 
-            // all 64 scores of this thread in one TMEM round trip (a round trip costs about 200 cycles)
-            float s[kHalfCols];
-            {
-                uint32_t su[kHalfCols];
-                tmem_ld64_wait(t_s + static_cast<uint32_t>(hb * kHalfCols), su);
+            // hide page padding / keys after the causal limit of page e (16 scores), and take the page's maximum
+            auto page_max = [&](int e, float (&sc)[kPageTokens]) -> float {
+                const int nv = static_cast<int>((nvp >> (8 * e)) & 0xffu);
+                if (nv < kPageTokens) {
 #pragma unroll
-                for (int x = 0; x < kHalfCols; ++x) s[x] = __uint_as_float(su[x]);
-            }
-            // hide page padding / keys after the causal limit, and take the maximum page by page
-            float mx;
-            {
-                float pm[kHalfPages];
-#pragma unroll
-                for (int e = 0; e < kHalfPages; ++e) {
-                    const int nv = static_cast<int>((nvp >> (8 * e)) & 0xffu);
-                    const int b = e * kPageTokens;
-                    if (nv < kPageTokens) {
-#pragma unroll
-                        for (int x = 0; x < kPageTokens; ++x)
-                            if (x >= nv) s[b + x] = kNegInf;
-                    }
-                    float a = fmax3(s[b], s[b + 1], s[b + 2]);
-#pragma unroll
-                    for (int x = 3; x < 15; x += 2) a = fmax3(a, s[b + x], s[b + x + 1]);
-                    pm[e] = fmaxf(a, s[b + 15]);
+                    for (int x = 0; x < kPageTokens; ++x)
+                        if (x >= nv) sc[x] = kNegInf;
                 }
-                mx = fmaxf(fmaxf(pm[0], pm[1]), fmaxf(pm[2], pm[3]));
-            }
+                float a = fmax3(sc[0], sc[1], sc[2]);
+#pragma unroll
+                for (int x = 3; x < 15; x += 2) a = fmax3(a, sc[x], sc[x + 1]);
+                return fmaxf(a, sc[15]);
+            };
+            const uint32_t t_half = t_s + static_cast<uint32_t>(hb * kHalfCols);
+
             // The reference maximum needs the other half's columns too.  Waiting for them every tile would put a
             // two-warp barrier on the critical path, so the exchange lags by one tile: this tile's exponentials
             // use the maximum over all EARLIER tiles (both halves know it: the partner's maximum of the previous
             // tile has been in shared memory since before that tile's P was handed over), and this tile's
             // maximum only moves the reference for the next one.  A probability may then exceed 1 by the factor
             // 2^(jump of this tile over everything before it), harmless in floating point up to kMaxJump.  The
-            // first tile, and any tile that starts without a reference, exchange synchronously.
+            // first tile, and any tile that starts without a reference, need their own maximum first: a pass over
+            // the scores for the maximum alone, exchanged synchronously.
             const bool sync_tile = (jj == 0) || __any_sync(0xffffffffu, m == kNegInf);   // same rows, same m in both halves
-            xmax_own[(jj & 1) * kXmaxPar] = mx;
             float mx_ref;
             if (sync_tile) {
+                float mx0 = kNegInf;
+#pragma unroll 1
+                for (int e = 0; e < kHalfPages; ++e) {
+                    uint32_t su[kPageTokens];
+                    tmem_ld16_wait(t_half + static_cast<uint32_t>(e * kPageTokens), su);
+                    float sc[kPageTokens];
+#pragma unroll
+                    for (int x = 0; x < kPageTokens; ++x) sc[x] = __uint_as_float(su[x]);
+                    mx0 = fmaxf(mx0, page_max(e, sc));
+                }
+                xmax_own[(jj & 1) * kXmaxPar] = mx0;
                 ok = pair_sync();
                 if (!ok) break;
-                mx_ref = fmaxf(mx, xmax_other[(jj & 1) * kXmaxPar]);
+                mx_ref = fmaxf(mx0, xmax_other[(jj & 1) * kXmaxPar]);
             } else {
                 mx_ref = fmaxf(mx_prev, xmax_other[((jj - 1) & 1) * kXmaxPar]);
             }
-            mx_prev = mx;
             if (q4 == 0) ENL_TR(warp >> 2, jj, 2);
 
             float late = 1.f;
@@ -696,28 +694,39 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                 }
             }
             const float m_use = (m == kNegInf) ? 0.f : m;
-            if (__any_sync(0xffffffffu, mx * scale > m_use + kMaxJump)) {
-                // beyond what the lagging reference can carry: keep the result finite and report it
-                if (mx * scale > m_use + kMaxJump) atomicExch(p.status, 3);
-                const float cap = (m_use + kMaxJump) / scale;
-#pragma unroll
-                for (int x = 0; x < kHalfCols; ++x) s[x] = fminf(s[x], cap);
-            }
+            const float cap = (m_use + kMaxJump) * inv_scale;       // largest score the reference can carry
 
-            // p = exp2(s * scale - m) page by page; the page's sum goes to shared memory (the owner credits it to
-            // its slot later), its sixteen probabilities go as eight bf16 pairs (even key in the low half) into P.
-            // Each half keeps its P inside its own 64 columns of S_i (page e at columns hb*64 + 8e .. +7).
+            // The scores are taken page by page (16 per thread and load; the next page's load is in flight while
+            // this one is worked on): mask, maximum (for the next tile's reference), p = exp2(s * scale - m).  The
+            // page's sum goes to shared memory (the owner credits it to its slot later), its sixteen probabilities
+            // go as eight bf16 pairs (even key in the low half) into P.  Each half keeps its P inside its own 64
+            // columns of S_i: page e at columns hb*64 + 8e .. +7, which only covers scores already taken.
             const uint64_t sc2 = pack2(scale, scale), nm2 = pack2(-m_use, -m_use);
             float *sum_dst = xsum + (jj % 3) * (kQTiles * kPagesPerTile * 128) + hb * (kHalfPages * 128);
+            float mx = kNegInf;
+            uint32_t su[2][kPageTokens];
+            tmem_ld16_issue(t_half, su[0]);
 #pragma unroll
             for (int e = 0; e < kHalfPages; ++e) {
+                tmem_ld16_arrived(su[e & 1]);
+                if (e + 1 < kHalfPages) tmem_ld16_issue(t_half + static_cast<uint32_t>((e + 1) * kPageTokens), su[(e + 1) & 1]);
+                float sc[kPageTokens];
+#pragma unroll
+                for (int x = 0; x < kPageTokens; ++x) sc[x] = __uint_as_float(su[e & 1][x]);
+                const float pm = page_max(e, sc);
+                mx = fmaxf(mx, pm);
+                if (pm > cap) {
+                    // beyond what the lagging reference can carry: keep the result finite and report it
+                    atomicExch(p.status, 3);
+#pragma unroll
+                    for (int x = 0; x < kPageTokens; ++x) sc[x] = fminf(sc[x], cap);
+                }
                 uint64_t pr[kPageTokens / 2];
                 uint32_t pk[kPageTokens / 2];
 #pragma unroll
                 for (int x = 0; x < kPageTokens / 2; ++x) {
-                    const int b = e * kPageTokens + 2 * x;
                     float a0, a1;
-                    unpack2(fma2(pack2(s[b], s[b + 1]), sc2, nm2), a0, a1);
+                    unpack2(fma2(pack2(sc[2 * x], sc[2 * x + 1]), sc2, nm2), a0, a1);
                     a0 = ex2(a0);
                     a1 = ex2(a1);
                     pr[x] = pack2(a0, a1);
@@ -731,6 +740,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                 unpack2(add2(q0, q1), b0, b1);
                 sum_dst[e * 128] = b0 + b1;
             }
+            if (!sync_tile) xmax_own[(jj & 1) * kXmaxPar] = mx;     // (a synchronous tile has published it already)
+            mx_prev = mx;
             if (q4 == 0) ENL_TR(warp >> 2, jj, 3);
             tmem_st_wait();
             tc_fence_before();
