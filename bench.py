@@ -362,7 +362,30 @@ def main():
         # Two sets of device input buffers and two copy streams: the upload of layer l + 1 and the download of
         # layer l - 1 run while layer l computes (PCIe is full duplex); events order them against the stream the
         # library launches on.
-        dbuf = [(torch.empty_like(qs[0]), torch.empty_like(kns[0]), torch.empty_like(vns[0])) for _ in range(2)]
+        # A layer's q | k_new | v_new travel as one copy, and so do its out | mass: fewer, larger transfers and half
+        # the host calls per layer (the C ABI takes plain pointers, so the tensors are views into the packed buffers).
+        # Queuing a whole step's uploads, attends and downloads at once was slower: the link carries about 65 GB/s
+        # in both directions together, and the per-layer interleaving keeps both directions busy all the time.
+        def packed(parts, device, pin=False):
+            sizes = [(x.nbytes + 255) // 256 * 256 for x in parts]
+            buf = torch.empty(sum(sizes), dtype=torch.uint8, device=device)
+            if pin:
+                buf = buf.pin_memory()
+            views, off = [], 0
+            for x, n in zip(parts, sizes):
+                views.append(buf[off:off + x.nbytes].view(x.dtype).view(x.shape))
+                off += n
+            return buf, views
+        dbuf, hin, dout, hout = [], [], [], []
+        if not wl.decode_steps:
+            dbuf = [packed((qs[0], kns[0], vns[0]), dev) for _ in range(2)]
+            for layer in range(L):
+                hb, hv3 = packed((qs[layer], kns[layer], vns[layer]), "cpu", pin=True)
+                for dst, src in zip(hv3, (hq[layer], hk[layer], hv[layer])):
+                    dst.copy_(src)
+                hin.append(hb)
+                dout.append(packed((outs[layer], masses[layer]), dev))
+                hout.append(torch.empty(dout[-1][0].numel(), dtype=torch.uint8).pin_memory())
         main = torch.cuda.current_stream(dev)
         s_up, s_dn = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
         ev_free = [None, None]
@@ -383,25 +406,26 @@ def main():
                     bi += hq[layer][t:t + 1].nbytes + 2 * hk[layer][t:t + 1].nbytes
                     attend(layer, qs[layer], kns[layer], vns[layer], outs[layer], masses[layer], t)
                 else:
-                    dq, dk, dv = dbuf[layer & 1]
+                    din, (dq, dk, dv) = dbuf[layer & 1]
                     with torch.cuda.stream(s_up):
                         if ev_free[layer & 1] is not None:
                             s_up.wait_event(ev_free[layer & 1])      # the attend that last read this buffer set
-                        dq.copy_(hq[layer], non_blocking=True)
-                        dk.copy_(hk[layer], non_blocking=True)
-                        dv.copy_(hv[layer], non_blocking=True)
+                        din.copy_(hin[layer], non_blocking=True)
                         ev_up = torch.cuda.Event()
                         ev_up.record(s_up)
                     main.wait_event(ev_up)
                     bi += hq[layer].nbytes + hk[layer].nbytes + hv[layer].nbytes
-                    attend(layer, dq, dk, dv, outs[layer], masses[layer], t)
+                    attend(layer, dq, dk, dv, dout[layer][1][0], dout[layer][1][1], t)
                 ev_done = torch.cuda.Event()
                 ev_done.record(main)
                 ev_free[layer & 1] = ev_done
                 with torch.cuda.stream(s_dn):
                     s_dn.wait_event(ev_done)
-                    ho[layer].copy_(outs[layer], non_blocking=True)
-                    hm[layer].copy_(masses[layer], non_blocking=True)
+                    if wl.decode_steps:
+                        ho[layer].copy_(outs[layer], non_blocking=True)
+                        hm[layer].copy_(masses[layer], non_blocking=True)
+                    else:
+                        hout[layer].copy_(dout[layer][0], non_blocking=True)
                 bo += ho[layer].nbytes + hm[layer].nbytes
             ev_last = torch.cuda.Event()
             ev_last.record(s_dn)
