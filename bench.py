@@ -379,13 +379,14 @@ def main():
         dbuf, hin, dout, hout = [], [], [], []
         if not wl.decode_steps:
             dbuf = [packed((qs[0], kns[0], vns[0]), dev) for _ in range(2)]
-            for layer in range(L):
+        for layer in range(L):
+            if not wl.decode_steps:
                 hb, hv3 = packed((qs[layer], kns[layer], vns[layer]), "cpu", pin=True)
                 for dst, src in zip(hv3, (hq[layer], hk[layer], hv[layer])):
                     dst.copy_(src)
                 hin.append(hb)
-                dout.append(packed((outs[layer], masses[layer]), dev))
-                hout.append(torch.empty(dout[-1][0].numel(), dtype=torch.uint8).pin_memory())
+            dout.append(packed((outs[layer], masses[layer]), dev))
+            hout.append(torch.empty(dout[-1][0].numel(), dtype=torch.uint8).pin_memory())
         main = torch.cuda.current_stream(dev)
         s_up, s_dn = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
         ev_free = [None, None]
@@ -404,7 +405,7 @@ def main():
                     kns[layer][t:t + 1].copy_(hk[layer][t:t + 1], non_blocking=True)
                     vns[layer][t:t + 1].copy_(hv[layer][t:t + 1], non_blocking=True)
                     bi += hq[layer][t:t + 1].nbytes + 2 * hk[layer][t:t + 1].nbytes
-                    attend(layer, qs[layer], kns[layer], vns[layer], outs[layer], masses[layer], t)
+                    attend(layer, qs[layer], kns[layer], vns[layer], dout[layer][1][0], dout[layer][1][1], t)
                 else:
                     din, (dq, dk, dv) = dbuf[layer & 1]
                     with torch.cuda.stream(s_up):
@@ -421,11 +422,7 @@ def main():
                 ev_free[layer & 1] = ev_done
                 with torch.cuda.stream(s_dn):
                     s_dn.wait_event(ev_done)
-                    if wl.decode_steps:
-                        ho[layer].copy_(outs[layer], non_blocking=True)
-                        hm[layer].copy_(masses[layer], non_blocking=True)
-                    else:
-                        hout[layer].copy_(dout[layer][0], non_blocking=True)
+                    hout[layer].copy_(dout[layer][0], non_blocking=True)
                 bo += ho[layer].nbytes + hm[layer].nbytes
             ev_last = torch.cuda.Event()
             ev_last.record(s_dn)
