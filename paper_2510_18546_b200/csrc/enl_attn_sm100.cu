@@ -1063,6 +1063,27 @@ cudaError_t prepare_attention(int head_dim)
     return cudaErrorInvalidValue;
 }
 
+bool attention_pairs_supported()
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = Cfg<128>::kSmemBytes;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, attn_kernel<128>, &cfg) != cudaSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    return n > 0;
+}
+
 cudaError_t launch_attention(const AttnParams &p, int head_dim, int n_items, cudaStream_t st)
 {
     if (n_items <= 0) return cudaSuccess;

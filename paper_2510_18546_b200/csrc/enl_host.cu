@@ -97,6 +97,7 @@ struct enl_cache {
     bool plan_has_mass = false;
     bool plan_decode = false;               // the plan is for the one-token decode kernel
     bool plan_pair = false;                 // two splits whose CTAs merge inside the attention kernel (cluster of two)
+    bool pairs_ok = false;                  // the device can co-schedule two of the attention kernel's CTAs as a cluster
     std::vector<int32_t> key_sel, key_cu, key_len;   // what the current plan was built from
     int32_t plan_entries = 0, plan_items = 0, plan_splits = 1, plan_batch = 0, plan_max_slots = 0;
     std::vector<int32_t> seen;              // duplicate detection stamps
@@ -256,6 +257,7 @@ extern "C" int enl_cache_create(const enl_cache_desc_t *desc, enl_cache_t **out)
         }
     }
     if (prepare_attention(d.head_dim) != cudaSuccess || prepare_decode(d.head_dim) != cudaSuccess) { cudaGetLastError(); destroy(c); return ENL_E_CUDA; }
+    c->pairs_ok = d.head_dim == 128 && attention_pairs_supported();   // else two splits go through the scratch buffer
     if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); destroy(c); return ENL_E_CUDA; }
     *out = c;
     return ENL_OK;
@@ -546,7 +548,7 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
         // Two splits of a head_dim-128 call are launched as clusters of two CTAs, which exchange their partial
         // results through distributed shared memory: no scratch round trip and no merge kernel.  Every CTA must
         // have at least one tile, and the items of a pair must be neighbours (they are: same tile count, stable sort).
-        c->plan_pair = !decode && n_splits == 2 && d.head_dim == 128 && min_tiles >= 2;
+        c->plan_pair = !decode && n_splits == 2 && d.head_dim == 128 && min_tiles >= 2 && (c->pairs_ok || !c->gpu);
         c->key_sel.assign(a->sel_ids, a->sel_ids + a->n_sel);
         c->key_cu = cu_key;
         c->key_len = sel_len;

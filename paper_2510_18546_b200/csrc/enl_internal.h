@@ -151,5 +151,7 @@ cudaError_t launch_page_copy(const uint8_t *src_k, const uint8_t *src_v, uint8_t
 size_t attention_smem_bytes(int head_dim);
 // Opts the attention kernel into its dynamic shared memory size on the current device.
 cudaError_t prepare_attention(int head_dim);
+// can the device run the head_dim-128 kernel as clusters of two CTAs (the in-kernel merge of two KV splits)?
+bool attention_pairs_supported();
 
 }  // namespace enl
