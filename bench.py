@@ -1,8 +1,8 @@
 #!/usr/bin/env python
 """Benchmark of the selective-KV attention hot path.
 
-A "step" is one planning step of the workload: for every layer one group store (the K/V of one
-group rewritten in place, Sec. 3.2), the gather plan (built at the first layer, reused by the
+A "step" is one planning step of the workload: one group store (the K/V of one group rewritten in
+place in every layer, Sec. 3.2), the gather plan (built at the first layer, reused by the
 others), and one `enl_attend` per layer (attention + fused per-group mass, plus the split merge
 when KV splits are used).  Layers run sequentially on one stream, as in the planner.
 
@@ -289,11 +289,18 @@ def main():
                            cu_q=cq if multi else None, cu_new=cn if multi else None, split_hint=args.split,
                            stream=stream)
 
+    store_ks, store_vs = [x[1] for x in store_src], [x[2] for x in store_src]
+    store_pages = (int(store_ks[0].shape[0]) + 15) // 16
+    store_launches = ((L + 63) // 64) * max(1, (store_pages + 63) // 64)
+
+    def store_step():
+        # the group's K/V of every layer rewritten in place by one launch (Sec. 3.2: a group's rows of all layers
+        # come out of one prefill)
+        enl.enl_group_store_all_layers(cache, store_src[0][0], store_ks, store_vs, stream=stream)
+
     def step(i, timed_events=None):
         t = (i % wl.decode_steps) if wl.decode_steps else None
-        for layer in range(L):
-            gid, k, v = store_src[layer]
-            enl.enl_group_store(cache, gid, layer, k, v, stream=stream)
+        store_step()
         # the attention launches of a step run back to back (chained by programmatic dependent launch, as in
         # use); one pair of events around the L of them gives the kernel's average duration in that context
         if timed_events is not None:
@@ -394,9 +401,7 @@ def main():
         def e2e_step(i):
             t = (i % wl.decode_steps) if wl.decode_steps else None
             bi = bo = 0
-            for layer in range(L):
-                gid, k, v = store_src[layer]
-                enl.enl_group_store(cache, gid, layer, k, v, stream=stream)
+            store_step()
             for layer in range(L):
                 if wl.decode_steps:
                     # the step's inputs: one query row and the new token's K/V row, appended to the
@@ -497,7 +502,7 @@ def main():
         _, _, _, cpu = oracle_sample(wl0)
 
     # attention (+ merge kernel when the splits go through the scratch buffer) + page scatter
-    launches_per_step = L * (1 + (1 if plan["merge_kind"] == 1 else 0)) + L
+    launches_per_step = L * (1 + (1 if plan["merge_kind"] == 1 else 0)) + store_launches
     enl.enl_cache_free(cache)
     if rank == 0:
         line = {"metric": metric_name(wl), "value": value, "unit": unit, "n_gpus": world, "steps": args.steps,

@@ -99,6 +99,22 @@ int enl_cache_create(const enl_cache_desc_t *desc, enl_cache_t **out);
 int enl_group_store(enl_cache_t *c, int32_t group_id, int32_t layer, int32_t n_tokens,
                     const void *k_dev, const void *v_dev, int32_t mode, void *cuda_stream);
 
+/*
+ * Sec. 3.2, the same operation for every layer at once: a group's description (or the new
+ * objects appended to it) passes through all layers of the planner in one prefill, so the K/V
+ * of all layers arrive together.  One kernel launch per 64 pages instead of one per layer.
+ *   k_dev, v_dev : HOST arrays of n_layers device pointers, k_dev[l] = layer l's
+ *                  [n_tokens][n_kv_heads][head_dim] bf16 rows; consumed before the call
+ *                  returns.  May be NULL only on a bookkeeping-only cache.
+ *   mode         : as in enl_group_store, applied to every layer.
+ * Before the call every layer must hold the same length of the group (or none): ENL_E_INVAL
+ * otherwise.  All or nothing: a call that returns an error has changed no layer.
+ * Errors: as enl_group_store.
+ */
+int enl_group_store_all_layers(enl_cache_t *c, int32_t group_id, int32_t n_tokens,
+                               const void *const *k_dev, const void *const *v_dev, int32_t mode,
+                               void *cuda_stream);
+
 typedef struct {
     int32_t layer;
     int32_t batch;                     /* independent episodes in this call, >= 1              */

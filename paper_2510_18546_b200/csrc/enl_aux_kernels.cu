@@ -3,6 +3,8 @@
 // partial outputs, sum of the partial per-slot masses).
 #include <cuda_bf16.h>
 
+#include <algorithm>
+
 #include "enl_internal.h"
 
 namespace enl {
@@ -29,6 +31,33 @@ __global__ void page_scatter_kernel(uint4 *__restrict__ kpool, uint4 *__restrict
                                   chunks_per_row + ch;
         kpool[dst] = k[id];
         vpool[dst] = v[id];
+    }
+}
+
+// grid (blocks, layers): the same scatter for several layers of one group at once
+__global__ void page_scatter_layers_kernel(uint4 *__restrict__ kpool, uint4 *__restrict__ vpool, long long layer_chunks,
+                                           const __grid_constant__ LayerSrc src, long long src_chunk_off,
+                                           const __grid_constant__ PageRun run, int first_pos, int n_tokens,
+                                           int Hkv, int chunks_per_row)
+{
+    const long long total = static_cast<long long>(n_tokens) * Hkv * chunks_per_row;
+    const uint4 *k = static_cast<const uint4 *>(src.k[blockIdx.y]) + src_chunk_off;
+    const uint4 *v = static_cast<const uint4 *>(src.v[blockIdx.y]) + src_chunk_off;
+    uint4 *kp = kpool + layer_chunks * blockIdx.y, *vp = vpool + layer_chunks * blockIdx.y;
+    pdl_trigger();
+    pdl_wait();                                             // an attention kernel may still be reading these pages
+    for (long long id = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; id < total;
+         id += static_cast<long long>(gridDim.x) * blockDim.x) {
+        const int ch = static_cast<int>(id % chunks_per_row);
+        const long long th = id / chunks_per_row;
+        const int head = static_cast<int>(th % Hkv);
+        const int tok = static_cast<int>(th / Hkv);
+        const int pos = first_pos + tok;
+        const int page = run.ids[pos / kPageTokens - run.first_page];
+        const long long dst = ((static_cast<long long>(page) * Hkv + head) * kPageTokens + pos % kPageTokens) *
+                                  chunks_per_row + ch;
+        kp[dst] = k[id];
+        vp[dst] = v[id];
     }
 }
 
@@ -206,6 +235,35 @@ cudaError_t launch_page_scatter(void *kpool_layer, void *vpool_layer, const void
     const cudaError_t e = cudaLaunchKernelEx(&cfg, page_scatter_kernel, static_cast<uint4 *>(kpool_layer),
                                              static_cast<uint4 *>(vpool_layer), static_cast<const uint4 *>(k),
                                              static_cast<const uint4 *>(v), run, first_pos, n_tokens, Hkv, cpr);
+    return e != cudaSuccess ? e : cudaGetLastError();
+}
+
+cudaError_t launch_page_scatter_layers(void *kpool, void *vpool, size_t layer_bytes, int layer0, int n_layers,
+                                       const LayerSrc &src, size_t src_off, const PageRun &run, int first_pos,
+                                       int n_tokens, int Hkv, int D, cudaStream_t st)
+{
+    if (n_tokens <= 0 || n_layers <= 0) return cudaSuccess;
+    if (n_layers > kScatterLayers) return cudaErrorInvalidValue;
+    const int cpr = D * 2 / 16;
+    const long long total = static_cast<long long>(n_tokens) * Hkv * cpr;
+    const int threads = 256;
+    long long blocks = (total + threads - 1) / threads;
+    const long long cap = std::max(1, 148 * 8 / n_layers);
+    if (blocks > cap) blocks = cap;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(blocks), static_cast<unsigned>(n_layers));
+    cfg.blockDim = dim3(threads);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    uint4 *kp = reinterpret_cast<uint4 *>(static_cast<uint8_t *>(kpool) + layer_bytes * layer0);
+    uint4 *vp = reinterpret_cast<uint4 *>(static_cast<uint8_t *>(vpool) + layer_bytes * layer0);
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, page_scatter_layers_kernel, kp, vp,
+                                             static_cast<long long>(layer_bytes / 16), src,
+                                             static_cast<long long>(src_off / 16), run, first_pos, n_tokens, Hkv, cpr);
     return e != cudaSuccess ? e : cudaGetLastError();
 }
 

@@ -357,6 +357,77 @@ extern "C" int enl_group_store(enl_cache_t *c, int32_t group_id, int32_t layer, 
     return ENL_OK;
 }
 
+extern "C" int enl_group_store_all_layers(enl_cache_t *c, int32_t group_id, int32_t n_tokens, const void *const *k_dev,
+                                          const void *const *v_dev, int32_t mode, void *cuda_stream)
+{
+    if (!c) return ENL_E_INVAL;
+    if (group_id < 0 || group_id >= c->d.max_groups) return ENL_E_NOGROUP;
+    if (n_tokens < 0) return ENL_E_INVAL;
+    if (mode != ENL_REPLACE && mode != ENL_APPEND) return ENL_E_INVAL;
+    const int L = c->d.n_layers;
+    if (c->gpu && n_tokens > 0) {
+        if (!k_dev || !v_dev) return ENL_E_INVAL;
+        for (int l = 0; l < L; ++l) {
+            if (!k_dev[l] || !v_dev[l]) return ENL_E_INVAL;
+            if ((reinterpret_cast<uintptr_t>(k_dev[l]) | reinterpret_cast<uintptr_t>(v_dev[l])) & 15) return ENL_E_INVAL;
+        }
+    }
+    Group &g = c->groups[group_id];
+    if (!g.resident) return ENL_E_EVICTED;
+    const int32_t old_len = g.len.empty() ? -1 : g.len[0];
+    for (int l = 1; l < L && !g.len.empty(); ++l)
+        if (g.len[l] != old_len) return ENL_E_INVAL;            // the layers must agree before they move together
+    const int64_t new_len64 = (mode == ENL_APPEND && old_len > 0) ? static_cast<int64_t>(old_len) + n_tokens : n_tokens;
+    if (new_len64 > 0x3fffffff) return ENL_E_INVAL;
+    const int32_t new_len = static_cast<int32_t>(new_len64);
+    const int32_t first_pos = new_len - n_tokens;
+    const int need_pages = ceil_div(new_len, kPageTokens);
+    const int have = static_cast<int>(g.pages.size());
+    if (need_pages > have && static_cast<size_t>(need_pages - have) > c->free_pages.size()) return ENL_E_NOMEM;
+
+    // commit the table change
+    for (int i = have; i < need_pages; ++i) {
+        g.pages.push_back(c->free_pages.back());
+        c->free_pages.pop_back();
+    }
+    g.len.assign(L, new_len);
+    g.host_current = false;                                  // the device copy is newer now
+    while (static_cast<int>(g.pages.size()) > need_pages) { // pages no layer needs any more
+        c->free_pages.push_back(g.pages.back());
+        g.pages.pop_back();
+    }
+    ++c->epoch;
+
+    if (!c->gpu || n_tokens == 0) return ENL_OK;
+    DeviceGuard dg(c->d.device);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const size_t row_bytes = static_cast<size_t>(c->d.n_kv_heads) * c->d.head_dim * 2;
+    for (int layer0 = 0; layer0 < L; layer0 += kScatterLayers) {
+        const int nl = std::min(kScatterLayers, L - layer0);
+        LayerSrc src;
+        for (int l = 0; l < kScatterLayers; ++l) {
+            src.k[l] = l < nl ? k_dev[layer0 + l] : nullptr;
+            src.v[l] = l < nl ? v_dev[layer0 + l] : nullptr;
+        }
+        int pos = first_pos;
+        while (pos < new_len) {
+            PageRun run;
+            run.first_page = pos / kPageTokens;
+            const int last_page = std::min((new_len - 1) / kPageTokens, run.first_page + kScatterPages - 1);
+            for (int i = run.first_page; i <= last_page; ++i) run.ids[i - run.first_page] = g.pages[i];
+            const int end = std::min(new_len, (last_page + 1) * kPageTokens);
+            const size_t src_off = static_cast<size_t>(pos - first_pos) * row_bytes;
+            if (launch_page_scatter_layers(c->kpool, c->vpool, c->layer_bytes, layer0, nl, src, src_off, run, pos,
+                                           end - pos, c->d.n_kv_heads, c->d.head_dim, st) != cudaSuccess) {
+                cudaGetLastError();
+                return ENL_E_CUDA;
+            }
+            pos = end;
+        }
+    }
+    return ENL_OK;
+}
+
 extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda_stream)
 {
     if (!c || !a) return ENL_E_INVAL;

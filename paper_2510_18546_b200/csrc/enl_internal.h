@@ -143,6 +143,16 @@ struct PageRun {
 cudaError_t launch_page_scatter(void *kpool_layer, void *vpool_layer, const void *k, const void *v,
                                 const PageRun &run, int first_pos, int n_tokens,
                                 int Hkv, int D, cudaStream_t st);
+// The same for up to kScatterLayers layers in one launch: layer l reads k[l] + src_off, v[l] + src_off (bytes)
+// and writes the pool of layer layer0 + l.
+constexpr int kScatterLayers = 64;
+struct LayerSrc {
+    const void *k[kScatterLayers];
+    const void *v[kScatterLayers];
+};
+cudaError_t launch_page_scatter_layers(void *kpool, void *vpool, size_t layer_bytes, int layer0, int n_layers,
+                                       const LayerSrc &src, size_t src_off, const PageRun &run, int first_pos,
+                                       int n_tokens, int Hkv, int D, cudaStream_t st);
 // Copies whole pages (all kv heads) between two pools of the page format, every layer, K and V: pairs[i] =
 // {source page, destination page}; the pools may be device memory or pinned host memory.
 cudaError_t launch_page_copy(const uint8_t *src_k, const uint8_t *src_v, uint8_t *dst_k, uint8_t *dst_v,

@@ -23,7 +23,7 @@ ENL_OK, ENL_E_INVAL, ENL_E_NOGROUP, ENL_E_NOMEM, ENL_E_CUDA, ENL_E_TIMEOUT, ENL_
 ENL_STATIC_MAX_SEGMENTS, ENL_STATIC_MAX_KEYS, ENL_STATIC_SCRATCH_BYTES = 255, 65536, 4 << 20
 
 EXPORTS = ("enl_cache_create", "enl_group_store", "enl_attend", "enl_cache_free", "enl_strerror",
-           "enl_group_len", "enl_cache_status", "enl_plan_inspect", "enl_attend_static", "enl_cluster_assign",
+           "enl_group_store_all_layers", "enl_group_len", "enl_cache_status", "enl_plan_inspect", "enl_attend_static", "enl_cluster_assign",
            "enl_select_knapsack", "enl_tier_enable", "enl_group_evict", "enl_step_prepare", "enl_group_resident")
 
 
@@ -82,6 +82,9 @@ def lib() -> ctypes.CDLL:
         L.enl_group_store.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
                                       ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p]
         L.enl_group_store.restype = ctypes.c_int
+        L.enl_group_store_all_layers.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p,
+                                                 ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p]
+        L.enl_group_store_all_layers.restype = ctypes.c_int
         L.enl_attend.argtypes = [ctypes.c_void_p, ctypes.POINTER(AttendArgs), ctypes.c_void_p]
         L.enl_attend.restype = ctypes.c_int
         L.enl_cache_free.argtypes = [ctypes.c_void_p]
@@ -152,6 +155,23 @@ def enl_group_store(cache: int, group_id: int, layer: int, k, v, mode: int = ENL
     rc = lib().enl_group_store(cache, group_id, layer, n, _ptr(k), _ptr(v), mode, stream or None)
     if rc != ENL_OK:
         raise EnlError(rc, "enl_group_store")
+
+
+def enl_group_store_all_layers(cache: int, group_id: int, ks, vs, mode: int = ENL_REPLACE, stream: int = 0,
+                               n_tokens: Optional[int] = None) -> None:
+    """``ks``/``vs``: one ``[n, Hkv, D]`` bf16 CUDA tensor per layer (or None with ``n_tokens`` on a bookkeeping
+    cache).  Every layer of the group is written by one launch."""
+    if ks is None:
+        n, kp, vp = int(n_tokens), None, None
+    else:
+        n = int(ks[0].shape[0])
+        if any(int(t.shape[0]) != n for t in list(ks) + list(vs)):
+            raise ValueError("every layer must bring the same number of rows")
+        kp = (ctypes.c_void_p * len(ks))(*[_ptr(t) for t in ks])
+        vp = (ctypes.c_void_p * len(vs))(*[_ptr(t) for t in vs])
+    rc = lib().enl_group_store_all_layers(cache, group_id, n, kp, vp, mode, stream or None)
+    if rc != ENL_OK:
+        raise EnlError(rc, "enl_group_store_all_layers")
 
 
 def enl_attend(cache: int, layer: int, sel_ids: Sequence[int], q, k_new, v_new, out, group_mass=None,

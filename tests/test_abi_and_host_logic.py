@@ -240,3 +240,30 @@ def test_merge_kind_follows_splits_shape_and_tile_count():
         assert enl.enl_plan_inspect(c)["merge_kind"] == 1
     finally:
         enl.enl_cache_free(c)
+
+
+def test_store_all_layers_moves_every_layer_together_or_not_at_all():
+    c = host_cache()                                    # two layers
+    try:
+        enl.enl_group_store_all_layers(c, 2, None, None, n_tokens=40)
+        assert [enl.enl_group_len(c, 2, l) for l in range(2)] == [40, 40]
+        enl.enl_group_store_all_layers(c, 2, None, None, mode=enl.ENL_APPEND, n_tokens=9)      # Sec. 3.2: append
+        assert [enl.enl_group_len(c, 2, l) for l in range(2)] == [49, 49]
+        got = plan(c, 1, [2], 3, 3)
+        assert list(got) == [0, 49]
+        enl.enl_group_store(c, 2, 0, None, None, mode=enl.ENL_APPEND, n_tokens=1)              # layers now disagree
+        with pytest.raises(enl.EnlError) as e:
+            enl.enl_group_store_all_layers(c, 2, None, None, mode=enl.ENL_APPEND, n_tokens=5)
+        assert e.value.code == enl.ENL_E_INVAL
+        assert [enl.enl_group_len(c, 2, l) for l in range(2)] == [50, 49]                      # nothing moved
+        enl.enl_group_store(c, 2, 1, None, None, mode=enl.ENL_APPEND, n_tokens=1)
+        enl.enl_group_store_all_layers(c, 2, None, None, mode=enl.ENL_REPLACE, n_tokens=0)     # an empty group
+        assert [enl.enl_group_len(c, 2, l) for l in range(2)] == [0, 0]
+        with pytest.raises(enl.EnlError) as e:
+            enl.enl_group_store_all_layers(c, 99, None, None, n_tokens=1)
+        assert e.value.code == enl.ENL_E_NOGROUP
+        with pytest.raises(enl.EnlError) as e:
+            enl.enl_group_store_all_layers(c, 3, None, None, n_tokens=100000)                  # more than the pool holds
+        assert e.value.code == enl.ENL_E_NOMEM and enl.enl_group_len(c, 3, 0) == -1
+    finally:
+        enl.enl_cache_free(c)

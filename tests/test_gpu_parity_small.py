@@ -121,6 +121,43 @@ def test_split_merge_kinds():
     run_case(wl, split_hint=0, expect_merge=3)
 
 
+def test_store_all_layers_equals_layer_by_layer_stores():
+    """Every layer of a group written by one launch (replace, then append) reads back exactly as the same rows
+    written layer by layer."""
+    wl = synth.make_small(21, 3, 8, 2, 128, [[70, 33, 5]], [[1, 0, 2]], [40], [40], name="all_layers")
+    dev = torch.device("cuda:0")
+    caches = [enl.enl_cache_create(3, 8, 2, 128, wl.n_groups, wl.pool_tokens + 64, device=0, max_batch=1,
+                                   max_q_tokens=40) for _ in range(2)]
+    try:
+        kv = [wl.pool_kv(layer, 0, dev) for layer in range(3)]
+        offs = wl.pool_offsets(0)
+        for g in range(3):
+            a, b = int(offs[g]), int(offs[g + 1])
+            cut = a + (b - a) // 2                      # first half stored, second half appended
+            for layer in range(3):
+                enl.enl_group_store(caches[0], g, layer, kv[layer][0][a:cut], kv[layer][1][a:cut])
+                enl.enl_group_store(caches[0], g, layer, kv[layer][0][cut:b], kv[layer][1][cut:b], mode=enl.ENL_APPEND)
+            enl.enl_group_store_all_layers(caches[1], g, [kv[l][0][a:cut] for l in range(3)],
+                                           [kv[l][1][a:cut] for l in range(3)])
+            enl.enl_group_store_all_layers(caches[1], g, [kv[l][0][cut:b] for l in range(3)],
+                                           [kv[l][1][cut:b] for l in range(3)], mode=enl.ENL_APPEND)
+        sel = wl.sel_ids()
+        for layer in range(3):
+            q, kn, vn = wl.new_qkv(layer, dev)
+            res = []
+            for c in caches:
+                out = torch.empty_like(q)
+                mass = torch.full((40, 8, len(sel) + 1), float("nan"), dtype=torch.float32, device=dev)
+                enl.enl_attend(c, layer, sel, q, kn, vn, out, mass)
+                res.append((out, mass))
+            torch.cuda.synchronize()
+            assert torch.equal(res[0][0], res[1][0]) and torch.equal(res[0][1], res[1][1])
+            assert [enl.enl_group_len(caches[1], g, layer) for g in range(3)] == [70, 33, 5]
+    finally:
+        for c in caches:
+            enl.enl_cache_free(c)
+
+
 def test_zero_length_group_has_zero_mass():
     wl = synth.make_small(8, 1, 8, 2, 64, [[12, 0, 20]], [[0, 1, 2]], [33], [33], name="zero_len")
     with Session(wl, [0]) as s:
