@@ -158,6 +158,36 @@ def test_store_all_layers_equals_layer_by_layer_stores():
             enl.enl_cache_free(c)
 
 
+def test_store_all_layers_beyond_one_launch():
+    """More than 64 pages and more than 64 layers: the store is cut into several launches."""
+    n_layers, n_tok = 66, 1100
+    dev = torch.device("cuda:0")
+    gen = torch.Generator(device=dev).manual_seed(5)
+    ks = [torch.randn(n_tok, 1, 64, generator=gen, device=dev).to(torch.bfloat16) for _ in range(n_layers)]
+    vs = [torch.randn(n_tok, 1, 64, generator=gen, device=dev).to(torch.bfloat16) for _ in range(n_layers)]
+    q = torch.randn(7, 2, 64, generator=gen, device=dev).to(torch.bfloat16)
+    kn = torch.randn(7, 1, 64, generator=gen, device=dev).to(torch.bfloat16)
+    vn = torch.randn(7, 1, 64, generator=gen, device=dev).to(torch.bfloat16)
+    caches = [enl.enl_cache_create(n_layers, 2, 1, 64, 2, 1200, device=0, max_batch=1, max_q_tokens=7) for _ in range(2)]
+    try:
+        for layer in range(n_layers):
+            enl.enl_group_store(caches[0], 1, layer, ks[layer], vs[layer])
+        enl.enl_group_store_all_layers(caches[1], 1, ks, vs)
+        for layer in (0, 63, 64, 65):
+            res = []
+            for c in caches:
+                out = torch.empty_like(q)
+                mass = torch.full((7, 2, 2), float("nan"), dtype=torch.float32, device=dev)
+                enl.enl_attend(c, layer, [1], q, kn, vn, out, mass)
+                res.append((out, mass))
+            torch.cuda.synchronize()
+            assert torch.equal(res[0][0], res[1][0]) and torch.equal(res[0][1], res[1][1])
+            assert torch.isfinite(res[1][1]).all()
+    finally:
+        for c in caches:
+            enl.enl_cache_free(c)
+
+
 def test_zero_length_group_has_zero_mass():
     wl = synth.make_small(8, 1, 8, 2, 64, [[12, 0, 20]], [[0, 1, 2]], [33], [33], name="zero_len")
     with Session(wl, [0]) as s:
