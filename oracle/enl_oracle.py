@@ -165,28 +165,6 @@ class OracleCache:
                                  q, k_new, v_new, rows=rows, want_mass=want_mass)
         return out, mass, sel_off([k.shape[0] for k in ks])
 
-    def attend_batch(
-        self,
-        layer: int,
-        sel_ids: Sequence[int],
-        cu_sel: Sequence[int],
-        cu_q: Sequence[int],
-        cu_new: Sequence[int],
-        q,
-        k_new,
-        v_new,
-        rows_per_episode: Optional[List[Optional[Sequence[int]]]] = None,
-    ):
-        """Varlen batch of independent episodes: a plain loop over ``attend``."""
-        res = []
-        for b in range(len(cu_q) - 1):
-            ids = list(sel_ids[cu_sel[b]:cu_sel[b + 1]])
-            rows = rows_per_episode[b] if rows_per_episode is not None else None
-            res.append(self.attend(layer, ids, q[cu_q[b]:cu_q[b + 1]],
-                                   k_new[cu_new[b]:cu_new[b + 1]], v_new[cu_new[b]:cu_new[b + 1]],
-                                   rows=rows))
-        return res
-
 
 # ---- clustering reduce and retrieval knapsack (the consumers / producers around the attention) ----
 

@@ -114,9 +114,10 @@ __global__ void combine_kernel(const CombineParams p)
         for (int x = 0; x < V; ++x) acc[x] = 0.f;
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
+            // a split that saw no key has weight 0 and never wrote its partial output: what sits there is stale
             const float w = (lv[k] != ninf) ? ex2f(lv[k] - lse) : 0.f;
 #pragma unroll
-            for (int x = 0; x < V; ++x) acc[x] += w * ov[k][x];
+            for (int x = 0; x < V; ++x) acc[x] = (w != 0.f) ? fmaf(w, ov[k][x], acc[x]) : acc[x];
         }
         __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(p.out) + rh * D + lane * V;
 #pragma unroll

@@ -549,7 +549,7 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
         }
         if (!decode) {
             n_splits = 1;
-            if (a->split_hint >= 1) n_splits = a->split_hint;
+            if (a->split_hint >= 1) n_splits = std::min(a->split_hint, std::max(1, min_tiles));   // no CTA without a tile
             else if (base_items < 120) n_splits = std::max(1, std::min(static_cast<int>(148 / base_items), min_tiles / 2));
             n_splits = std::min<int64_t>(n_splits, std::max<int64_t>(1, c->cap_items / base_items));
             n_splits = std::min(n_splits, kMaxSplits);

@@ -228,7 +228,8 @@ def test_merge_kind_follows_splits_shape_and_tile_count():
         plan(c, 0, [0, 1], 64, 64, split_hint=3)
         assert enl.enl_plan_inspect(c)["merge_kind"] == 1
         plan(c, 0, [], 64, 64, split_hint=2)                    # one tile in all: a second CTA would have nothing to do
-        assert enl.enl_plan_inspect(c)["merge_kind"] == 1
+        p = enl.enl_plan_inspect(c)
+        assert p["merge_kind"] == 0 and p["n_splits"] == 1      # the hint is clamped: no CTA without a tile
         plan(c, 0, [0, 1], 1, 9)
         assert enl.enl_plan_inspect(c)["merge_kind"] == 3
     finally:

@@ -115,7 +115,7 @@ def test_split_merge_kinds():
     run_case(wl, split_hint=3, expect_merge=1)
     c = SMALL["empty_select"]                       # one tile only: nothing for a second CTA of a pair to do
     wl = synth.make_small(7, 1, c["Hq"], c["Hkv"], c["D"], c["pool"], c["sel"], c["n_q"], c["n_new"], name="kinds1")
-    run_case(wl, split_hint=2, expect_merge=1)
+    run_case(wl, split_hint=2, expect_merge=0)
     c = SMALL["decode_grown"]
     wl = synth.make_small(7, 1, c["Hq"], c["Hkv"], c["D"], c["pool"], c["sel"], c["n_q"], c["n_new"], name="kinds2")
     run_case(wl, split_hint=0, expect_merge=3)

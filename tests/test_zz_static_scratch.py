@@ -8,8 +8,9 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import enl_oracle as orc
 from paper_2510_18546_b200 import enl, synth
-from tests.helpers import MASS_MAX_ABS, OUT_MAX_ABS, OUT_MEAN_ABS, Session
+from tests.helpers import MASS_MAX_ABS, OUT_MAX_ABS, OUT_MEAN_ABS, Session, check_close
 
 pytestmark = pytest.mark.gpu
 
@@ -28,6 +29,11 @@ def both_paths(s, wl, sel, t, want_mass=True):
     enl.enl_attend_static([int(wl.pool_lens[0][g]) for g in sel], t + 1, q[t], kc, vc, out_s, mass_s,
                           stream=torch.cuda.current_stream(s.device).cuda_stream)
     torch.cuda.synchronize()
+    # the float64 oracle on the same contiguous keys, the segments as its slots: a mistake shared by the two
+    # one-token CUDA paths would pass a comparison of one with the other
+    ro, rm = orc.attend_slots(wl.n_q_heads, wl.n_kv_heads, wl.head_dim, [x.cpu() for x in ks[:-1]],
+                              [x.cpu() for x in vs[:-1]], q[t:t + 1].cpu(), kn[:t + 1].cpu(), vn[:t + 1].cpu())
+    check_close(out_s[None], ro, mass_s[None] if want_mass else None, rm if want_mass else None, "static vs oracle")
     return out_a[0], (mass_a[0, :, :len(sel) + 1] if want_mass else None), out_s, mass_s
 
 
