@@ -57,8 +57,7 @@ enum {                                            /* return codes               
     ENL_E_CUDA     = -4,   /* a CUDA call failed, or a GPU operation on a bookkeeping cache    */
     ENL_E_TIMEOUT  = -5,   /* a bounded wait inside a kernel expired (see enl_cache_status)    */
     ENL_E_LIMIT    = -6,   /* a size beyond the fixed maxima of enl_attend_static              */
-    ENL_E_RANGE    = -7,   /* scores of one 128-key tile exceeded the maximum of all earlier    */
-                           /*   keys by more than 2^100 (see enl_cache_status)                  */
+                           /* -7 is not used                                                    */
     ENL_E_EVICTED  = -8    /* the group's K/V is in the slow tier only (see enl_step_prepare)   */
 };
 
@@ -168,10 +167,7 @@ const char *enl_strerror(int code);
 int32_t enl_group_len(const enl_cache_t *c, int32_t group_id, int32_t layer);
 
 /* Synchronises the device and returns ENL_OK, or ENL_E_TIMEOUT if any kernel of this cache
- * gave up on a bounded wait since the last call, or ENL_E_RANGE if a prefill call met scaled
- * scores (q.k/sqrt(D), in log2 units) that exceed the largest score of all earlier 128-key tiles
- * of the same row by more than 100: its probabilities were clamped and the result is not exact
- * (the flag is then cleared). */
+ * gave up on a bounded wait since the last call (the flag is then cleared). */
 int enl_cache_status(enl_cache_t *c);
 
 /*

@@ -10,19 +10,21 @@
 //   p   = exp2(S * c - m)    one thread per row, fp32; padding and causally hidden columns -> 0
 //   O_i += P_i V             tcgen05.mma, P (bf16) read from TMEM, V from shared memory
 // The row sum of p is split by the slot (selected group, or the new tokens) each 16-key page belongs
-// to; when a slot ends its log2-sum-exp is parked in the mass buffer, and after the last tile the row
-// turns those into probabilities.  With KV splits every split writes partial results that a second
-// kernel merges.
+// to; when a slot ends its log2-sum-exp is parked in the mass buffer, and after the last tile the
+// warp turns those into probabilities.  With KV splits every split writes partial results that a
+// second kernel merges, or (two splits, head_dim 128) the two CTAs of a cluster merge in place.
 //
-// Roles: 16 softmax warps -- Q tile i = warps 8i..8i+7, and within a tile warps 0-3 take key columns 0..63
-// of every S tile ("half A"), warps 4-7 columns 64..127 ("half B"), so that every row is shared by two
-// threads of two warps with the same TMEM lane quadrant; they exchange the row maximum (and half B's page
-// sums, which half A credits to the slots) through shared memory behind a two-warp mbarrier.  Four
-// softmax warps per scheduler overlap each other's exp2, max, pack and TMEM traffic.  Warp 16 is the TMA
-// producer, warp 17 the MMA issuer (and TMEM owner), warps 18-19 idle: they complete the fifth warpgroup
-// so that setmaxnreg can move registers to the softmax warpgroups.
-// TMEM columns: S0 [0,128) S1 [128,256) O0 [256,384) O1 [384,512); P_i (bf16) overwrites columns [0,32) and
-// [64,96) of S_i, each softmax half inside its own columns.
+// Roles (12 warps): warps 0-3 are the softmax warpgroup of Q tile 0, warps 4-7 that of Q tile 1: one
+// thread per query row holds the row's 128 scores of a tile in registers, so the row maximum, the
+// exponentials and the eight page sums need no exchange between threads.  Warp 8 is the TMA producer,
+// warp 9 the MMA issuer (and TMEM owner), warps 10-11 idle: they complete the third warpgroup so that
+// setmaxnreg can move its registers to the softmax warpgroups.
+// The two Q tiles alternate on the tensor pipe: while one tile's softmax runs, the pipe does the other
+// tile's P V and the next Q K^T.  P is handed over in two halves of 64 keys so that P V starts while
+// the second half's exponentials are still being taken; everything that is not needed for P (row and
+// page sums, slot book-keeping) is done after the hand-over, under the MMAs.
+// TMEM columns: S0 [0,128) S1 [128,256) O0 [256,384) O1 [384,512); P_i (bf16 pairs) overwrites columns
+// [0,64) of S_i once the row's scores are in registers.
 #include <cuda_bf16.h>
 
 #include "enl_internal.h"
@@ -31,16 +33,16 @@
 namespace enl {
 namespace {
 
-constexpr int kThreads      = 640;
-constexpr int kSoftmaxWarps = 16;
-constexpr int kRegsSoftmax  = 104;            // the launch gives 640 x 96 registers; what warpgroup 4 releases (4 x 8 per thread) is what the four softmax warpgroups gain
-constexpr int kRegsOther    = 64;
-constexpr int kProducerWarp = 16;
-constexpr int kMmaWarp      = 17;
+constexpr int kThreads      = 384;
+constexpr int kSoftmaxWarps = 8;
+constexpr int kRegsSoftmax  = 216;            // 256 x 216 + 128 x 72 = 384 x 168, what the launch allocates
+constexpr int kRegsOther    = 72;
+constexpr int kProducerWarp = 8;
+constexpr int kMmaWarp      = 9;
 constexpr uint32_t kTmemCols = 512;
-constexpr float kRescaleThreshold = 8.0f;     // log2 units: p stays below 2^8 between max updates
-constexpr float kMaxJump = 100.0f;            // log2 units: most a tile's scores may exceed the maximum of all earlier tiles
+constexpr float kRescaleThreshold = 8.0f;     // log2 units: p stays below 2^8 between updates of the reference
 constexpr unsigned long long kWaitLimitNs = 1000ull * 1000ull * 1000ull;
+constexpr uint32_t kFull = 0xffffffffu;
 
 template <int D>
 struct Cfg {
@@ -49,13 +51,8 @@ struct Cfg {
     static constexpr int kTileBytes = kHalves * kHalfBytes;
     static constexpr int kStages    = (D == 128) ? 4 : 8;
     static constexpr int kBarOff    = (kQTiles + kStages) * kTileBytes;
-    // exchange area of the softmax thread pairs: row maxima [parity][tile][half][128], page sums
-    // [tile mod 3][tile][8 pages][128], 1 / row sum [tile][128]
-    static constexpr int kXmaxOff   = kBarOff + 512;
-    static constexpr int kXsumOff   = kXmaxOff + 2 * kQTiles * 2 * 128 * 4;
-    static constexpr int kXinvOff   = kXsumOff + 3 * kQTiles * kPagesPerTile * 128 * 4;
     // pair merge: what the other CTA of the cluster knows about this CTA's rows, [tile][128] x (m, l, shared-slot log-sum, -)
-    static constexpr int kXpeerOff  = kXinvOff + kQTiles * 128 * 4;
+    static constexpr int kXpeerOff  = kBarOff + 512;
     static constexpr int kSmemBytes = kXpeerOff + kQTiles * 128 * 16 + 1024;   // + alignment slack
 };
 
@@ -176,7 +173,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             }
         }
     }
-    return __all_sync(0xffffffffu, ok);
+    return __all_sync(kFull, ok);
 }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tm, int x, int y, uint32_t bar)
 {
@@ -254,6 +251,11 @@ __device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b)
     asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
     return d;
 }
+__device__ __forceinline__ uint32_t bf16x2(float lo, float hi)
+{
+    const __nv_bfloat162 b = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t *>(&b);
+}
 
 // Shared-memory matrix descriptor, 128-byte swizzle, rows of 128 B, 8-row groups 1024 B apart.
 // K-major operand (the contraction dimension is contiguous): LBO unused.
@@ -280,16 +282,6 @@ __host__ __device__ constexpr uint32_t make_idesc(int n, bool b_mn_major)
 
 constexpr float kNegInf = -__builtin_huge_valf();
 
-// Optional phase timestamps of CTA 0 (development builds only; never compiled into the library).
-#ifdef ENL_TRACE
-__device__ long long g_trace[5][96][8];
-#define ENL_TR(role, tile, slot) do { if (blockIdx.x == 0 && lane == 0 && (tile) < 96) g_trace[role][tile][slot] = clock64(); } while (0)
-#define ENL_PIN(x) asm volatile("" : "+f"(x) :: "memory")
-#else
-#define ENL_TR(role, tile, slot) do { } while (0)
-#define ENL_PIN(x) do { } while (0)
-#endif
-
 // ---- the kernel ----------------------------------------------------------------------------
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant__ AttnParams p)
@@ -310,16 +302,15 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
     auto bar_kv_full  = [&](int s) { return bar0 + 8u * (1 + s); };
     auto bar_kv_empty = [&](int s) { return bar0 + 8u * (1 + C::kStages + s); };
     auto bar_s_full   = [&](int i) { return bar0 + 8u * (1 + 2 * C::kStages + i); };
-    auto bar_p_full   = [&](int i) { return bar0 + 8u * (3 + 2 * C::kStages + i); };
-    auto bar_o_done   = [&](int i) { return bar0 + 8u * (5 + 2 * C::kStages + i); };
-    auto bar_pair     = [&](int k) { return bar0 + 8u * (7 + 2 * C::kStages + k); };   // k = tile * 4 + lane quadrant
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + C::kBarOff + 8 * (15 + 2 * C::kStages));
+    auto bar_p_half   = [&](int i, int hf) { return bar0 + 8u * (3 + 2 * C::kStages + 2 * i + hf); };   // keys 0..63 / 64..127 of P_i
+    auto bar_o_done   = [&](int i) { return bar0 + 8u * (7 + 2 * C::kStages + i); };
     // pair merge (cluster of two): the peer's row sums have arrived / the peer's partial output has arrived /
-    // the peer's K/V ring is idle and may be written
-    const uint32_t bar_peer_ml = bar0 + 8u * (16 + 2 * C::kStages);
-    const uint32_t bar_peer_o = bar0 + 8u * (17 + 2 * C::kStages);
-    const uint32_t bar_peer_free = bar0 + 8u * (18 + 2 * C::kStages);
-    const uint32_t bar_peer_ack = bar0 + 8u * (19 + 2 * C::kStages);   // the peer has received what this CTA staged for it
+    // the peer's K/V ring is idle and may be written / the peer has received what this CTA staged for it
+    const uint32_t bar_peer_ml = bar0 + 8u * (9 + 2 * C::kStages);
+    const uint32_t bar_peer_o = bar0 + 8u * (10 + 2 * C::kStages);
+    const uint32_t bar_peer_free = bar0 + 8u * (11 + 2 * C::kStages);
+    const uint32_t bar_peer_ack = bar0 + 8u * (12 + 2 * C::kStages);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + C::kBarOff + 8 * (13 + 2 * C::kStages));
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     // work item
@@ -343,17 +334,17 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
         for (int s = 0; s < C::kStages; ++s) { mbar_init(bar_kv_full(s), 1); mbar_init(bar_kv_empty(s), 1); }
         for (int i = 0; i < kQTiles; ++i) {
             mbar_init(bar_s_full(i), 1);
-            mbar_init(bar_p_full(i), 8);          // one arrival per softmax warp of the tile
+            mbar_init(bar_p_half(i, 0), 4);       // one arrival per softmax warp of the tile
+            mbar_init(bar_p_half(i, 1), 4);
             mbar_init(bar_o_done(i), 1);
         }
-        for (int k = 0; k < 4 * kQTiles; ++k) mbar_init(bar_pair(k), 2);
         mbar_init(bar_peer_ml, 1);                                   // this thread's arrival below + 16 bytes per row from the peer
         mbar_init(bar_peer_o, 1);                                    // this thread's arrival below + 64 KB from the peer
         mbar_init(bar_peer_free, 1);
         mbar_init(bar_peer_ack, 1);
         if (p.pair_merge) {
             mbar_expect_tx(bar_peer_ml, static_cast<uint32_t>(n_qt * 128 * 16));
-            mbar_expect_tx(bar_peer_o, 8u * 8192u);
+            mbar_expect_tx(bar_peer_o, 4u * 16384u);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -450,11 +441,13 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                 }
                 __syncwarp();
             };
-            auto issue_pv = [&](int i, int st, bool first_tile) {
+            // O_i (+)= P_i[:, 64 hf .. 64 hf + 63] V[64 hf .. 64 hf + 63, :]; P of keys 2c, 2c+1 sits in column c of S_i
+            auto issue_pv = [&](int i, int st, int hf, bool first_tile) {
                 if (lane == 0) {
 #pragma unroll
-                    for (int kk = 0; kk < kTileKeys / 16; ++kk) {
-                        mma_ts(tmem_o(i), tmem_s(i) + static_cast<uint32_t>((kk >> 2) * 64 + (kk & 3) * 8),   // P of keys 64.. sits in columns 64..
+                    for (int k4 = 0; k4 < 4; ++k4) {
+                        const int kk = hf * 4 + k4;
+                        mma_ts(tmem_o(i), tmem_s(i) + static_cast<uint32_t>(kk * 8),
                                smem_desc(stage_addr(st) + static_cast<uint32_t>(kk * 16 * 128), C::kHalfBytes),
                                idesc_pv, (first_tile && kk == 0) ? 0u : 1u);
                     }
@@ -484,19 +477,19 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                 if (ok && more) ok = wait_full(fk);
                 if (!ok) break;
                 for (int i = 0; i < n_qt; ++i) {
-                    ENL_TR(4, jj, 4 * i);
-                    ok = mbar_wait(bar_p_full(i), static_cast<uint32_t>(jj & 1), abort_flag, p.status);
+                    for (int hf = 0; hf < 2 && ok; ++hf) {
+                        ok = mbar_wait(bar_p_half(i, hf), static_cast<uint32_t>(jj & 1), abort_flag, p.status);
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_pv(i, fv % C::kStages, hf, jj == 0);
+                    }
                     if (!ok) break;
-                    tc_fence_after();
-                    ENL_TR(4, jj, 4 * i + 1);
-                    issue_pv(i, fv % C::kStages, jj == 0);
                     if (i == n_qt - 1) commit_to(bar_kv_empty(fv % C::kStages));
                     if (!more) commit_to(bar_o_done(i));
                     if (more) {
                         issue_qk(i, fk % C::kStages);
                         if (i == n_qt - 1) commit_to(bar_kv_empty(fk % C::kStages));
                     }
-                    ENL_TR(4, jj, 4 * i + 2);
                 }
             }
             // pair merge: once every MMA of this CTA has completed, its K/V ring is idle and the peer may write
@@ -509,19 +502,16 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
       }
     } else {
       asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
-      if ((warp >> 3) < n_qt) {
-        // ================= softmax / epilogue: two threads per row, 64 key columns each =================
-        constexpr int kHalfCols = kTileKeys / 2;                   // 64 key columns = 4 pages per thread
-        constexpr int kHalfPages = kPagesPerTile / 2;
-        const int i = warp >> 3;                                   // Q tile
-        const int hb = (warp >> 2) & 1;                            // 0: columns 0..63 (owner of the row's sums), 1: 64..127
+      if ((warp >> 2) < n_qt) {
+        // ================= softmax / epilogue: one thread per query row =================
+        const int i = warp >> 2;                                   // Q tile
         const int q4 = warp & 3;                                   // TMEM lane quadrant
-        const bool owner = hb == 0;
         const int r = q4 * 32 + lane;
         const int t = it.t0 + i * tile_tokens + r / rep;           // episode-relative query token
         const int h = it.kvh * rep + r % rep;
         const bool row_valid = t < ep.n_q;
         const int c = min(ep.n_new - ep.n_q + t, ep.n_new - 1);    // last visible new key
+        const int c_lo = ep.n_new - ep.n_q + it.t0 + i * tile_tokens;   // the same for the tile's first row: every row sees at least this far
         const int G = ep.n_slots;
         const uint32_t lane_sel = static_cast<uint32_t>(q4 * 32) << 16;
         const uint32_t t_s = tmem_base + lane_sel + static_cast<uint32_t>(i * 128);
@@ -529,28 +519,12 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
         const bool split_mode = p.n_splits > 1 && !pair;
         const long long grow = static_cast<long long>(ep.q_off) + t;   // global query row
         const long long rh = (split_mode ? (static_cast<long long>(it.split) * p.n_q_total + grow) : grow) * p.Hq + h;
-        float *slot_out = nullptr;
-        if (row_valid && owner) {
+        float *slot_out = nullptr;                                 // where this row's slots are parked
+        if (row_valid) {
             if (split_mode) { if (p.part_slot) slot_out = p.part_slot + rh * p.mass_stride; }
             else if (p.mass) slot_out = p.mass + rh * p.mass_stride;
         }
         const float scale = p.scale_log2;
-        const float inv_scale = 1.f / scale;
-        float *xmax_own = reinterpret_cast<float *>(smem + C::kXmaxOff) + (i * 2 + hb) * 128 + r;          // + parity * kQTiles*2*128
-        float *xmax_other = reinterpret_cast<float *>(smem + C::kXmaxOff) + (i * 2 + (hb ^ 1)) * 128 + r;
-        constexpr int kXmaxPar = kQTiles * 2 * 128;
-        float *xsum = reinterpret_cast<float *>(smem + C::kXsumOff) + i * (kPagesPerTile * 128) + r;   // + (tile mod 3) * kQTiles*8*128 + page*128
-        float *xinv = reinterpret_cast<float *>(smem + C::kXinvOff) + i * 128 + r;
-        const uint32_t pbar = bar_pair(i * 4 + q4);
-        uint32_t n_sync = 0;
-        // the two warps that share 32 rows meet here; bounded like every other wait
-        auto pair_sync = [&]() -> bool {
-            __syncwarp();
-            if (lane == 0) mbar_arrive(pbar);
-            const bool done = mbar_wait(pbar, n_sync & 1u, abort_flag, p.status);
-            ++n_sync;
-            return done;
-        };
 
         // Pair merge: the slot in which the two splits meet is walked by both.  Split 0 writes it (adding what
         // split 1 sends); split 1 keeps its part in `bnd` instead of storing it.
@@ -562,472 +536,383 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
             const int first1 = (jb < ep.n_ctiles) ? (__ldg(p.stream_meta + ep.stream_off + jb * kPagesPerTile) >> 8) : G;
             if (last0 == first1) { shared_slot = last0; if (it.split == 1) skip_slot = last0; }
         }
-        float m = kNegInf, l = 0.f, acc = 0.f;                     // l, acc: owner only
-        float mx_prev = kNegInf;                                   // this thread's maximum of the previous tile (unscaled)
+        float m = kNegInf, l = 0.f, acc = 0.f;                     // reference (log2 units), row sum, sum of the current slot
         int cur_slot = -1;
-        // a page's sum goes to its slot; a slot that ends parks its log2-sum-exp
-        auto credit = [&](int slot, float v, float m_ref) {
-            if (slot != cur_slot) {
-                if (cur_slot == skip_slot) bnd = lg2(acc) + m_ref;
-                else if (slot_out && cur_slot >= 0) slot_out[cur_slot] = lg2(acc) + m_ref;
-                acc = 0.f;
-                cur_slot = slot;
-            }
-            acc += v;
-            l += v;
-        };
-        // The owner credits the eight page sums of tile j (its own four and half B's four, both parked in shared
-        // memory) only after it has handed P of tile j + 1 to the MMA warp: the slot book-keeping and its
-        // scattered stores then overlap the MMAs instead of delaying them.  `late` = the factor by which the
-        // running sums were rescaled since those page sums were taken.
-        auto credit_tile = [&](int jt, float late, float m_ref) {
-            const float *src = xsum + (jt % 3) * (kQTiles * kPagesPerTile * 128);
-            const int jg = j_beg + jt;
-            if (jg < ep.n_ctiles) {
-                const int4 *e4 = reinterpret_cast<const int4 *>(p.stream_meta + ep.stream_off + jg * kPagesPerTile);
-                const int4 a = __ldg(e4), b = __ldg(e4 + 1);
-                credit(a.x >> 8, src[0 * 128] * late, m_ref);
-                credit(a.y >> 8, src[1 * 128] * late, m_ref);
-                credit(a.z >> 8, src[2 * 128] * late, m_ref);
-                credit(a.w >> 8, src[3 * 128] * late, m_ref);
-                credit(b.x >> 8, src[4 * 128] * late, m_ref);
-                credit(b.y >> 8, src[5 * 128] * late, m_ref);
-                credit(b.z >> 8, src[6 * 128] * late, m_ref);
-                credit(b.w >> 8, src[7 * 128] * late, m_ref);
-            } else {
-                float v = 0.f;
-#pragma unroll
-                for (int e = 0; e < kPagesPerTile; ++e) v += src[e * 128];
-                credit(G, v * late, m_ref);
+        // the slot that ends parks its log2-sum-exp
+        auto park = [&](float m_ref) {
+            if (cur_slot >= 0) {
+                const float v = lg2(acc) + m_ref;
+                if (cur_slot == skip_slot) bnd = v;
+                else if (slot_out) slot_out[cur_slot] = v;
             }
         };
 
         for (int jj = 0; jj < n_tiles; ++jj) {
             const int j = j_beg + jj;
-            // valid keys of this thread's four pages, one byte each: page padding (cached tiles) or the causal
-            // limit (new-token tiles)
-            uint32_t nvp;
-            if (j < ep.n_ctiles) {
-                const int4 mv = __ldg(reinterpret_cast<const int4 *>(p.stream_meta + ep.stream_off + j * kPagesPerTile) + hb);
-                nvp = static_cast<uint32_t>(mv.x & 0xff) | (static_cast<uint32_t>(mv.y & 0xff) << 8) |
-                      (static_cast<uint32_t>(mv.z & 0xff) << 16) | (static_cast<uint32_t>(mv.w & 0xff) << 24);
+            const bool cached = j < ep.n_ctiles;
+            // Page words of the tile, one per lane 0..7 (slot << 8 | valid keys), and from them two warp-uniform
+            // masks: pages with padding, pages whose slot differs from the page before.  A new-token tile is one
+            // slot (G); its pages are masked from the causal limit of the tile's first row on.
+            int meta = (G << 8) | kPageTokens;
+            if (cached && lane < kPagesPerTile) meta = __ldg(p.stream_meta + ep.stream_off + j * kPagesPerTile + lane);
+            int prev = __shfl_up_sync(kFull, meta >> 8, 1);
+            if (lane == 0) prev = cur_slot;
+            const uint32_t chg_mask = __ballot_sync(kFull, (meta >> 8) != prev) & 0xffu;
+            uint32_t mask_pages;
+            int vis = kTileKeys;                                    // visible keys of this row in a new-token tile
+            if (cached) {
+                mask_pages = __ballot_sync(kFull, (meta & 0xff) < kPageTokens) & 0xffu;
             } else {
-                const int vis = c - (j - ep.n_ctiles) * kTileKeys - hb * kHalfCols + 1;   // visible keys of this half
-                nvp = 0;
-#pragma unroll
-                for (int e = 0; e < kHalfPages; ++e)
-                    nvp |= static_cast<uint32_t>(min(max(vis - e * kPageTokens, 0), kPageTokens)) << (8 * e);
+                const int kbase = (j - ep.n_ctiles) * kTileKeys;
+                vis = c - kbase + 1;
+                const int vis_lo = c_lo - kbase + 1;               // <= vis of every row of the tile
+                mask_pages = vis_lo >= kTileKeys ? 0u : (0xffu << (max(vis_lo, 0) / kPageTokens)) & 0xffu;
             }
-            if (q4 == 0) ENL_TR(warp >> 2, jj, 0);
+
             ok = mbar_wait(bar_s_full(i), static_cast<uint32_t>(jj & 1), abort_flag, p.status);
             if (!ok) break;
             tc_fence_after();
-            if (q4 == 0) ENL_TR(warp >> 2, jj, 1);
 
-            // hide page padding / keys after the causal limit of page e (16 scores), and take the page's maximum
-            auto page_max = [&](int e, float (&sc)[kPageTokens]) -> float {
-                const int nv = static_cast<int>((nvp >> (8 * e)) & 0xffu);
-                if (nv < kPageTokens) {
+            // the row's 128 scores
+            uint32_t su[kTileKeys];
 #pragma unroll
-                    for (int x = 0; x < kPageTokens; ++x)
-                        if (x >= nv) sc[x] = kNegInf;
-                }
-                float a = fmax3(sc[0], sc[1], sc[2]);
+            for (int k = 0; k < 4; ++k)
+                tmem_ld32_issue(t_s + static_cast<uint32_t>(k * 32), reinterpret_cast<uint32_t(&)[32]>(su[k * 32]));
+            tmem_ld_wait();
 #pragma unroll
-                for (int x = 3; x < 15; x += 2) a = fmax3(a, sc[x], sc[x + 1]);
-                return fmaxf(a, sc[15]);
-            };
-            const uint32_t t_half = t_s + static_cast<uint32_t>(hb * kHalfCols);
+            for (int k = 0; k < 4; ++k) tmem_ld32_arrived(reinterpret_cast<uint32_t(&)[32]>(su[k * 32]));
+            float s[kTileKeys];
+#pragma unroll
+            for (int x = 0; x < kTileKeys; ++x) s[x] = __uint_as_float(su[x]);
 
-            // The reference maximum needs the other half's columns too.  Waiting for them every tile would put a
-            // two-warp barrier on the critical path, so the exchange lags by one tile: this tile's exponentials
-            // use the maximum over all EARLIER tiles (both halves know it: the partner's maximum of the previous
-            // tile has been in shared memory since before that tile's P was handed over), and this tile's
-            // maximum only moves the reference for the next one.  A probability may then exceed 1 by the factor
-            // 2^(jump of this tile over everything before it), harmless in floating point up to kMaxJump.  The
-            // first tile, and any tile that starts without a reference, need their own maximum first: a pass over
-            // the scores for the maximum alone, exchanged synchronously.
-            const bool sync_tile = (jj == 0) || __any_sync(0xffffffffu, m == kNegInf);   // same rows, same m in both halves
-            float mx_ref;
-            if (sync_tile) {
-                float mx0 = kNegInf;
-#pragma unroll 1
-                for (int e = 0; e < kHalfPages; ++e) {
-                    uint32_t su[kPageTokens];
-                    tmem_ld16_wait(t_half + static_cast<uint32_t>(e * kPageTokens), su);
-                    float sc[kPageTokens];
+            // hide page padding / keys after the causal limit
+            if (mask_pages) {
 #pragma unroll
-                    for (int x = 0; x < kPageTokens; ++x) sc[x] = __uint_as_float(su[x]);
-                    mx0 = fmaxf(mx0, page_max(e, sc));
+                for (int e = 0; e < kPagesPerTile; ++e) {
+                    if ((mask_pages >> e) & 1u) {
+                        const int nv_e = __shfl_sync(kFull, meta & 0xff, e);
+                        const int bound = cached ? nv_e : vis - e * kPageTokens;
+#pragma unroll
+                        for (int x = 0; x < kPageTokens; ++x)
+                            if (x >= bound) s[e * kPageTokens + x] = kNegInf;
+                    }
                 }
-                xmax_own[(jj & 1) * kXmaxPar] = mx0;
-                ok = pair_sync();
-                if (!ok) break;
-                mx_ref = fmaxf(mx0, xmax_other[(jj & 1) * kXmaxPar]);
-            } else {
-                mx_ref = fmaxf(mx_prev, xmax_other[((jj - 1) & 1) * kXmaxPar]);
             }
-            if (q4 == 0) ENL_TR(warp >> 2, jj, 2);
 
-            float late = 1.f;
-            const float m_cand = mx_ref * scale;
+            // row maximum: four independent chains
+            float mx4[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                float a = fmax3(s[k * 32], s[k * 32 + 1], s[k * 32 + 2]);
+#pragma unroll
+                for (int x = 3; x < 31; x += 2) a = fmax3(a, s[k * 32 + x], s[k * 32 + x + 1]);
+                mx4[k] = fmaxf(a, s[k * 32 + 31]);
+            }
+            const float m_cand = fmaxf(fmax3(mx4[0], mx4[1], mx4[2]), mx4[3]) * scale;
+
+            // The reference moves only when the row maximum has grown by more than the threshold (probabilities
+            // stay below 2^threshold meanwhile); then the sums and the accumulator O_i are rescaled.  O_i holds
+            // the tiles so far and no MMA touches it now: S_i of this tile completed after P_i V of the previous.
             const bool need = m_cand > m + kRescaleThreshold;       // also true when m == -inf < m_cand
-            if (__any_sync(0xffffffffu, need)) {                     // same rows, same decision in both halves
-                // the reference moves by at most kMaxJump per tile, so that the rescale factor cannot underflow
-                // (only a row that has already been reported as out of range is ever held back by this)
-                const float m_new = (m == kNegInf) ? m_cand : fminf(fmaxf(m, m_cand), m + kMaxJump);
+            if (__any_sync(kFull, need)) {
+                const float m_new = fmaxf(m, m_cand);
                 const float alpha = (m_new == kNegInf) ? 1.f : ex2(m - m_new);
                 l *= alpha;
                 acc *= alpha;
-                late = alpha;
                 m = m_new;
-                if (jj > 0) {                                        // O_i holds the tiles so far; each half rescales D/2 columns
+                if (jj > 0) {
 #pragma unroll 1
                     for (int k = 0; k < D / 32; ++k) {
-                        uint32_t o[16];
-                        const uint32_t col = static_cast<uint32_t>(hb * (D / 2) + k * 16);
-                        tmem_ld16_wait(t_o + col, o);
+                        uint32_t o[32];
+                        tmem_ld32_wait(t_o + static_cast<uint32_t>(k * 32), o);
 #pragma unroll
-                        for (int x = 0; x < 16; ++x) o[x] = __float_as_uint(__uint_as_float(o[x]) * alpha);
-                        tmem_st16(t_o + col, o);
+                        for (int x = 0; x < 32; ++x) o[x] = __float_as_uint(__uint_as_float(o[x]) * alpha);
+                        tmem_st32(t_o + static_cast<uint32_t>(k * 32), o);
                     }
                 }
             }
             const float m_use = (m == kNegInf) ? 0.f : m;
-            const float cap = (m_use + kMaxJump) * inv_scale;       // largest score the reference can carry
 
-            // The scores are taken page by page (16 per thread and load; the next page's load is in flight while
-            // this one is worked on): mask, maximum (for the next tile's reference), p = exp2(s * scale - m).  The
-            // page's sum goes to shared memory (the owner credits it to its slot later), its sixteen probabilities
-            // go as eight bf16 pairs (even key in the low half) into P.  Each half keeps its P inside its own 64
-            // columns of S_i: page e at columns hb*64 + 8e .. +7, which only covers scores already taken.
+            // p = exp2(s * scale - m), kept in fp32 for the sums; bf16 pairs (even key in the low half) into P_i,
+            // 32 keys per store, handed to the MMA warp in two halves
             const uint64_t sc2 = pack2(scale, scale), nm2 = pack2(-m_use, -m_use);
-            float *sum_dst = xsum + (jj % 3) * (kQTiles * kPagesPerTile * 128) + hb * (kHalfPages * 128);
-            float mx = kNegInf;
-            uint32_t su[2][kPageTokens];
-            tmem_ld16_issue(t_half, su[0]);
 #pragma unroll
-            for (int e = 0; e < kHalfPages; ++e) {
-                tmem_ld16_arrived(su[e & 1]);
-                if (e + 1 < kHalfPages) tmem_ld16_issue(t_half + static_cast<uint32_t>((e + 1) * kPageTokens), su[(e + 1) & 1]);
-                float sc[kPageTokens];
+            for (int ch = 0; ch < 4; ++ch) {
+                uint32_t pk[16];
 #pragma unroll
-                for (int x = 0; x < kPageTokens; ++x) sc[x] = __uint_as_float(su[e & 1][x]);
-                const float pm = page_max(e, sc);
-                mx = fmaxf(mx, pm);
-                if (pm > cap) {
-                    // beyond what the lagging reference can carry: keep the result finite and report it
-                    atomicExch(p.status, 3);
-#pragma unroll
-                    for (int x = 0; x < kPageTokens; ++x) sc[x] = fminf(sc[x], cap);
-                }
-                uint64_t pr[kPageTokens / 2];
-                uint32_t pk[kPageTokens / 2];
-#pragma unroll
-                for (int x = 0; x < kPageTokens / 2; ++x) {
+                for (int x = 0; x < 16; ++x) {
                     float a0, a1;
-                    unpack2(fma2(pack2(sc[2 * x], sc[2 * x + 1]), sc2, nm2), a0, a1);
+                    unpack2(fma2(pack2(s[ch * 32 + 2 * x], s[ch * 32 + 2 * x + 1]), sc2, nm2), a0, a1);
                     a0 = ex2(a0);
                     a1 = ex2(a1);
-                    pr[x] = pack2(a0, a1);
-                    const __nv_bfloat162 bb = __floats2bfloat162_rn(a0, a1);
-                    pk[x] = *reinterpret_cast<const uint32_t *>(&bb);
+                    s[ch * 32 + 2 * x] = a0;
+                    s[ch * 32 + 2 * x + 1] = a1;
+                    pk[x] = bf16x2(a0, a1);
                 }
-                tmem_st8(t_s + static_cast<uint32_t>(hb * kHalfCols + e * 8), pk);
-                const uint64_t q0 = add2(add2(pr[0], pr[1]), add2(pr[2], pr[3]));
-                const uint64_t q1 = add2(add2(pr[4], pr[5]), add2(pr[6], pr[7]));
-                float b0, b1;
-                unpack2(add2(q0, q1), b0, b1);
-                sum_dst[e * 128] = b0 + b1;
+                tmem_st16(t_s + static_cast<uint32_t>(ch * 16), pk);
+                if (ch & 1) {
+                    tmem_st_wait();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_p_half(i, ch >> 1));
+                }
             }
-            if (!sync_tile) xmax_own[(jj & 1) * kXmaxPar] = mx;     // (a synchronous tile has published it already)
-            mx_prev = mx;
-            if (q4 == 0) ENL_TR(warp >> 2, jj, 3);
-            tmem_st_wait();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_p_full(i));
-            if (q4 == 0) ENL_TR(warp >> 2, jj, 4);
-            if (owner && jj > 0) credit_tile(jj - 1, late, m_use);
+
+            // under the MMAs: page sums, row sum, slots
+            float ps[kPagesPerTile];
+#pragma unroll
+            for (int e = 0; e < kPagesPerTile; ++e) {
+                uint64_t a2 = pack2(s[e * 16], s[e * 16 + 1]);
+#pragma unroll
+                for (int x = 1; x < 8; ++x) a2 = add2(a2, pack2(s[e * 16 + 2 * x], s[e * 16 + 2 * x + 1]));
+                float lo, hi;
+                unpack2(a2, lo, hi);
+                ps[e] = lo + hi;
+            }
+            const float tot = ((ps[0] + ps[1]) + (ps[2] + ps[3])) + ((ps[4] + ps[5]) + (ps[6] + ps[7]));
+            l += tot;
+            if (chg_mask == 0u) {
+                acc += tot;
+            } else {
+#pragma unroll
+                for (int e = 0; e < kPagesPerTile; ++e) {
+                    if ((chg_mask >> e) & 1u) {
+                        park(m_use);
+                        acc = 0.f;
+                        cur_slot = __shfl_sync(kFull, meta >> 8, e);
+                    }
+                    acc += ps[e];
+                }
+            }
         }
 
         // ---- per-row results ----
-        float m_use = (m == kNegInf) ? 0.f : m;
-        bool exported = false;
-        float w_peer = 0.f;
-        if (ok) ok = pair_sync();                                   // half B's sums of the last tile are in place
-        if (ok) {
-            if (owner && n_tiles > 0) credit_tile(n_tiles - 1, 1.f, m_use);
-            const float inv = (l > 0.f) ? 1.f / l : 0.f;
-            float pair_lse = kNegInf, pair_bnd = kNegInf;
-            const float lse = (l > 0.f) ? m_use + lg2(l) : kNegInf;
-            if (owner) {
-                if (cur_slot == skip_slot && cur_slot >= 0) bnd = lg2(acc) + m_use;
-                else if (slot_out && cur_slot >= 0) slot_out[cur_slot] = lg2(acc) + m_use;
-                if (pair) {
-                    // the two CTAs of the cluster tell each other (reference, sum, shared-slot part) of every row
-                    const uint32_t peer = cluster_rank() ^ 1u;
-                    const uint32_t mine = sbase + static_cast<uint32_t>(C::kXpeerOff + (i * 128 + r) * 16);
-                    peer_push4(peer_addr(mine, peer), m_use, l, bnd, 0.f, peer_addr(bar_peer_ml, peer));
-                }
+        const float m_use = (m == kNegInf) ? 0.f : m;
+        const float lse = (l > 0.f) ? m_use + lg2(l) : kNegInf;
+        // (row, head) index of row rr of this warp, or -1 beyond the episode's queries
+        auto row_index = [&](int rr) -> int {
+            const int r2 = q4 * 32 + rr;
+            const int t2 = it.t0 + i * tile_tokens + r2 / rep;
+            if (t2 >= ep.n_q) return -1;
+            const int g2 = ep.q_off + t2;
+            return (split_mode ? it.split * p.n_q_total + g2 : g2) * p.Hq + it.kvh * rep + r2 % rep;
+        };
+        // The warp's 32 rows x 128 bytes leave through the (idle) shared memory of the Q tile: row-per-thread
+        // stores would touch 32 different rows per instruction.  Each thread stages its own 128 bytes, 16-byte
+        // chunks swizzled by row, and the warp writes four whole row pieces per instruction.
+        int ridx8[8];
+#pragma unroll
+        for (int itr = 0; itr < 8; ++itr) ridx8[itr] = row_index(itr * 4 + (lane >> 3));
+        uint8_t *stg = smem + i * C::kTileBytes + q4 * 4096;
+        auto flush_piece = [&](const uint32_t (&w)[32], uint8_t *gbase, long long row_pitch, int piece) {
+#pragma unroll
+            for (int cch = 0; cch < 8; ++cch)
+                *reinterpret_cast<uint4 *>(stg + lane * 128 + ((cch ^ (lane & 7)) << 4)) =
+                    make_uint4(w[4 * cch], w[4 * cch + 1], w[4 * cch + 2], w[4 * cch + 3]);
+            __syncwarp();
+#pragma unroll
+            for (int itr = 0; itr < 8; ++itr) {
+                const int rr = itr * 4 + (lane >> 3), cch = lane & 7;
+                const uint4 v = *reinterpret_cast<const uint4 *>(stg + rr * 128 + ((cch ^ (rr & 7)) << 4));
+                if (ridx8[itr] >= 0)
+                    *reinterpret_cast<uint4 *>(gbase + ridx8[itr] * row_pitch + piece * 128 + cch * 16) = v;
             }
-            if constexpr (D == 128) {
-              if (pair && i != it.split && n_tiles > 0) {
-                // This CTA finishes Q tile `it.split`; the accumulator of the other tile goes to the peer, which
-                // finishes that one.  It goes as it is (relative to this CTA's own reference; the peer learns the
-                // weight from the row sums above), so that nothing but the last MMA stands before it: staged
-                // row-per-thread in the upper half of this CTA's ring (idle once both tiles' MMAs are done; 8 KB per
-                // warp, 16-byte chunks swizzled by row), then one bulk copy per warp into the lower half of the
-                // peer's ring, counted in bytes on the peer's barrier.
-                const uint32_t peer = cluster_rank() ^ 1u;
-                const uint32_t warp_off = static_cast<uint32_t>(kQTiles * C::kTileBytes + (hb * 4 + q4) * 8192);
-                constexpr uint32_t kExportStageOff = 65536;         // upper half of the ring (4 stages x 32 KB)
-                ok = mbar_wait(bar_o_done(i), 0, abort_flag, p.status);
-                if (ok && n_qt == 2) ok = mbar_wait(bar_o_done(i ^ 1), 0, abort_flag, p.status);
-                if (ok) {
-                    tc_fence_after();
-                    uint8_t *stage = smem + warp_off + kExportStageOff + lane * 256;
+            __syncwarp();
+        };
+        // Masses: parked log-sums -> shares of the row's total.  The warp takes its rows one after the other,
+        // lanes over the slots (coalesced), eight rows' loads in flight.  ref / extra: per row (held by the
+        // row's thread) the log-sum-exp of the whole row and, in a pair, the other split's part of the slot
+        // in which the splits meet.
+        const int my_ridx = row_index(lane);
+        auto finish_masses = [&](float ref_mine, float extra_mine, int first, int last) {
+            __syncwarp();                                           // the parked values of all lanes are visible
 #pragma unroll 1
-                    for (int k = 0; k < 2; ++k) {
-                        uint32_t o[32];
-                        tmem_ld32_wait(t_o + static_cast<uint32_t>(hb * (D / 2) + k * 32), o);
+            for (int r0 = 0; r0 < 32; r0 += 8) {
+#pragma unroll 1
+                for (int s0 = first + lane; s0 - lane <= last; s0 += 32) {
+                    float v[8];
+                    float *dst[8];
 #pragma unroll
-                        for (int cch = 0; cch < 8; ++cch)
-                            *reinterpret_cast<uint4 *>(stage + (((k * 8 + cch) ^ (lane & 7)) << 4)) =
-                                make_uint4(o[4 * cch], o[4 * cch + 1], o[4 * cch + 2], o[4 * cch + 3]);
+                    for (int x = 0; x < 8; ++x) {
+                        const int ri = __shfl_sync(kFull, my_ridx, r0 + x);
+                        dst[x] = (ri >= 0 && s0 <= last && s0 != skip_slot)
+                                     ? p.mass + static_cast<long long>(ri) * p.mass_stride + s0 : nullptr;
+                        v[x] = dst[x] ? __ldcg(dst[x]) : kNegInf;
                     }
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                    __syncwarp();
-                    ok = mbar_wait<true>(bar_peer_free, 0, abort_flag, p.status);
-                    if (ok && lane == 0)
-                        peer_bulk_copy(peer_addr(sbase + warp_off, peer), sbase + warp_off + kExportStageOff, 8192,
-                                       peer_addr(bar_peer_o, peer));
-                    exported = ok;
-                }
-              }
-            }
-            if (owner && ok) {
-                if (pair) {
-                    ok = mbar_wait<true>(bar_peer_ml, 0, abort_flag, p.status);
-                    const float4 pe = *reinterpret_cast<const float4 *>(smem + C::kXpeerOff + (i * 128 + r) * 16);
-                    const bool va = l > 0.f, vb = pe.y > 0.f;
-                    const float M = fmaxf(va ? m_use : kNegInf, vb ? pe.x : kNegInf);
-                    const float fa = va ? ex2(m_use - M) : 0.f;
-                    const float L = (va ? l * fa : 0.f) + (vb ? pe.y * ex2(pe.x - M) : 0.f);
-                    pair_lse = (L > 0.f) ? M + lg2(L) : kNegInf;
-                    pair_bnd = pe.z;
-                    *xinv = (L > 0.f) ? fa / L : 0.f;                // weight of this CTA's unnormalised O
-                    w_peer = (L > 0.f && vb) ? ex2(pe.x - M) / L : 0.f;   // and of the peer's
-                    xmax_other[0] = w_peer;                          // for half B (its slot of the exchange area is idle)
-                } else if (split_mode) {
-                    if (row_valid) {
-                        // slots this split did not walk contribute nothing
-                        int first = G + 1, last = -1;
-                        if (n_tiles > 0) {
-                            first = (j_beg < ep.n_ctiles)
-                                        ? (p.stream_meta[ep.stream_off + j_beg * kPagesPerTile] >> 8) : G;
-                            last = (j_end > ep.n_ctiles)
-                                       ? G : (p.stream_meta[ep.stream_off + j_end * kPagesPerTile - 1] >> 8);
+#pragma unroll
+                    for (int x = 0; x < 8; ++x) {
+                        const float ref = __shfl_sync(kFull, ref_mine, r0 + x);
+                        const float extra = __shfl_sync(kFull, extra_mine, r0 + x);
+                        if (dst[x]) {
+                            float w = (ref != kNegInf) ? ex2(v[x] - ref) : 0.f;
+                            if (s0 == shared_slot && ref != kNegInf) w += ex2(extra - ref);
+                            *dst[x] = w;
                         }
-                        if (slot_out)
-                            for (int sl = 0; sl <= G; ++sl)
-                                if (sl < first || sl > last) slot_out[sl] = kNegInf;
-                        p.part_lse[rh] = lse;
-                    }
-                }
-                if (!pair) *xinv = inv;
-                // the row's final log-sum-exp (and the other split's part of the shared slot) for both halves: the
-                // maximum exchange area is idle after the loop
-                xmax_own[0] = pair ? pair_lse : lse;
-                xmax_own[kXmaxPar] = pair_bnd;
-            }
-            if (ok) ok = pair_sync();                               // 1 / row sum (pair merge: the weight) reaches half B
-        }
-        // Masses: parked log-sums -> shares of the row's total, eight slots at a time (eight loads in flight; one
-        // load, one exponential and one store per trip would pay a memory round trip per slot).  Without a peer the
-        // owner does them while half B already writes its output channels and the last MMAs drain.  In a pair both
-        // halves share them, after the output: the other CTA waits for that.  (Both orders were timed.)
-        auto finish_masses = [&]() {
-            if (!(row_valid && p.mass && !split_mode) || (!pair && !owner)) return;
-            float *slots = p.mass + rh * p.mass_stride;
-            const float *xref = owner ? xmax_own : xmax_other;      // written by the owner before the last pair sync
-            const float ref = xref[0], extra = xref[kXmaxPar];
-            int first = 0, last = G;
-            if (pair) {                                             // the slots this CTA walked
-                first = (j_beg < ep.n_ctiles) ? (p.stream_meta[ep.stream_off + j_beg * kPagesPerTile] >> 8) : G;
-                last = (j_end > ep.n_ctiles) ? G : (p.stream_meta[ep.stream_off + j_end * kPagesPerTile - 1] >> 8);
-            }
-            for (int s0 = first + (pair ? 8 * hb : 0); s0 <= last; s0 += (pair ? 16 : 8)) {
-                float v[8];
-#pragma unroll
-                for (int x = 0; x < 8; ++x) v[x] = (s0 + x <= last) ? slots[s0 + x] : kNegInf;
-#pragma unroll
-                for (int x = 0; x < 8; ++x) {
-                    const int sl = s0 + x;
-                    if (sl <= last && sl != skip_slot) {            // the shared slot is written by split 0 alone
-                        float w = (ref != kNegInf) ? ex2(v[x] - ref) : 0.f;
-                        if (sl == shared_slot && ref != kNegInf) w += ex2(extra - ref);
-                        slots[sl] = w;
                     }
                 }
             }
         };
-        const bool masses_first = !pair;
-        if (ok && masses_first) finish_masses();
-        if (pair && !owner) w_peer = xmax_own[0];
-        if (ok && n_tiles > 0 && !(pair && i != it.split)) {
-            const float inv = *xinv;
-            ok = mbar_wait(bar_o_done(i), 0, abort_flag, p.status);
-            if (ok) {
-                tc_fence_after();
-                if constexpr (D == 128) {
-                  if (pair) {
-                    // This CTA finishes Q tile `it.split`: its own accumulator and what the peer sent (see the export
-                    // above), each with its weight.  Thread (warp, lane) reads what thread (warp, lane) of the peer wrote.
-                    const uint32_t peer = cluster_rank() ^ 1u;
-                    const uint32_t ring_off = static_cast<uint32_t>(kQTiles * C::kTileBytes + (hb * 4 + q4) * 8192 + lane * 256);
-                    if (i == it.split) {
-                        uint8_t *stg = smem + i * C::kTileBytes + (hb * 4 + q4) * 4096;
-#pragma unroll 1
-                        for (int k = 0; k < 2 && ok; ++k) {         // 32 channels per pass
-                            uint32_t o[32];
-                            tmem_ld32_wait(t_o + static_cast<uint32_t>(hb * (D / 2) + k * 32), o);
-                            if (k == 0) {
-                                ok = mbar_wait<true>(bar_peer_o, 0, abort_flag, p.status);
-                                // the peer may retire once its staging area has been read out: tell it
-                                if (ok && hb == 0 && q4 == 0 && lane == 0) peer_arrive_relaxed(peer_addr(bar_peer_ack, peer));
-                            }
-                            if (!ok) break;
-#pragma unroll
-                            for (int cch = 0; cch < 4; ++cch) {
-                                const float4 a = *reinterpret_cast<const float4 *>(smem + ring_off + (((k * 8 + 2 * cch) ^ (lane & 7)) << 4));
-                                const float4 b = *reinterpret_cast<const float4 *>(smem + ring_off + (((k * 8 + 2 * cch + 1) ^ (lane & 7)) << 4));
-                                auto mix = [&](uint32_t own, float theirs) { return fmaf(__uint_as_float(own), inv, theirs * w_peer); };
-                                const __nv_bfloat162 b0 = __floats2bfloat162_rn(mix(o[8 * cch + 0], a.x), mix(o[8 * cch + 1], a.y));
-                                const __nv_bfloat162 b1 = __floats2bfloat162_rn(mix(o[8 * cch + 2], a.z), mix(o[8 * cch + 3], a.w));
-                                const __nv_bfloat162 b2 = __floats2bfloat162_rn(mix(o[8 * cch + 4], b.x), mix(o[8 * cch + 5], b.y));
-                                const __nv_bfloat162 b3 = __floats2bfloat162_rn(mix(o[8 * cch + 6], b.z), mix(o[8 * cch + 7], b.w));
-                                *reinterpret_cast<uint4 *>(stg + lane * 128 + (((k * 4 + cch) ^ (lane & 7)) << 4)) =
-                                    make_uint4(*reinterpret_cast<const uint32_t *>(&b0), *reinterpret_cast<const uint32_t *>(&b1),
-                                               *reinterpret_cast<const uint32_t *>(&b2), *reinterpret_cast<const uint32_t *>(&b3));
-                            }
-                        }
-                        __syncwarp();
-                        if (ok) {
-#pragma unroll 1
-                            for (int itr = 0; itr < 8; ++itr) {
-                                const int rr = itr * 4 + (lane >> 3), cch = lane & 7;
-                                const int r2 = q4 * 32 + rr;
-                                const int t2 = it.t0 + i * tile_tokens + r2 / rep;
-                                const long long rh2 = (static_cast<long long>(ep.q_off) + t2) * p.Hq + it.kvh * rep + r2 % rep;
-                                const uint4 v = *reinterpret_cast<const uint4 *>(stg + rr * 128 + ((cch ^ (rr & 7)) << 4));
-                                if (t2 < ep.n_q)
-                                    *reinterpret_cast<uint4 *>(static_cast<__nv_bfloat16 *>(p.out) + rh2 * D + hb * (D / 2) + cch * 8) = v;
-                            }
-                        }
-                    }
-                  } else {
-                    // Row-per-thread stores would touch 32 different rows per instruction.  Each warp stages its
-                    // 32 rows x 128 bytes in the (now idle) shared memory of its Q tile, 16-byte chunks swizzled by
-                    // row, and writes them out four whole 128-byte row pieces per instruction.
-                    uint8_t *stg = smem + i * C::kTileBytes + (hb * 4 + q4) * 4096;
-                    auto row_index = [&](int rr, bool &valid) -> long long {     // (row, head) index of staged row rr
-                        const int r2 = q4 * 32 + rr;
-                        const int t2 = it.t0 + i * tile_tokens + r2 / rep;
-                        valid = t2 < ep.n_q;
-                        const long long g2 = static_cast<long long>(ep.q_off) + t2;
-                        return (split_mode ? (static_cast<long long>(it.split) * p.n_q_total + g2) : g2) * p.Hq +
-                               it.kvh * rep + r2 % rep;
-                    };
-                    if (split_mode) {
-#pragma unroll 1
-                        for (int k = 0; k < 2; ++k) {               // 32 fp32 channels per pass
-                            uint32_t o[32];
-                            const int col = hb * (D / 2) + k * 32;
-                            tmem_ld32_wait(t_o + static_cast<uint32_t>(col), o);
-#pragma unroll
-                            for (int cch = 0; cch < 8; ++cch)
-                                *reinterpret_cast<float4 *>(stg + lane * 128 + ((cch ^ (lane & 7)) << 4)) =
-                                    make_float4(__uint_as_float(o[4 * cch]) * inv, __uint_as_float(o[4 * cch + 1]) * inv,
-                                                __uint_as_float(o[4 * cch + 2]) * inv, __uint_as_float(o[4 * cch + 3]) * inv);
-                            __syncwarp();
-#pragma unroll 1
-                            for (int itr = 0; itr < 8; ++itr) {
-                                const int rr = itr * 4 + (lane >> 3), cch = lane & 7;
-                                bool valid;
-                                const long long rh2 = row_index(rr, valid);
-                                const float4 v = *reinterpret_cast<const float4 *>(stg + rr * 128 + ((cch ^ (rr & 7)) << 4));
-                                if (valid) *reinterpret_cast<float4 *>(p.part_o + rh2 * D + col + cch * 4) = v;
-                            }
-                            __syncwarp();
-                        }
-                    } else {
-#pragma unroll
-                        for (int k = 0; k < 2; ++k) {               // 64 bf16 channels = 128 bytes per row
-                            uint32_t o[32];
-                            tmem_ld32_wait(t_o + static_cast<uint32_t>(hb * (D / 2) + k * 32), o);
-#pragma unroll
-                            for (int cch = 0; cch < 4; ++cch) {
-                                uint32_t w[4];
-#pragma unroll
-                                for (int y = 0; y < 4; ++y) {
-                                    const __nv_bfloat162 b = __floats2bfloat162_rn(
-                                        __uint_as_float(o[8 * cch + 2 * y]) * inv, __uint_as_float(o[8 * cch + 2 * y + 1]) * inv);
-                                    w[y] = *reinterpret_cast<const uint32_t *>(&b);
-                                }
-                                *reinterpret_cast<uint4 *>(stg + lane * 128 + (((k * 4 + cch) ^ (lane & 7)) << 4)) =
-                                    make_uint4(w[0], w[1], w[2], w[3]);
-                            }
-                        }
-                        __syncwarp();
-#pragma unroll 1
-                        for (int itr = 0; itr < 8; ++itr) {
-                            const int rr = itr * 4 + (lane >> 3), cch = lane & 7;
-                            bool valid;
-                            const long long rh2 = row_index(rr, valid);
-                            const uint4 v = *reinterpret_cast<const uint4 *>(stg + rr * 128 + ((cch ^ (rr & 7)) << 4));
-                            if (valid)
-                                *reinterpret_cast<uint4 *>(static_cast<__nv_bfloat16 *>(p.out) + rh2 * D + hb * (D / 2) + cch * 8) = v;
-                        }
-                    }
-                  }
-                } else {
-#pragma unroll
-                for (int k = 0; k < D / 64; ++k) {                  // this half's D/2 output channels
-                    uint32_t o[32];
-                    const int col = hb * (D / 2) + k * 32;
-                    tmem_ld32_wait(t_o + static_cast<uint32_t>(col), o);
-                    if (row_valid) {
-                        if (split_mode) {
-                            float4 *dst = reinterpret_cast<float4 *>(p.part_o + rh * D + col);
-#pragma unroll
-                            for (int x = 0; x < 8; ++x)
-                                dst[x] = make_float4(__uint_as_float(o[4 * x]) * inv, __uint_as_float(o[4 * x + 1]) * inv,
-                                                     __uint_as_float(o[4 * x + 2]) * inv, __uint_as_float(o[4 * x + 3]) * inv);
-                        } else {
-                            uint4 *dst = reinterpret_cast<uint4 *>(
-                                static_cast<__nv_bfloat16 *>(p.out) + rh * D + col);
-#pragma unroll
-                            for (int x = 0; x < 4; ++x) {
-                                uint32_t w[4];
-#pragma unroll
-                                for (int y = 0; y < 4; ++y) {
-                                    const __nv_bfloat162 b = __floats2bfloat162_rn(
-                                        __uint_as_float(o[8 * x + 2 * y]) * inv,
-                                        __uint_as_float(o[8 * x + 2 * y + 1]) * inv);
-                                    w[y] = *reinterpret_cast<const uint32_t *>(&b);
-                                }
-                                dst[x] = make_uint4(w[0], w[1], w[2], w[3]);
-                            }
-                        }
-                    }
-                }
-                }
+        // slots this CTA walked (all of them without splits)
+        int first_slot = 0, last_slot = G;
+        if (p.n_splits > 1) {
+            first_slot = G + 1;
+            last_slot = -1;
+            if (n_tiles > 0) {
+                first_slot = (j_beg < ep.n_ctiles) ? (__ldg(p.stream_meta + ep.stream_off + j_beg * kPagesPerTile) >> 8) : G;
+                last_slot = (j_end > ep.n_ctiles) ? G : (__ldg(p.stream_meta + ep.stream_off + j_end * kPagesPerTile - 1) >> 8);
             }
         }
-        if (ok && !masses_first) finish_masses();
-        // what this CTA staged for its peer must have been fetched before the CTA may retire
-        if (exported) ok = mbar_wait<true>(bar_peer_ack, 0, abort_flag, p.status);
+
+        bool exported = false;
+        if (ok) {
+            park(m_use);
+            if (!pair && !split_mode) {
+                // ---- the whole key stream was this CTA's: output and masses ----
+                if (p.mass) finish_masses(lse, kNegInf, 0, G);
+                if (n_tiles > 0) {
+                    const float inv = (l > 0.f) ? 1.f / l : 0.f;
+                    ok = mbar_wait(bar_o_done(i), 0, abort_flag, p.status);
+                    if (ok) {
+                        tc_fence_after();
+#pragma unroll 1
+                        for (int pc = 0; pc < D / 64; ++pc) {        // 64 bf16 channels = 128 bytes per row and piece
+                            uint32_t o[32], w[32];
+#pragma unroll
+                            for (int k = 0; k < 2; ++k) {
+                                tmem_ld32_wait(t_o + static_cast<uint32_t>(pc * 64 + k * 32), o);
+#pragma unroll
+                                for (int x = 0; x < 16; ++x)
+                                    w[k * 16 + x] = bf16x2(__uint_as_float(o[2 * x]) * inv, __uint_as_float(o[2 * x + 1]) * inv);
+                            }
+                            flush_piece(w, static_cast<uint8_t *>(p.out), D * 2, pc);
+                        }
+                    }
+                }
+            } else if (split_mode) {
+                // ---- partial results for the merge kernel: O / l in fp32, the row's log-sum-exp, raw slot log-sums ----
+                if (row_valid) p.part_lse[rh] = lse;
+                if (p.part_slot) {
+                    __syncwarp();
+#pragma unroll 1
+                    for (int rr = 0; rr < 32; ++rr) {               // slots this split did not walk contribute nothing
+                        const int ri = __shfl_sync(kFull, my_ridx, rr);
+                        if (ri < 0) continue;
+                        float *slots = p.part_slot + static_cast<long long>(ri) * p.mass_stride;
+                        for (int sl = lane; sl <= G; sl += 32)
+                            if (sl < first_slot || sl > last_slot) slots[sl] = kNegInf;
+                    }
+                }
+                if (n_tiles > 0) {
+                    const float inv = (l > 0.f) ? 1.f / l : 0.f;
+                    ok = mbar_wait(bar_o_done(i), 0, abort_flag, p.status);
+                    if (ok) {
+                        tc_fence_after();
+#pragma unroll 1
+                        for (int pc = 0; pc < D / 32; ++pc) {        // 32 fp32 channels = 128 bytes per row and piece
+                            uint32_t o[32];
+                            tmem_ld32_wait(t_o + static_cast<uint32_t>(pc * 32), o);
+#pragma unroll
+                            for (int x = 0; x < 32; ++x) o[x] = __float_as_uint(__uint_as_float(o[x]) * inv);
+                            flush_piece(o, reinterpret_cast<uint8_t *>(p.part_o), D * 4, pc);
+                        }
+                    }
+                }
+            } else {
+              if constexpr (D == 128) {
+                // ---- pair merge: the two CTAs of the cluster hold the two halves of the key stream ----
+                const uint32_t peer = cluster_rank() ^ 1u;
+                // they tell each other (reference, sum, shared-slot part) of every row
+                {
+                    const uint32_t mine = sbase + static_cast<uint32_t>(C::kXpeerOff + (i * 128 + r) * 16);
+                    peer_push4(peer_addr(mine, peer), m_use, l, bnd, 0.f, peer_addr(bar_peer_ml, peer));
+                }
+                constexpr uint32_t kRingOff = kQTiles * C::kTileBytes;
+                constexpr uint32_t kExportStageOff = 65536;         // upper half of the ring (4 stages x 32 KB)
+                const uint32_t warp_off = kRingOff + static_cast<uint32_t>(q4 * 16384);
+                if (i != it.split && n_tiles > 0) {
+                    // This CTA finishes Q tile `it.split`; the accumulator of the other tile goes to the peer, which
+                    // finishes that one.  It goes as it is (relative to this CTA's own reference; the peer learns the
+                    // weight from the row sums above), so that nothing but the last MMA stands before it: staged
+                    // row-per-thread in the upper half of this CTA's ring (idle once both tiles' MMAs are done; 16 KB
+                    // per warp, 16-byte chunks swizzled by row), then one bulk copy per warp into the lower half of
+                    // the peer's ring, counted in bytes on the peer's barrier.
+                    ok = mbar_wait(bar_o_done(i), 0, abort_flag, p.status);
+                    if (ok && n_qt == 2) ok = mbar_wait(bar_o_done(i ^ 1), 0, abort_flag, p.status);
+                    if (ok) {
+                        tc_fence_after();
+                        uint8_t *stage = smem + warp_off + kExportStageOff + lane * 512;
+#pragma unroll 1
+                        for (int k = 0; k < 4; ++k) {
+                            uint32_t o[32];
+                            tmem_ld32_wait(t_o + static_cast<uint32_t>(k * 32), o);
+#pragma unroll
+                            for (int cch = 0; cch < 8; ++cch)
+                                *reinterpret_cast<uint4 *>(stage + (((k * 8 + cch) ^ (lane & 7)) << 4)) =
+                                    make_uint4(o[4 * cch], o[4 * cch + 1], o[4 * cch + 2], o[4 * cch + 3]);
+                        }
+                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                        __syncwarp();
+                        ok = mbar_wait<true>(bar_peer_free, 0, abort_flag, p.status);
+                        if (ok && lane == 0)
+                            peer_bulk_copy(peer_addr(sbase + warp_off, peer), sbase + warp_off + kExportStageOff, 16384,
+                                           peer_addr(bar_peer_o, peer));
+                        exported = ok;
+                    }
+                }
+                // the merged row: reference, sum, weights of the two accumulators
+                float pair_lse = kNegInf, pair_bnd = kNegInf, w_own = 0.f, w_peer = 0.f;
+                if (ok) ok = mbar_wait<true>(bar_peer_ml, 0, abort_flag, p.status);
+                if (ok) {
+                    const float4 pe = *reinterpret_cast<const float4 *>(smem + C::kXpeerOff + (i * 128 + r) * 16);
+                    const bool va = l > 0.f, vb = pe.y > 0.f;
+                    const float M = fmaxf(va ? m_use : kNegInf, vb ? pe.x : kNegInf);
+                    const float fa = va ? ex2(m_use - M) : 0.f;
+                    const float fb = vb ? ex2(pe.x - M) : 0.f;
+                    const float L = (va ? l * fa : 0.f) + (vb ? pe.y * fb : 0.f);
+                    pair_lse = (L > 0.f) ? M + lg2(L) : kNegInf;
+                    pair_bnd = pe.z;
+                    w_own = (L > 0.f) ? fa / L : 0.f;
+                    w_peer = (L > 0.f) ? fb / L : 0.f;
+                }
+                if (ok && i == it.split && n_tiles > 0) {
+                    // this CTA finishes the tile: its own accumulator and what the peer sent, each with its weight;
+                    // thread (warp, lane) reads what thread (warp, lane) of the peer wrote
+                    ok = mbar_wait(bar_o_done(i), 0, abort_flag, p.status);
+                    if (ok) {
+                        tc_fence_after();
+                        ok = mbar_wait<true>(bar_peer_o, 0, abort_flag, p.status);
+                        // the peer may retire once its staging area has been read out: tell it
+                        if (ok && q4 == 0 && lane == 0) peer_arrive_relaxed(peer_addr(bar_peer_ack, peer));
+                    }
+                    if (ok) {
+                        const uint8_t *theirs = smem + warp_off + lane * 512;
+#pragma unroll 1
+                        for (int pc = 0; pc < 2; ++pc) {
+                            uint32_t o[32], w[32];
+#pragma unroll
+                            for (int k = 0; k < 2; ++k) {
+                                tmem_ld32_wait(t_o + static_cast<uint32_t>(pc * 64 + k * 32), o);
+#pragma unroll
+                                for (int cch = 0; cch < 8; ++cch) {
+                                    const float4 a = *reinterpret_cast<const float4 *>(
+                                        theirs + ((((pc * 2 + k) * 8 + cch) ^ (lane & 7)) << 4));
+                                    auto mix = [&](uint32_t own, float th) { return fmaf(__uint_as_float(own), w_own, th * w_peer); };
+                                    w[k * 16 + 2 * cch] = bf16x2(mix(o[4 * cch], a.x), mix(o[4 * cch + 1], a.y));
+                                    w[k * 16 + 2 * cch + 1] = bf16x2(mix(o[4 * cch + 2], a.z), mix(o[4 * cch + 3], a.w));
+                                }
+                            }
+                            flush_piece(w, static_cast<uint8_t *>(p.out), D * 2, pc);
+                        }
+                    }
+                }
+                // each CTA writes the slots it walked against the merged log-sum-exp; the slot both walked is
+                // written by split 0, which adds the part split 1 sent
+                if (ok && p.mass) finish_masses(pair_lse, pair_bnd, first_slot, last_slot);
+                // what this CTA staged for its peer must have been fetched before the CTA may retire
+                if (exported) ok = mbar_wait<true>(bar_peer_ack, 0, abort_flag, p.status);
+              }
+            }
+        }
       }
     }
 
@@ -1041,13 +926,6 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
 }
 
 }  // namespace
-
-#ifdef ENL_TRACE
-extern "C" int enl_debug_trace(long long *out)
-{
-    return cudaMemcpyFromSymbol(out, g_trace, sizeof(g_trace)) == cudaSuccess ? 0 : -1;
-}
-#endif
 
 size_t attention_smem_bytes(int head_dim)
 {

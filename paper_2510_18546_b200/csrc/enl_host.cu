@@ -167,7 +167,6 @@ extern "C" const char *enl_strerror(int code)
         case ENL_E_CUDA: return "CUDA error, or GPU operation on a bookkeeping-only cache";
         case ENL_E_TIMEOUT: return "a bounded wait inside a kernel expired";
         case ENL_E_LIMIT: return "size beyond the fixed maxima of the entry point that allocates nothing";
-        case ENL_E_RANGE: return "scores rose by more than 2^100 within one key tile; probabilities were clamped";
         case ENL_E_EVICTED: return "the group is in the slow tier only; enl_step_prepare loads it";
         default: return "unknown error";
     }
@@ -290,7 +289,7 @@ extern "C" int enl_cache_status(enl_cache_t *c)
         cudaMemset(c->status_dev, 0, sizeof st);
         // a decode launch that gave up may have left its split counters half counted
         cudaMemset(c->counters_dev, 0, sizeof(int32_t) * c->d.max_batch * c->d.n_kv_heads);
-        return st == 3 ? ENL_E_RANGE : ENL_E_TIMEOUT;
+        return ENL_E_TIMEOUT;
     }
     return ENL_OK;
 }

@@ -19,7 +19,7 @@ ENL_BF16 = 1
 ENL_DEVICE_NONE = -1
 ENL_REPLACE, ENL_APPEND = 0, 1
 ENL_PLAN_ONLY = 1
-ENL_OK, ENL_E_INVAL, ENL_E_NOGROUP, ENL_E_NOMEM, ENL_E_CUDA, ENL_E_TIMEOUT, ENL_E_LIMIT, ENL_E_RANGE, ENL_E_EVICTED = 0, -1, -2, -3, -4, -5, -6, -7, -8
+ENL_OK, ENL_E_INVAL, ENL_E_NOGROUP, ENL_E_NOMEM, ENL_E_CUDA, ENL_E_TIMEOUT, ENL_E_LIMIT, ENL_E_EVICTED = 0, -1, -2, -3, -4, -5, -6, -8
 ENL_STATIC_MAX_SEGMENTS, ENL_STATIC_MAX_KEYS, ENL_STATIC_SCRATCH_BYTES = 255, 65536, 4 << 20
 
 EXPORTS = ("enl_cache_create", "enl_group_store", "enl_attend", "enl_cache_free", "enl_strerror",
