@@ -193,21 +193,27 @@ __device__ __forceinline__ void tc_commit(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-// D[tmem] (+)= A[smem] * B[smem]
-__device__ __forceinline__ void mma_ss(uint32_t d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc)
+// D[tmem] (+)= A[smem] * B[smem] and D[tmem] (+)= A[tmem] * B[smem], issued by one thread.  The shared-memory
+// descriptors are given as (low word, high word): the high word is constant and the low word (the start address
+// field) moves by a small constant from one MMA to the next, so the issuing thread spends one integer add per
+// operand instead of rebuilding descriptors: a lone thread pays the full latency of every instruction, and it has
+// to stay ahead of a pipe that retires an MMA every ~65 cycles.
+__device__ __forceinline__ void mma_ss2(uint32_t d, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                        uint32_t idesc, uint32_t acc)
 {
     asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "mov.b64 da, {%1, %2};\n\tmov.b64 db, {%3, %4};\n\tsetp.ne.b32 p, %6, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}"
+        ::"r"(d), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(acc) : "memory");
 }
-// D[tmem] (+)= A[tmem] * B[smem]
-__device__ __forceinline__ void mma_ts(uint32_t d, uint32_t a, uint64_t bdesc, uint32_t idesc, uint32_t acc)
+__device__ __forceinline__ void mma_ts2(uint32_t d, uint32_t a, uint32_t b_lo, uint32_t b_hi, uint32_t idesc, uint32_t acc)
 {
     asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-        ::"r"(d), "r"(a), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+        "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
+        "mov.b64 db, {%2, %3};\n\tsetp.ne.b32 p, %5, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}"
+        ::"r"(d), "r"(a), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(acc) : "memory");
 }
 __device__ __forceinline__ float ex2(float x)
 {
@@ -429,13 +435,22 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
             constexpr uint32_t idesc_pv = make_idesc(D, true);
             auto tmem_s = [&](int i) { return tmem_base + static_cast<uint32_t>(i * 128); };
             auto tmem_o = [&](int i) { return tmem_base + static_cast<uint32_t>(256 + i * 128); };
+            // descriptor words: Q tile i and ring stage st start (kTileBytes >> 4) address units apart
+            const uint64_t dq0 = smem_desc(q_addr(0), 16), dk0 = smem_desc(stage_addr(0), 16),
+                           dv0 = smem_desc(stage_addr(0), C::kHalfBytes);
+            const uint32_t dq_lo = static_cast<uint32_t>(dq0), dq_hi = static_cast<uint32_t>(dq0 >> 32);
+            const uint32_t dk_lo = static_cast<uint32_t>(dk0), dk_hi = static_cast<uint32_t>(dk0 >> 32);
+            const uint32_t dv_lo = static_cast<uint32_t>(dv0), dv_hi = static_cast<uint32_t>(dv0 >> 32);
+            constexpr uint32_t kTileUnits = C::kTileBytes >> 4;
             auto issue_qk = [&](int i, int st) {
                 if (lane == 0) {
+                    const uint32_t a = dq_lo + static_cast<uint32_t>(i) * kTileUnits, b = dk_lo + static_cast<uint32_t>(st) * kTileUnits;
+                    const uint32_t d = tmem_s(i);
 #pragma unroll
                     for (int kk = 0; kk < D / 16; ++kk) {
-                        const uint32_t off = static_cast<uint32_t>((kk >> 2) * C::kHalfBytes + (kk & 3) * 32);
-                        mma_ss(tmem_s(i), smem_desc(q_addr(i) + off, 16), smem_desc(stage_addr(st) + off, 16),
-                               idesc_qk, kk > 0 ? 1u : 0u);
+                        constexpr uint32_t kHalfUnits = C::kHalfBytes >> 4;
+                        const uint32_t off = static_cast<uint32_t>((kk >> 2) * kHalfUnits + (kk & 3) * 2);   // 32 bytes per 16 channels
+                        mma_ss2(d, a + off, dq_hi, b + off, dk_hi, idesc_qk, kk > 0 ? 1u : 0u);
                     }
                     tc_commit(bar_s_full(i));
                 }
@@ -444,13 +459,12 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
             // O_i (+)= P_i[:, 64 hf .. 64 hf + 63] V[64 hf .. 64 hf + 63, :]; P of keys 2c, 2c+1 sits in column c of S_i
             auto issue_pv = [&](int i, int st, int hf, bool first_tile) {
                 if (lane == 0) {
+                    const uint32_t b = dv_lo + static_cast<uint32_t>(st) * kTileUnits + static_cast<uint32_t>(hf) * (4u * 128u);
+                    const uint32_t d = tmem_o(i), a = tmem_s(i) + static_cast<uint32_t>(hf * 32);
 #pragma unroll
-                    for (int k4 = 0; k4 < 4; ++k4) {
-                        const int kk = hf * 4 + k4;
-                        mma_ts(tmem_o(i), tmem_s(i) + static_cast<uint32_t>(kk * 8),
-                               smem_desc(stage_addr(st) + static_cast<uint32_t>(kk * 16 * 128), C::kHalfBytes),
-                               idesc_pv, (first_tile && kk == 0) ? 0u : 1u);
-                    }
+                    for (int k4 = 0; k4 < 4; ++k4)                      // 16 keys = 16 rows of 128 B = 128 address units, 8 columns of P
+                        mma_ts2(d, a + static_cast<uint32_t>(k4 * 8), b + static_cast<uint32_t>(k4 * 128), dv_hi, idesc_pv,
+                                (first_tile && hf == 0 && k4 == 0) ? 0u : 1u);
                 }
                 __syncwarp();
             };
@@ -547,14 +561,22 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
             }
         };
 
+        // Page words of a tile, one per lane 0..7 (slot << 8 | valid keys); a new-token tile is one slot (G).  They
+        // are fetched one tile ahead: the load's latency would otherwise sit between two tiles of this warp.
+        auto load_meta = [&](int j) -> int {
+            int w = (G << 8) | kPageTokens;
+            if (j < ep.n_ctiles && lane < kPagesPerTile) w = __ldg(p.stream_meta + ep.stream_off + j * kPagesPerTile + lane);
+            return w;
+        };
+        int meta_next = n_tiles > 0 ? load_meta(j_beg) : 0;
+
         for (int jj = 0; jj < n_tiles; ++jj) {
             const int j = j_beg + jj;
             const bool cached = j < ep.n_ctiles;
-            // Page words of the tile, one per lane 0..7 (slot << 8 | valid keys), and from them two warp-uniform
-            // masks: pages with padding, pages whose slot differs from the page before.  A new-token tile is one
-            // slot (G); its pages are masked from the causal limit of the tile's first row on.
-            int meta = (G << 8) | kPageTokens;
-            if (cached && lane < kPagesPerTile) meta = __ldg(p.stream_meta + ep.stream_off + j * kPagesPerTile + lane);
+            // From the page words two warp-uniform masks: pages with padding, pages whose slot differs from the
+            // page before.  The pages of a new-token tile are masked from the causal limit of the tile's first row on.
+            const int meta = meta_next;
+            if (jj + 1 < n_tiles) meta_next = load_meta(j + 1);
             int prev = __shfl_up_sync(kFull, meta >> 8, 1);
             if (lane == 0) prev = cur_slot;
             const uint32_t chg_mask = __ballot_sync(kFull, (meta >> 8) != prev) & 0xffu;
@@ -586,29 +608,32 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
             for (int x = 0; x < kTileKeys; ++x) s[x] = __uint_as_float(su[x]);
 
             // hide page padding / keys after the causal limit
-            if (mask_pages) {
-#pragma unroll
-                for (int e = 0; e < kPagesPerTile; ++e) {
-                    if ((mask_pages >> e) & 1u) {
-                        const int nv_e = __shfl_sync(kFull, meta & 0xff, e);
-                        const int bound = cached ? nv_e : vis - e * kPageTokens;
-#pragma unroll
-                        for (int x = 0; x < kPageTokens; ++x)
-                            if (x >= bound) s[e * kPageTokens + x] = kNegInf;
-                    }
+            for (uint32_t todo = mask_pages; todo; todo &= todo - 1u) {
+                const int e = __ffs(static_cast<int>(todo)) - 1;    // warp-uniform
+                const int nv_e = __shfl_sync(kFull, meta & 0xff, e);
+                const int bound = cached ? nv_e : vis - e * kPageTokens;
+                switch (e) {
+#define ENL_MASK_PAGE(E)                                                          \
+                    case E:                                                       \
+                        _Pragma("unroll") for (int x = 0; x < kPageTokens; ++x)   \
+                            if (x >= bound) s[E * kPageTokens + x] = kNegInf;     \
+                        break;
+                    ENL_MASK_PAGE(0) ENL_MASK_PAGE(1) ENL_MASK_PAGE(2) ENL_MASK_PAGE(3)
+                    ENL_MASK_PAGE(4) ENL_MASK_PAGE(5) ENL_MASK_PAGE(6) ENL_MASK_PAGE(7)
+#undef ENL_MASK_PAGE
                 }
             }
 
-            // row maximum: four independent chains
-            float mx4[4];
+            // row maximum: eight independent chains
+            float mx8[kPagesPerTile];
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                float a = fmax3(s[k * 32], s[k * 32 + 1], s[k * 32 + 2]);
+            for (int k = 0; k < kPagesPerTile; ++k) {
+                float a = fmax3(s[k * 16], s[k * 16 + 1], s[k * 16 + 2]);
 #pragma unroll
-                for (int x = 3; x < 31; x += 2) a = fmax3(a, s[k * 32 + x], s[k * 32 + x + 1]);
-                mx4[k] = fmaxf(a, s[k * 32 + 31]);
+                for (int x = 3; x < 15; x += 2) a = fmax3(a, s[k * 16 + x], s[k * 16 + x + 1]);
+                mx8[k] = fmaxf(a, s[k * 16 + 15]);
             }
-            const float m_cand = fmaxf(fmax3(mx4[0], mx4[1], mx4[2]), mx4[3]) * scale;
+            const float m_cand = fmax3(fmax3(mx8[0], mx8[1], mx8[2]), fmax3(mx8[3], mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])) * scale;
 
             // The reference moves only when the row maximum has grown by more than the threshold (probabilities
             // stay below 2^threshold meanwhile); then the sums and the accumulator O_i are rescaled.  O_i holds
@@ -633,21 +658,24 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
             }
             const float m_use = (m == kNegInf) ? 0.f : m;
 
-            // p = exp2(s * scale - m), kept in fp32 for the sums; bf16 pairs (even key in the low half) into P_i,
-            // 32 keys per store, handed to the MMA warp in two halves
+            // p = exp2(s * scale - m) in fp32; bf16 pairs (even key in the low half) into P_i, 32 keys per store, handed
+            // to the MMA warp in two halves.  The page sums (of the fp32 values) are taken along the way: their adds
+            // fill issue slots that the exponentials leave free.
             const uint64_t sc2 = pack2(scale, scale), nm2 = pack2(-m_use, -m_use);
+            uint64_t ps2[kPagesPerTile];
 #pragma unroll
             for (int ch = 0; ch < 4; ++ch) {
                 uint32_t pk[16];
 #pragma unroll
                 for (int x = 0; x < 16; ++x) {
+                    const int e = ch * 2 + (x >> 3);
                     float a0, a1;
                     unpack2(fma2(pack2(s[ch * 32 + 2 * x], s[ch * 32 + 2 * x + 1]), sc2, nm2), a0, a1);
                     a0 = ex2(a0);
                     a1 = ex2(a1);
-                    s[ch * 32 + 2 * x] = a0;
-                    s[ch * 32 + 2 * x + 1] = a1;
+                    const uint64_t p2 = pack2(a0, a1);
                     pk[x] = bf16x2(a0, a1);
+                    ps2[e] = (x & 7) ? add2(ps2[e], p2) : p2;
                 }
                 tmem_st16(t_s + static_cast<uint32_t>(ch * 16), pk);
                 if (ch & 1) {
@@ -658,15 +686,12 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                 }
             }
 
-            // under the MMAs: page sums, row sum, slots
+            // under the MMAs: row sum, slots
             float ps[kPagesPerTile];
 #pragma unroll
             for (int e = 0; e < kPagesPerTile; ++e) {
-                uint64_t a2 = pack2(s[e * 16], s[e * 16 + 1]);
-#pragma unroll
-                for (int x = 1; x < 8; ++x) a2 = add2(a2, pack2(s[e * 16 + 2 * x], s[e * 16 + 2 * x + 1]));
                 float lo, hi;
-                unpack2(a2, lo, hi);
+                unpack2(ps2[e], lo, hi);
                 ps[e] = lo + hi;
             }
             const float tot = ((ps[0] + ps[1]) + (ps[2] + ps[3])) + ((ps[4] + ps[5]) + (ps[6] + ps[7]));
