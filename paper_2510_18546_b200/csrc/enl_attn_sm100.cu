@@ -35,8 +35,8 @@ namespace {
 
 constexpr int kThreads      = 384;
 constexpr int kSoftmaxWarps = 8;
-constexpr int kRegsSoftmax  = 216;            // 256 x 216 + 128 x 72 = 384 x 168, what the launch allocates
-constexpr int kRegsOther    = 72;
+constexpr int kRegsSoftmax  = 208;            // 256 x 208 + 128 x 80 <= 384 x 168, what the launch allocates
+constexpr int kRegsOther    = 80;
 constexpr int kProducerWarp = 8;
 constexpr int kMmaWarp      = 9;
 constexpr uint32_t kTmemCols = 512;
@@ -84,6 +84,17 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok) : "r"(bar), "r"(parity), "r"(kSuspendHintNs) : "memory");
+    return ok != 0;
+}
+// A test that never suspends (about 35 cycles until its result can be used, half of a poll with a suspend hint).
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
 // The same poll with acquire semantics at cluster scope: data another CTA of the cluster wrote before its
@@ -153,7 +164,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
                                           int32_t *status)
 {
     auto poll = [&]() { return kCluster ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity); };
-    bool ok = poll();
+    bool ok = kCluster ? poll() : mbar_test(bar, parity);       // the common case: already complete
     if (!ok) {
         // the clock is read only every 16 failed polls (the first reading starts the limit): a poll already
         // sleeps inside the instruction
@@ -189,31 +200,36 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *tm,
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after()  { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar)
-{
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-// D[tmem] (+)= A[smem] * B[smem] and D[tmem] (+)= A[tmem] * B[smem], issued by one thread.  The shared-memory
-// descriptors are given as (low word, high word): the high word is constant and the low word (the start address
-// field) moves by a small constant from one MMA to the next, so the issuing thread spends one integer add per
-// operand instead of rebuilding descriptors: a lone thread pays the full latency of every instruction, and it has
-// to stay ahead of a pipe that retires an MMA every ~65 cycles.
+// D[tmem] (+)= A[smem] * B[smem] and D[tmem] (+)= A[tmem] * B[smem].  The whole warp executes the surrounding code
+// and these wrappers; only the lane with `issue` != 0 issues the instruction.  Issuing from inside a one-lane branch
+// was measured at ~60 cycles per MMA (a diverged warp pays the full latency of every instruction and cannot use the
+// uniform datapath for the descriptors), against ~10 cycles this way; the pipe retires an MMA every ~65 cycles.
+// The shared-memory descriptors are given as (low word, high word): the high word is constant and the low word (the
+// start address field) moves by a small constant from one MMA to the next.
 __device__ __forceinline__ void mma_ss2(uint32_t d, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
-                                        uint32_t idesc, uint32_t acc)
+                                        uint32_t idesc, uint32_t acc, uint32_t issue)
 {
     asm volatile(
-        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
-        "mov.b64 da, {%1, %2};\n\tmov.b64 db, {%3, %4};\n\tsetp.ne.b32 p, %6, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}"
-        ::"r"(d), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(acc) : "memory");
+        "{\n\t.reg .pred p, q;\n\t.reg .b64 da, db;\n\t"
+        "mov.b64 da, {%1, %2};\n\tmov.b64 db, {%3, %4};\n\tsetp.ne.b32 p, %6, 0;\n\tsetp.ne.b32 q, %7, 0;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}"
+        ::"r"(d), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(acc), "r"(issue) : "memory");
 }
-__device__ __forceinline__ void mma_ts2(uint32_t d, uint32_t a, uint32_t b_lo, uint32_t b_hi, uint32_t idesc, uint32_t acc)
+__device__ __forceinline__ void mma_ts2(uint32_t d, uint32_t a, uint32_t b_lo, uint32_t b_hi, uint32_t idesc, uint32_t acc,
+                                        uint32_t issue)
 {
     asm volatile(
-        "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
-        "mov.b64 db, {%2, %3};\n\tsetp.ne.b32 p, %5, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}"
-        ::"r"(d), "r"(a), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(acc) : "memory");
+        "{\n\t.reg .pred p, q;\n\t.reg .b64 db;\n\t"
+        "mov.b64 db, {%2, %3};\n\tsetp.ne.b32 p, %5, 0;\n\tsetp.ne.b32 q, %6, 0;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}"
+        ::"r"(d), "r"(a), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(acc), "r"(issue) : "memory");
+}
+__device__ __forceinline__ void tc_commit_if(uint32_t bar, uint32_t issue)
+{
+    asm volatile(
+        "{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %1, 0;\n\t"
+        "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+        ::"r"(bar), "r"(issue) : "memory");
 }
 __device__ __forceinline__ float ex2(float x)
 {
@@ -442,40 +458,43 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
             const uint32_t dk_lo = static_cast<uint32_t>(dk0), dk_hi = static_cast<uint32_t>(dk0 >> 32);
             const uint32_t dv_lo = static_cast<uint32_t>(dv0), dv_hi = static_cast<uint32_t>(dv0 >> 32);
             constexpr uint32_t kTileUnits = C::kTileBytes >> 4;
+            const uint32_t issue = lane == 0 ? 1u : 0u;
             auto issue_qk = [&](int i, int st) {
-                if (lane == 0) {
-                    const uint32_t a = dq_lo + static_cast<uint32_t>(i) * kTileUnits, b = dk_lo + static_cast<uint32_t>(st) * kTileUnits;
-                    const uint32_t d = tmem_s(i);
+                const uint32_t a = dq_lo + static_cast<uint32_t>(i) * kTileUnits, b = dk_lo + static_cast<uint32_t>(st) * kTileUnits;
+                const uint32_t d = tmem_s(i);
 #pragma unroll
-                    for (int kk = 0; kk < D / 16; ++kk) {
-                        constexpr uint32_t kHalfUnits = C::kHalfBytes >> 4;
-                        const uint32_t off = static_cast<uint32_t>((kk >> 2) * kHalfUnits + (kk & 3) * 2);   // 32 bytes per 16 channels
-                        mma_ss2(d, a + off, dq_hi, b + off, dk_hi, idesc_qk, kk > 0 ? 1u : 0u);
-                    }
-                    tc_commit(bar_s_full(i));
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    constexpr uint32_t kHalfUnits = C::kHalfBytes >> 4;
+                    const uint32_t off = static_cast<uint32_t>((kk >> 2) * kHalfUnits + (kk & 3) * 2);   // 32 bytes per 16 channels
+                    mma_ss2(d, a + off, dq_hi, b + off, dk_hi, idesc_qk, kk > 0 ? 1u : 0u, issue);
                 }
-                __syncwarp();
+                tc_commit_if(bar_s_full(i), issue);
             };
             // O_i (+)= P_i[:, 64 hf .. 64 hf + 63] V[64 hf .. 64 hf + 63, :]; P of keys 2c, 2c+1 sits in column c of S_i
             auto issue_pv = [&](int i, int st, int hf, bool first_tile) {
-                if (lane == 0) {
-                    const uint32_t b = dv_lo + static_cast<uint32_t>(st) * kTileUnits + static_cast<uint32_t>(hf) * (4u * 128u);
-                    const uint32_t d = tmem_o(i), a = tmem_s(i) + static_cast<uint32_t>(hf * 32);
+                const uint32_t b = dv_lo + static_cast<uint32_t>(st) * kTileUnits + static_cast<uint32_t>(hf) * (4u * 128u);
+                const uint32_t d = tmem_o(i), a = tmem_s(i) + static_cast<uint32_t>(hf * 32);
 #pragma unroll
-                    for (int k4 = 0; k4 < 4; ++k4)                      // 16 keys = 16 rows of 128 B = 128 address units, 8 columns of P
-                        mma_ts2(d, a + static_cast<uint32_t>(k4 * 8), b + static_cast<uint32_t>(k4 * 128), dv_hi, idesc_pv,
-                                (first_tile && hf == 0 && k4 == 0) ? 0u : 1u);
-                }
-                __syncwarp();
+                for (int k4 = 0; k4 < 4; ++k4)                          // 16 keys = 16 rows of 128 B = 128 address units, 8 columns of P
+                    mma_ts2(d, a + static_cast<uint32_t>(k4 * 8), b + static_cast<uint32_t>(k4 * 128), dv_hi, idesc_pv,
+                            (first_tile && hf == 0 && k4 == 0) ? 0u : 1u, issue);
             };
-            auto commit_to = [&](uint32_t bar) {
-                if (lane == 0) tc_commit(bar);
-                __syncwarp();
-            };
+            auto commit_to = [&](uint32_t bar) { tc_commit_if(bar, issue); };
             auto wait_full = [&](int f) {
                 return mbar_wait(bar_kv_full(f % C::kStages), static_cast<uint32_t>((f / C::kStages) & 1),
                                  abort_flag, p.status);
             };
+
+            // A barrier the issuer will need is tested one batch of MMAs ahead ("armed"), so that the test's latency
+            // passes while the batch is issued; only a barrier that was not complete then is waited for.  The queue in
+            // front of the pipe holds about four MMAs: a wait of a few hundred cycles between two batches empties it.
+            struct Pending { uint32_t bar, par; bool pre; };
+            auto arm = [&](uint32_t bar, uint32_t par) { return Pending{bar, par, mbar_test(bar, par)}; };
+            auto await = [&](const Pending &w) {
+                return __all_sync(kFull, w.pre) ? true : mbar_wait(w.bar, w.par, abort_flag, p.status);
+            };
+            auto full_bar = [&](int f) { return bar_kv_full(f % C::kStages); };
+            auto full_par = [&](int f) { return static_cast<uint32_t>((f / C::kStages) & 1); };
 
             ok = mbar_wait(bar_q_full, 0, abort_flag, p.status);
             if (ok) ok = wait_full(0);
@@ -484,25 +503,42 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                 for (int i = 0; i < n_qt; ++i) issue_qk(i, 0);
                 commit_to(bar_kv_empty(0));
             }
+            Pending w_v = arm(full_bar(1), full_par(1));                // V of the first tile
+            Pending w_p = arm(bar_p_half(0, 0), 0u);                    // first half of P_0
             for (int jj = 0; jj < n_tiles && ok; ++jj) {
                 const int fv = 2 * jj + 1, fk = 2 * jj + 2;             // ring slots of V_jj and K_{jj+1}
                 const bool more = jj + 1 < n_tiles;
-                ok = wait_full(fv);
-                if (ok && more) ok = wait_full(fk);
-                if (!ok) break;
+                const uint32_t par = static_cast<uint32_t>(jj & 1);
                 for (int i = 0; i < n_qt; ++i) {
-                    for (int hf = 0; hf < 2 && ok; ++hf) {
-                        ok = mbar_wait(bar_p_half(i, hf), static_cast<uint32_t>(jj & 1), abort_flag, p.status);
-                        if (!ok) break;
-                        tc_fence_after();
-                        issue_pv(i, fv % C::kStages, hf, jj == 0);
-                    }
+                    const bool last_i = i == n_qt - 1;
+                    if (i == 0) ok = await(w_v);
+                    if (ok) ok = await(w_p);
                     if (!ok) break;
-                    if (i == n_qt - 1) commit_to(bar_kv_empty(fv % C::kStages));
+                    tc_fence_after();
+                    const Pending w_h1 = arm(bar_p_half(i, 1), par);
+                    issue_pv(i, fv % C::kStages, 0, jj == 0);
+                    ok = await(w_h1);
+                    if (!ok) break;
+                    tc_fence_after();
+                    Pending w_k = {0u, 0u, true};
+                    if (more && i == 0) w_k = arm(full_bar(fk), full_par(fk));
+                    if (!more && !last_i) w_p = arm(bar_p_half(i + 1, 0), par);
+                    issue_pv(i, fv % C::kStages, 1, false);
+                    if (last_i) commit_to(bar_kv_empty(fv % C::kStages));
                     if (!more) commit_to(bar_o_done(i));
                     if (more) {
+                        ok = await(w_k);
+                        if (!ok) break;
+                        tc_fence_after();
+                        // what follows Q_i K^T: the next tile's P of this key tile, or (after the last Q tile) V and P_0 of the next
+                        if (!last_i) {
+                            w_p = arm(bar_p_half(i + 1, 0), par);
+                        } else {
+                            w_v = arm(full_bar(fv + 2), full_par(fv + 2));
+                            w_p = arm(bar_p_half(0, 0), par ^ 1u);
+                        }
                         issue_qk(i, fk % C::kStages);
-                        if (i == n_qt - 1) commit_to(bar_kv_empty(fk % C::kStages));
+                        if (last_i) commit_to(bar_kv_empty(fk % C::kStages));
                     }
                 }
             }
