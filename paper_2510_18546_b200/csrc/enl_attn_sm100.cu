@@ -40,6 +40,7 @@ constexpr int kRegsOther    = 80;
 constexpr int kProducerWarp = 8;
 constexpr int kMmaWarp      = 9;
 constexpr uint32_t kTmemCols = 512;
+constexpr int kParkSlots = 28;                // calls with up to this many mass slots park their slot sums in shared memory
 constexpr float kRescaleThreshold = 8.0f;     // log2 units: p stays below 2^8 between updates of the reference
 constexpr unsigned long long kWaitLimitNs = 1000ull * 1000ull * 1000ull;
 constexpr uint32_t kFull = 0xffffffffu;
@@ -53,7 +54,9 @@ struct Cfg {
     static constexpr int kBarOff    = (kQTiles + kStages) * kTileBytes;
     // pair merge: what the other CTA of the cluster knows about this CTA's rows, [tile][128] x (m, l, shared-slot log-sum, -)
     static constexpr int kXpeerOff  = kBarOff + 512;
-    static constexpr int kSmemBytes = kXpeerOff + kQTiles * 128 * 16 + 1024;   // + alignment slack
+    // slot log-sums of calls with at most kParkSlots slots, [tile][slot][128 rows] fp32 (what is left of the 227 KB)
+    static constexpr int kParkOff   = kXpeerOff + kQTiles * 128 * 16;
+    static constexpr int kSmemBytes = kParkOff + kQTiles * kParkSlots * 128 * 4 + 1024;   // + alignment slack
 };
 
 // ---- small PTX wrappers ------------------------------------------------------------------
@@ -569,11 +572,15 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
         const bool split_mode = p.n_splits > 1 && !pair;
         const long long grow = static_cast<long long>(ep.q_off) + t;   // global query row
         const long long rh = (split_mode ? (static_cast<long long>(it.split) * p.n_q_total + grow) : grow) * p.Hq + h;
-        float *slot_out = nullptr;                                 // where this row's slots are parked
+        // Where this row's slot log-sums are parked until the row's total is known: shared memory when the call has few
+        // slots (one store per slot end, no round trip to the L2 at the end), else the buffer that takes the result.
+        float *slot_out = nullptr;
         if (row_valid) {
             if (split_mode) { if (p.part_slot) slot_out = p.part_slot + rh * p.mass_stride; }
             else if (p.mass) slot_out = p.mass + rh * p.mass_stride;
         }
+        const bool park_smem = G + 1 <= kParkSlots;
+        float *park_row = reinterpret_cast<float *>(smem + C::kParkOff) + i * (kParkSlots * 128) + r;   // + slot * 128
         const float scale = p.scale_log2;
 
         // Pair merge: the slot in which the two splits meet is walked by both.  Split 0 writes it (adding what
@@ -593,6 +600,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
             if (cur_slot >= 0) {
                 const float v = lg2(acc) + m_ref;
                 if (cur_slot == skip_slot) bnd = v;
+                else if (park_smem) park_row[cur_slot * 128] = v;
                 else if (slot_out) slot_out[cur_slot] = v;
             }
         };
@@ -780,12 +788,24 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
             }
             __syncwarp();
         };
-        // Masses: parked log-sums -> shares of the row's total.  The warp takes its rows one after the other,
-        // lanes over the slots (coalesced), eight rows' loads in flight.  ref / extra: per row (held by the
-        // row's thread) the log-sum-exp of the whole row and, in a pair, the other split's part of the slot
-        // in which the splits meet.
+        // Masses: parked log-sums -> shares of the row's total.  ref / extra: per row (held by the row's thread) the
+        // log-sum-exp of the whole row and, in a pair, the other split's part of the slot in which the splits meet.
+        // Few slots: they were parked in shared memory.  Otherwise (the scoring pass has a thousand slots) the warp takes
+        // its rows one after the other, lanes over the slots (coalesced), eight rows' loads in flight.
         const int my_ridx = row_index(lane);
         auto finish_masses = [&](float ref_mine, float extra_mine, int first, int last) {
+            if (park_smem) {                                        // every thread converts its own row out of shared memory
+                if (my_ridx < 0) return;
+                float *slots = p.mass + static_cast<long long>(my_ridx) * p.mass_stride;
+#pragma unroll 4
+                for (int sl = first; sl <= last; ++sl) {
+                    if (sl == skip_slot) continue;
+                    float w = (ref_mine != kNegInf) ? ex2(park_row[sl * 128] - ref_mine) : 0.f;
+                    if (sl == shared_slot && ref_mine != kNegInf) w += ex2(extra_mine - ref_mine);
+                    slots[sl] = w;
+                }
+                return;
+            }
             __syncwarp();                                           // the parked values of all lanes are visible
 #pragma unroll 1
             for (int r0 = 0; r0 < 32; r0 += 8) {
@@ -852,7 +872,11 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
             } else if (split_mode) {
                 // ---- partial results for the merge kernel: O / l in fp32, the row's log-sum-exp, raw slot log-sums ----
                 if (row_valid) p.part_lse[rh] = lse;
-                if (p.part_slot) {
+                if (p.part_slot && park_smem) {
+                    if (slot_out)
+                        for (int sl = 0; sl <= G; ++sl)
+                            slot_out[sl] = (sl < first_slot || sl > last_slot) ? kNegInf : park_row[sl * 128];
+                } else if (p.part_slot) {
                     __syncwarp();
 #pragma unroll 1
                     for (int rr = 0; rr < 32; ++rr) {               // slots this split did not walk contribute nothing
@@ -935,6 +959,10 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                     w_own = (L > 0.f) ? fa / L : 0.f;
                     w_peer = (L > 0.f) ? fb / L : 0.f;
                 }
+                // each CTA writes the slots it walked against the merged log-sum-exp; the slot both walked is
+                // written by split 0, which adds the part split 1 sent.  (Before the output: the peer's accumulator is
+                // still on its way.)
+                if (ok && p.mass) finish_masses(pair_lse, pair_bnd, first_slot, last_slot);
                 if (ok && i == it.split && n_tiles > 0) {
                     // this CTA finishes the tile: its own accumulator and what the peer sent, each with its weight;
                     // thread (warp, lane) reads what thread (warp, lane) of the peer wrote
@@ -966,9 +994,6 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                         }
                     }
                 }
-                // each CTA writes the slots it walked against the merged log-sum-exp; the slot both walked is
-                // written by split 0, which adds the part split 1 sent
-                if (ok && p.mass) finish_masses(pair_lse, pair_bnd, first_slot, last_slot);
                 // what this CTA staged for its peer must have been fetched before the CTA may retire
                 if (exported) ok = mbar_wait<true>(bar_peer_ack, 0, abort_flag, p.status);
               }
