@@ -45,8 +45,11 @@ enum { ENL_DEVICE_NONE = -1 };                   /* bookkeeping-only cache: tabl
 enum { ENL_REPLACE = 0, ENL_APPEND = 1 };        /* enl_group_store modes                    */
 
 enum {                                            /* enl_attend_args_t.flags                  */
-    ENL_PLAN_ONLY = 1u                            /* validate + build the gather plan + fill  */
+    ENL_PLAN_ONLY = 1u,                           /* validate + build the gather plan + fill  */
                                                   /* sel_off_out, enqueue nothing             */
+    ENL_MASS_ONLY = 2u                            /* only group_mass / group_mass_sum are     */
+                                                  /* wanted: `out` is not written (may be     */
+                                                  /* NULL); needs group_mass                  */
 };
 
 enum {                                            /* return codes                             */
@@ -137,7 +140,21 @@ typedef struct {
                                        /*   of its selected groups' lengths                    */
     int32_t split_hint;                /* 0 = library chooses the number of KV splits,         */
                                        /*   k >= 1 = use k splits (clamped to what fits)       */
-    uint32_t flags;                    /* ENL_PLAN_ONLY                                        */
+    uint32_t flags;                    /* ENL_PLAN_ONLY, ENL_MASS_ONLY                         */
+    /* Sec. 3.3 consumes only an average of the mass over an object's tokens, the q heads and  */
+    /* the scored layers.  With group_mass_sum the call ADDS, for every object o and slot s,   */
+    /* the sum over the object's query rows and all q heads of the row's mass on s to          */
+    /* group_mass_sum[o * sum_stride + s] (one reduction inside the attention kernel, one      */
+    /* atomic add per warp, object and slot), so that the caller zeroes the array once, lets   */
+    /* the scored layers accumulate and never reads the per-row masses back:                   */
+    /* enl_cluster_assign_sums turns the sums into averages and decisions.                     */
+    float *group_mass_sum;             /* device fp32 [n_obj][sum_stride] or NULL; needs       */
+                                       /*   group_mass (which the kernel still fills)          */
+    int32_t sum_stride;                /* >= max_b(G_b) + 1                                    */
+    int32_t n_obj;                     /* objects; 0 when group_mass_sum is NULL               */
+    const int32_t *obj_off;            /* HOST [n_obj+1], ascending: object o owns query rows  */
+                                       /*   obj_off[o] .. obj_off[o+1]-1 (global over the      */
+                                       /*   batch); rows outside every span are not summed     */
 } enl_attend_args_t;
 
 /*
@@ -253,6 +270,17 @@ typedef struct {
  * layers or ENL_CLUSTER_MAX_OBJECTS objects per call), ENL_E_CUDA.
  */
 int enl_cluster_assign(const enl_cluster_args_t *args, void *cuda_stream);
+
+/*
+ * The same decision from the sums that enl_attend accumulated in group_mass_sum over the scored
+ * layers: avg[o][g] = mass_sum[o * sum_stride + g] / (rows of object o * n_q_heads * n_layers),
+ * assign as above.  mass_sum, avg [n_obj][n_groups] and assign [n_obj] are device memory, obj_off
+ * is HOST [n_obj+1] (the spans given to enl_attend).  Enqueued on the stream; allocates nothing.
+ * Errors: ENL_E_INVAL, ENL_E_LIMIT (more than ENL_CLUSTER_MAX_OBJECTS objects), ENL_E_CUDA.
+ */
+int enl_cluster_assign_sums(const float *mass_sum, int32_t sum_stride, int32_t n_groups, int32_t n_obj,
+                            const int32_t *obj_off, int32_t n_q_heads, int32_t n_layers, float threshold,
+                            float *avg, int32_t *assign, void *cuda_stream);
 
 /* ---- retrieval knapsack: what produces the select list ----------------------------------------- */
 

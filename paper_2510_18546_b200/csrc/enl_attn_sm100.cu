@@ -792,25 +792,33 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
         // log-sum-exp of the whole row and, in a pair, the other split's part of the slot in which the splits meet.
         // Few slots: they were parked in shared memory.  Otherwise (the scoring pass has a thousand slots) the warp takes
         // its rows one after the other, lanes over the slots (coalesced), eight rows' loads in flight.
+        // With mass_sum (Sec. 3.3 consumes only averages over an object's tokens and the q heads) the masses of the
+        // warp's rows that belong to one object are added up on the way, lane by slot, and leave as one atomic add per
+        // object and slot.
         const int my_ridx = row_index(lane);
+        const int my_obj = (p.mass_sum && row_valid) ? __ldg(p.row_obj + grow) : -1;
         auto finish_masses = [&](float ref_mine, float extra_mine, int first, int last) {
             if (park_smem) {                                        // every thread converts its own row out of shared memory
                 if (my_ridx < 0) return;
                 float *slots = p.mass + static_cast<long long>(my_ridx) * p.mass_stride;
+                float *sums = my_obj >= 0 ? p.mass_sum + static_cast<long long>(my_obj) * p.sum_stride : nullptr;
 #pragma unroll 4
                 for (int sl = first; sl <= last; ++sl) {
                     if (sl == skip_slot) continue;
                     float w = (ref_mine != kNegInf) ? ex2(park_row[sl * 128] - ref_mine) : 0.f;
                     if (sl == shared_slot && ref_mine != kNegInf) w += ex2(extra_mine - ref_mine);
                     slots[sl] = w;
+                    if (sums) atomicAdd(sums + sl, w);
                 }
                 return;
             }
             __syncwarp();                                           // the parked values of all lanes are visible
 #pragma unroll 1
-            for (int r0 = 0; r0 < 32; r0 += 8) {
+            for (int s0 = first + lane; s0 - lane <= last; s0 += 32) {
+                float run = 0.f;                                    // this slot's sum over the rows of the current object
+                int run_obj = -1;
 #pragma unroll 1
-                for (int s0 = first + lane; s0 - lane <= last; s0 += 32) {
+                for (int r0 = 0; r0 < 32; r0 += 8) {
                     float v[8];
                     float *dst[8];
 #pragma unroll
@@ -824,13 +832,25 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                     for (int x = 0; x < 8; ++x) {
                         const float ref = __shfl_sync(kFull, ref_mine, r0 + x);
                         const float extra = __shfl_sync(kFull, extra_mine, r0 + x);
+                        const int obj = __shfl_sync(kFull, my_obj, r0 + x);
+                        float w = 0.f;
                         if (dst[x]) {
-                            float w = (ref != kNegInf) ? ex2(v[x] - ref) : 0.f;
+                            w = (ref != kNegInf) ? ex2(v[x] - ref) : 0.f;
                             if (s0 == shared_slot && ref != kNegInf) w += ex2(extra - ref);
                             *dst[x] = w;
                         }
+                        if (p.mass_sum) {                           // warp-uniform: obj is the same in every lane
+                            if (obj != run_obj) {
+                                if (run_obj >= 0 && s0 <= last)
+                                    atomicAdd(p.mass_sum + static_cast<long long>(run_obj) * p.sum_stride + s0, run);
+                                run = 0.f;
+                                run_obj = obj;
+                            }
+                            run += w;
+                        }
                     }
                 }
+                if (run_obj >= 0 && s0 <= last) atomicAdd(p.mass_sum + static_cast<long long>(run_obj) * p.sum_stride + s0, run);
             }
         };
         // slots this CTA walked (all of them without splits)
@@ -850,7 +870,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
             if (!pair && !split_mode) {
                 // ---- the whole key stream was this CTA's: output and masses ----
                 if (p.mass) finish_masses(lse, kNegInf, 0, G);
-                if (n_tiles > 0) {
+                if (n_tiles > 0 && !p.mass_only) {
                     const float inv = (l > 0.f) ? 1.f / l : 0.f;
                     ok = mbar_wait(bar_o_done(i), 0, abort_flag, p.status);
                     if (ok) {

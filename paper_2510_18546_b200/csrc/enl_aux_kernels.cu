@@ -209,9 +209,9 @@ cudaError_t launch_page_copy(const uint8_t *src_k, const uint8_t *src_v, uint8_t
                              int n_layers, int page_bytes, cudaStream_t st)
 {
     if (n_pairs <= 0) return cudaSuccess;
-    page_copy_kernel<<<dim3(n_pairs, n_layers, 2), 256, 0, st>>>(src_k, src_v, dst_k, dst_v, src_layer_bytes,
-                                                                dst_layer_bytes, pairs, page_bytes);
-    return cudaGetLastError();
+    const cudaError_t e = launch_pdl_n(page_copy_kernel, dim3(n_pairs, n_layers, 2), dim3(256), st, src_k, src_v, dst_k, dst_v,
+                                       src_layer_bytes, dst_layer_bytes, pairs, page_bytes);
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 cudaError_t launch_page_scatter(void *kpool_layer, void *vpool_layer, const void *k, const void *v,

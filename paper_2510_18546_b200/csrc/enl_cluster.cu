@@ -85,7 +85,56 @@ __global__ void cluster_pick_kernel(const float *avg, int32_t *assign, int n_gro
     if (lane == 0) assign[obj] = (arg >= 0 && best > threshold) ? arg : -1;
 }
 
+// avg[o][g] = sum[o][g] / (rows of o * q heads * layers): the sums come out of the attention kernel itself
+struct SumParams {
+    int32_t obj_off[kMaxObjects + 1];
+    const float *sum;
+    float *avg;
+    int32_t sum_stride, n_groups, n_obj;
+    float per_row;                                     // 1 / (q heads * layers)
+};
+__global__ void cluster_scale_kernel(const __grid_constant__ SumParams p)
+{
+    const int obj = blockIdx.y;
+    const int g = blockIdx.x * blockDim.x + threadIdx.x;
+    enl::pdl_trigger();
+    enl::pdl_wait();
+    if (g >= p.n_groups) return;
+    const int rows = p.obj_off[obj + 1] - p.obj_off[obj];
+    const float inv = rows > 0 ? p.per_row / static_cast<float>(rows) : 0.f;
+    p.avg[static_cast<long long>(obj) * p.n_groups + g] = p.sum[static_cast<long long>(obj) * p.sum_stride + g] * inv;
+}
+
 }  // namespace
+
+extern "C" int enl_cluster_assign_sums(const float *mass_sum, int32_t sum_stride, int32_t n_groups, int32_t n_obj,
+                                       const int32_t *obj_off, int32_t n_q_heads, int32_t n_layers, float threshold,
+                                       float *avg, int32_t *assign, void *cuda_stream)
+{
+    if (!mass_sum || !obj_off || !avg || !assign) return ENL_E_INVAL;
+    if (n_groups < 1 || n_obj < 1 || n_q_heads < 1 || n_layers < 1 || sum_stride < n_groups) return ENL_E_INVAL;
+    if (n_obj > kMaxObjects) return ENL_E_LIMIT;
+    SumParams p;
+    if (obj_off[0] < 0) return ENL_E_INVAL;
+    for (int o = 0; o <= n_obj; ++o) {
+        if (o > 0 && obj_off[o] < obj_off[o - 1]) return ENL_E_INVAL;
+        p.obj_off[o] = obj_off[o];
+    }
+    p.sum = mass_sum;
+    p.avg = avg;
+    p.sum_stride = sum_stride;
+    p.n_groups = n_groups;
+    p.n_obj = n_obj;
+    p.per_row = 1.f / (static_cast<float>(n_q_heads) * static_cast<float>(n_layers));
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const dim3 grid((n_groups + 127) / 128, n_obj);
+    if (enl::launch_pdl(cluster_scale_kernel, grid, dim3(128), 0, st, p) != cudaSuccess) { cudaGetLastError(); return ENL_E_CUDA; }
+    if (enl::launch_pdl_n(cluster_pick_kernel, dim3((n_obj + 3) / 4), dim3(128), st, avg, assign, n_groups, n_obj, threshold) != cudaSuccess) {
+        cudaGetLastError();
+        return ENL_E_CUDA;
+    }
+    return ENL_OK;
+}
 
 extern "C" int enl_cluster_assign(const enl_cluster_args_t *a, void *cuda_stream)
 {
@@ -116,7 +165,10 @@ extern "C" int enl_cluster_assign(const enl_cluster_args_t *a, void *cuda_stream
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     const dim3 grid(a->n_obj, (a->n_groups + kGroupsPerCta - 1) / kGroupsPerCta);
     if (enl::launch_pdl(cluster_avg_kernel, grid, dim3(kWarps * 32), 0, st, p) != cudaSuccess) { cudaGetLastError(); return ENL_E_CUDA; }
-    cluster_pick_kernel<<<(a->n_obj + 3) / 4, 128, 0, st>>>(a->avg, a->assign, a->n_groups, a->n_obj, a->threshold);
-    if (cudaGetLastError() != cudaSuccess) return ENL_E_CUDA;
+    if (enl::launch_pdl_n(cluster_pick_kernel, dim3((a->n_obj + 3) / 4), dim3(128), st, a->avg, a->assign, a->n_groups,
+                          a->n_obj, a->threshold) != cudaSuccess) {
+        cudaGetLastError();
+        return ENL_E_CUDA;
+    }
     return ENL_OK;
 }

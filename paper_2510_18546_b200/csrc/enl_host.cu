@@ -89,12 +89,14 @@ struct enl_cache {
     // gather plan: host image (pinned when there is a GPU), device copy, capacities
     int32_t cap_entries = 0, cap_items = 0;
     uint8_t *plan_host = nullptr, *plan_dev = nullptr;
-    size_t off_eps = 0, off_items = 0, off_stream = 0, off_meta = 0, off_rowslots = 0, plan_bytes = 0;
+    size_t off_eps = 0, off_items = 0, off_stream = 0, off_meta = 0, off_rowslots = 0, off_rowobj = 0, plan_bytes = 0;
     cudaEvent_t plan_copied = nullptr;
     bool plan_valid = false, plan_on_device = false;
     uint64_t plan_epoch = 0;
     int32_t plan_split_hint = 0;
     bool plan_has_mass = false;
+    bool plan_direct = false;               // built for a call that wants mass sums or no output: one split, general kernel
+    std::vector<int32_t> key_obj;           // object spans the row -> object map was built from
     bool plan_decode = false;               // the plan is for the one-token decode kernel
     bool plan_pair = false;                 // two splits whose CTAs merge inside the attention kernel (cluster of two)
     bool pairs_ok = false;                  // the device can co-schedule two of the attention kernel's CTAs as a cluster
@@ -123,6 +125,7 @@ struct enl_cache {
     int32_t *h_stream() { return reinterpret_cast<int32_t *>(plan_host + off_stream); }
     int32_t *h_meta() { return reinterpret_cast<int32_t *>(plan_host + off_meta); }
     int32_t *h_rowslots() { return reinterpret_cast<int32_t *>(plan_host + off_rowslots); }
+    int32_t *h_rowobj() { return reinterpret_cast<int32_t *>(plan_host + off_rowobj); }
 };
 
 namespace {
@@ -214,7 +217,8 @@ extern "C" int enl_cache_create(const enl_cache_desc_t *desc, enl_cache_t **out)
     c->off_stream = align256(c->off_items + sizeof(Item) * c->cap_items);
     c->off_meta = align256(c->off_stream + sizeof(int32_t) * c->cap_entries);
     c->off_rowslots = align256(c->off_meta + sizeof(int32_t) * c->cap_entries);
-    c->plan_bytes = align256(c->off_rowslots + sizeof(int32_t) * d.max_q_tokens);
+    c->off_rowobj = align256(c->off_rowslots + sizeof(int32_t) * d.max_q_tokens);
+    c->plan_bytes = align256(c->off_rowobj + sizeof(int32_t) * d.max_q_tokens);
 
     if (!c->gpu) {
         c->plan_host = new (std::nothrow) uint8_t[c->plan_bytes];
@@ -432,7 +436,9 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
     if (!c || !a) return ENL_E_INVAL;
     const enl_cache_desc_t &d = c->d;
     const bool plan_only = (a->flags & ENL_PLAN_ONLY) != 0;
-    if (a->flags & ~static_cast<uint32_t>(ENL_PLAN_ONLY)) return ENL_E_INVAL;
+    const bool mass_only = (a->flags & ENL_MASS_ONLY) != 0;
+    if (a->flags & ~static_cast<uint32_t>(ENL_PLAN_ONLY | ENL_MASS_ONLY)) return ENL_E_INVAL;
+    if (mass_only && !a->group_mass) return ENL_E_INVAL;
     if (!c->gpu && !plan_only) return ENL_E_CUDA;
     if (a->layer < 0 || a->layer >= d.n_layers) return ENL_E_INVAL;
     if (a->batch < 1 || a->batch > d.max_batch) return ENL_E_INVAL;
@@ -454,13 +460,22 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
         max_slots = std::max(max_slots, ns);
     }
     if (!plan_only) {
-        if (!a->q || !a->k_new || !a->v_new || !a->out) return ENL_E_INVAL;
+        if (!a->q || !a->k_new || !a->v_new || (!a->out && !mass_only)) return ENL_E_INVAL;
         const uintptr_t al = reinterpret_cast<uintptr_t>(a->q) | reinterpret_cast<uintptr_t>(a->k_new) |
                              reinterpret_cast<uintptr_t>(a->v_new) | reinterpret_cast<uintptr_t>(a->out);
         if (al & 15) return ENL_E_INVAL;
         if (a->group_mass && (reinterpret_cast<uintptr_t>(a->group_mass) & 3)) return ENL_E_INVAL;
     }
     if (a->group_mass && a->mass_stride < max_slots + 1) return ENL_E_INVAL;
+    const bool has_sum = a->group_mass_sum != nullptr;
+    if (has_sum) {
+        if (!a->group_mass || !a->obj_off || a->n_obj < 1 || a->sum_stride < max_slots + 1) return ENL_E_INVAL;
+        if (reinterpret_cast<uintptr_t>(a->group_mass_sum) & 3) return ENL_E_INVAL;
+        if (a->obj_off[0] < 0 || a->obj_off[a->n_obj] > a->n_q) return ENL_E_INVAL;
+        for (int o = 0; o < a->n_obj; ++o)
+            if (a->obj_off[o + 1] < a->obj_off[o]) return ENL_E_INVAL;
+    }
+    const bool direct = has_sum || mass_only;       // these results leave the attention kernel itself: no KV splits
 
     // ---- select list: ids, duplicates, lengths (Sec. 3.4: a group is selected at most once) ----
     std::vector<int32_t> sel_len(a->n_sel);
@@ -493,8 +508,13 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
     cu_key.insert(cu_key.end(), cu_q, cu_q + B + 1);
     cu_key.insert(cu_key.end(), cu_new, cu_new + B + 1);
     const bool has_mass = a->group_mass != nullptr;
+    bool same_obj = !has_sum;
+    if (has_sum)
+        same_obj = c->key_obj.size() == static_cast<size_t>(a->n_obj) + 1 &&
+                   std::memcmp(c->key_obj.data(), a->obj_off, sizeof(int32_t) * (a->n_obj + 1)) == 0;
     const bool reuse = c->plan_valid && c->plan_epoch == c->epoch && c->plan_split_hint == a->split_hint &&
-                       c->plan_has_mass == has_mass && c->key_cu == cu_key && c->key_len == sel_len &&
+                       c->plan_has_mass == has_mass && c->plan_direct == direct && same_obj &&
+                       c->key_cu == cu_key && c->key_len == sel_len &&
                        c->key_sel.size() == static_cast<size_t>(a->n_sel) &&
                        (a->n_sel == 0 || std::memcmp(c->key_sel.data(), a->sel_ids, sizeof(int32_t) * a->n_sel) == 0);
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
@@ -526,7 +546,7 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
         };
         // One query token per episode: the streaming decode kernel, whose CTAs cover at most kDecodeMaxPages
         // pages each and always hand their partial results to the merge kernel.
-        bool decode = c->rep <= 8;
+        bool decode = c->rep <= 8 && !direct;
         int need = 1, fewest = 0x7fffffff;
         for (int b = 0; b < B && decode; ++b) {
             if (cu_q[b + 1] - cu_q[b] != 1) decode = false;
@@ -548,7 +568,8 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
         }
         if (!decode) {
             n_splits = 1;
-            if (a->split_hint >= 1) n_splits = std::min(a->split_hint, std::max(1, min_tiles));   // no CTA without a tile
+            if (direct) n_splits = 1;
+            else if (a->split_hint >= 1) n_splits = std::min(a->split_hint, std::max(1, min_tiles));   // no CTA without a tile
             else if (base_items < 120) n_splits = std::max(1, std::min(static_cast<int>(148 / base_items), min_tiles / 2));
             n_splits = std::min<int64_t>(n_splits, std::max<int64_t>(1, c->cap_items / base_items));
             n_splits = std::min(n_splits, kMaxSplits);
@@ -586,6 +607,15 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
             e.n_ctiles = (ne - e.stream_off) / kPagesPerTile;
             for (int r = e.q_off; r < e.q_off + e.n_q; ++r) rowslots[r] = e.n_slots;
         }
+        if (has_sum) {
+            int32_t *rowobj = c->h_rowobj();
+            std::fill(rowobj, rowobj + a->n_q, -1);
+            for (int o = 0; o < a->n_obj; ++o)
+                for (int r = a->obj_off[o]; r < a->obj_off[o + 1]; ++r) rowobj[r] = o;
+            c->key_obj.assign(a->obj_off, a->obj_off + a->n_obj + 1);
+        } else {
+            c->key_obj.clear();
+        }
         // CTAs, heaviest first (late token blocks see more new-token tiles)
         struct Work { Item it; int tiles; };
         std::vector<Work> work;
@@ -614,6 +644,7 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
         c->plan_epoch = c->epoch;
         c->plan_split_hint = a->split_hint;
         c->plan_has_mass = has_mass;
+        c->plan_direct = direct;
         c->plan_decode = decode;
         // Two splits of a head_dim-128 call are launched as clusters of two CTAs, which exchange their partial
         // results through distributed shared memory: no scratch round trip and no merge kernel.  Every CTA must
@@ -638,6 +669,8 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
                                      cudaMemcpyHostToDevice, st) == cudaSuccess)) &&
                    cudaMemcpyAsync(c->plan_dev + c->off_rowslots, c->plan_host + c->off_rowslots,
                                    sizeof(int32_t) * a->n_q, cudaMemcpyHostToDevice, st) == cudaSuccess &&
+                   (!has_sum || cudaMemcpyAsync(c->plan_dev + c->off_rowobj, c->plan_host + c->off_rowobj,
+                                                sizeof(int32_t) * a->n_q, cudaMemcpyHostToDevice, st) == cudaSuccess) &&
                    cudaEventRecord(c->plan_copied, st) == cudaSuccess;
         if (!okc) { cudaGetLastError(); c->plan_valid = false; return ENL_E_CUDA; }
         c->plan_on_device = true;
@@ -719,6 +752,10 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
     p.n_splits = c->plan_splits;
     p.pair_merge = c->plan_pair ? 1 : 0;
     p.scale_log2 = 1.4426950408889634f / sqrtf(static_cast<float>(d.head_dim));
+    p.mass_sum = a->group_mass_sum;
+    p.row_obj = has_sum ? reinterpret_cast<const int32_t *>(c->plan_dev + c->off_rowobj) : nullptr;
+    p.sum_stride = a->sum_stride;
+    p.mass_only = mass_only ? 1 : 0;
     const bool scratch_merge = p.n_splits > 1 && !c->plan_pair;
     if (scratch_merge) {
         const size_t rows = static_cast<size_t>(p.n_splits) * a->n_q * d.n_q_heads;

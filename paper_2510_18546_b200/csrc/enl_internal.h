@@ -55,6 +55,10 @@ struct AttnParams {
     int32_t n_splits;
     int32_t pair_merge;     // 1: two splits, launched as clusters of two CTAs that merge through distributed shared memory
     float   scale_log2;     // log2(e) / sqrt(D)
+    float  *mass_sum;       // fp32 [n_obj][sum_stride] or null: per object the masses summed over its rows and the q heads (added to)
+    const int32_t *row_obj; // [n_q_total]: object of every query row, -1 = none (only with mass_sum)
+    int32_t sum_stride;
+    int32_t mass_only;      // 1: the output rows are not written
 };
 
 // Decode (one query token per episode): pages of the key stream one CTA may cover, and the most splits
@@ -125,6 +129,21 @@ inline cudaError_t launch_pdl(Kernel kernel, dim3 grid, dim3 block, size_t smem,
         cfg.numAttrs = 2;
     }
     return cudaLaunchKernelEx(&cfg, kernel, prm);
+}
+// the same for kernels that take several plain arguments
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl_n(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t st, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 #endif
 

@@ -18,13 +18,13 @@ LIB_PATH = os.path.join(_HERE, "libenl.so")
 ENL_BF16 = 1
 ENL_DEVICE_NONE = -1
 ENL_REPLACE, ENL_APPEND = 0, 1
-ENL_PLAN_ONLY = 1
+ENL_PLAN_ONLY, ENL_MASS_ONLY = 1, 2
 ENL_OK, ENL_E_INVAL, ENL_E_NOGROUP, ENL_E_NOMEM, ENL_E_CUDA, ENL_E_TIMEOUT, ENL_E_LIMIT, ENL_E_EVICTED = 0, -1, -2, -3, -4, -5, -6, -8
 ENL_STATIC_MAX_SEGMENTS, ENL_STATIC_MAX_KEYS, ENL_STATIC_SCRATCH_BYTES = 255, 65536, 4 << 20
 
 EXPORTS = ("enl_cache_create", "enl_group_store", "enl_attend", "enl_cache_free", "enl_strerror",
            "enl_group_store_all_layers", "enl_group_len", "enl_cache_status", "enl_plan_inspect", "enl_attend_static", "enl_cluster_assign",
-           "enl_select_knapsack", "enl_tier_enable", "enl_group_evict", "enl_step_prepare", "enl_group_resident")
+           "enl_cluster_assign_sums", "enl_select_knapsack", "enl_tier_enable", "enl_group_evict", "enl_step_prepare", "enl_group_resident")
 
 
 class CacheDesc(ctypes.Structure):
@@ -41,7 +41,9 @@ class AttendArgs(ctypes.Structure):
                 ("n_sel", ctypes.c_int32), ("n_q", ctypes.c_int32), ("n_new", ctypes.c_int32),
                 ("q", ctypes.c_void_p), ("k_new", ctypes.c_void_p), ("v_new", ctypes.c_void_p),
                 ("out", ctypes.c_void_p), ("group_mass", ctypes.c_void_p), ("mass_stride", ctypes.c_int32),
-                ("sel_off_out", ctypes.c_void_p), ("split_hint", ctypes.c_int32), ("flags", ctypes.c_uint32)]
+                ("sel_off_out", ctypes.c_void_p), ("split_hint", ctypes.c_int32), ("flags", ctypes.c_uint32),
+                ("group_mass_sum", ctypes.c_void_p), ("sum_stride", ctypes.c_int32), ("n_obj", ctypes.c_int32),
+                ("obj_off", ctypes.c_void_p)]
 
 
 class StaticArgs(ctypes.Structure):
@@ -103,6 +105,10 @@ def lib() -> ctypes.CDLL:
         L.enl_attend_static.restype = ctypes.c_int
         L.enl_cluster_assign.argtypes = [ctypes.POINTER(ClusterArgs), ctypes.c_void_p]
         L.enl_cluster_assign.restype = ctypes.c_int
+        L.enl_cluster_assign_sums.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p,
+                                              ctypes.c_int32, ctypes.c_int32, ctypes.c_float, ctypes.c_void_p, ctypes.c_void_p,
+                                              ctypes.c_void_p]
+        L.enl_cluster_assign_sums.restype = ctypes.c_int
         L.enl_select_knapsack.argtypes = [ctypes.c_int32, ctypes.c_void_p, ctypes.c_float, ctypes.c_void_p,
                                           ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p]
         L.enl_select_knapsack.restype = ctypes.c_int
@@ -158,7 +164,7 @@ def enl_group_store(cache: int, group_id: int, layer: int, k, v, mode: int = ENL
 
 
 def enl_group_store_all_layers(cache: int, group_id: int, ks, vs, mode: int = ENL_REPLACE, stream: int = 0,
-                               n_tokens: Optional[int] = None) -> None:
+                               n_tokens: Optional[int] = None, n_layers: Optional[int] = None) -> None:
     """``ks``/``vs``: one ``[n, Hkv, D]`` bf16 CUDA tensor per layer (or None with ``n_tokens`` on a bookkeeping
     cache).  Every layer of the group is written by one launch."""
     if ks is None:
@@ -167,6 +173,8 @@ def enl_group_store_all_layers(cache: int, group_id: int, ks, vs, mode: int = EN
         n = int(ks[0].shape[0])
         if any(int(t.shape[0]) != n for t in list(ks) + list(vs)):
             raise ValueError("every layer must bring the same number of rows")
+        if n_layers is not None and (len(ks) != n_layers or len(vs) != n_layers):
+            raise ValueError("one K and one V tensor per layer of the cache")
         kp = (ctypes.c_void_p * len(ks))(*[_ptr(t) for t in ks])
         vp = (ctypes.c_void_p * len(vs))(*[_ptr(t) for t in vs])
     rc = lib().enl_group_store_all_layers(cache, group_id, n, kp, vp, mode, stream or None)
@@ -177,8 +185,10 @@ def enl_group_store_all_layers(cache: int, group_id: int, ks, vs, mode: int = EN
 def enl_attend(cache: int, layer: int, sel_ids: Sequence[int], q, k_new, v_new, out, group_mass=None,
                cu_sel=None, cu_q=None, cu_new=None, n_q: Optional[int] = None, n_new: Optional[int] = None,
                mass_stride: Optional[int] = None, want_sel_off: bool = False, split_hint: int = 0,
-               flags: int = 0, stream: int = 0):
-    """One attend call.  Returns ``sel_off`` (numpy int32 ``[n_sel + batch]``) when asked, else None."""
+               flags: int = 0, stream: int = 0, group_mass_sum=None, obj_off=None):
+    """One attend call.  Returns ``sel_off`` (numpy int32 ``[n_sel + batch]``) when asked, else None.
+    ``group_mass_sum``: fp32 CUDA tensor ``[n_obj, stride]`` the call adds per-object mass sums to, with
+    ``obj_off`` the ``n_obj + 1`` row offsets of the objects."""
     sel = _i32(sel_ids)
     cs, cq, cn = _i32(cu_sel), _i32(cu_q), _i32(cu_new)
     batch = 1 if cq is None else len(cq) - 1
@@ -195,6 +205,11 @@ def enl_attend(cache: int, layer: int, sel_ids: Sequence[int], q, k_new, v_new, 
         int(group_mass.shape[-1]) if group_mass is not None else 0)
     a.sel_off_out = _np_ptr(so)
     a.split_hint, a.flags = split_hint, flags
+    oo = _i32(obj_off)
+    a.group_mass_sum = _ptr(group_mass_sum)
+    a.sum_stride = int(group_mass_sum.shape[-1]) if group_mass_sum is not None else 0
+    a.n_obj = (len(oo) - 1) if oo is not None else 0
+    a.obj_off = _np_ptr(oo)
     rc = lib().enl_attend(cache, ctypes.byref(a), stream or None)
     if rc != ENL_OK:
         raise EnlError(rc, "enl_attend")
@@ -231,6 +246,18 @@ def enl_cluster_assign(masses: Sequence, obj_off: Sequence[int], n_groups: int, 
     rc = lib().enl_cluster_assign(ctypes.byref(a), stream or None)
     if rc != ENL_OK:
         raise EnlError(rc, "enl_cluster_assign")
+
+
+def enl_cluster_assign_sums(mass_sum, obj_off: Sequence[int], n_groups: int, n_q_heads: int, n_layers: int,
+                            threshold: float, avg, assign, stream: int = 0) -> None:
+    """``mass_sum``: fp32 CUDA tensor ``[n_obj, stride]`` that the scoring attends added to (group_mass_sum);
+    ``avg``: fp32 ``[n_obj, n_groups]``, ``assign``: int32 ``[n_obj]`` CUDA tensors (outputs)."""
+    off = _i32(obj_off)
+    rc = lib().enl_cluster_assign_sums(_ptr(mass_sum), int(mass_sum.shape[-1]), int(n_groups), len(off) - 1, _np_ptr(off),
+                                       int(n_q_heads), int(n_layers), float(threshold), _ptr(avg), _ptr(assign),
+                                       stream or None)
+    if rc != ENL_OK:
+        raise EnlError(rc, "enl_cluster_assign_sums")
 
 
 def enl_select_knapsack(prob: Sequence[float], threshold: float, mem_bytes: Sequence[int], budget_bytes: int,

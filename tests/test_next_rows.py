@@ -171,3 +171,87 @@ def test_group_append_compute_step():
         wl1 = s.host_kv[(0, 0)]
         ro_old, _ = orc.attend_slots(8, 2, 128, [wl1[0][0][:70]], [wl1[1][0][:70]], probe_q.cpu(), probe_k.cpu(), probe_v.cpu())
         assert np.abs(before.float().cpu().numpy() - ro_old).max() <= 2e-2
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("shape", ["few_slots", "many_slots", "batch"])
+def test_mass_sums_from_the_attention_kernel_match_the_oracle(shape):
+    """Sec. 3.3 consumes only the average mass over an object's tokens, the q heads and the scored layers:
+    enl_attend adds the per-object sums itself (group_mass_sum), enl_cluster_assign_sums turns them into
+    averages and decisions.  Checked against the oracle's attention + oracle.cluster_assign, over two layers."""
+    from tests.helpers import Session
+    from paper_2510_18546_b200 import synth
+    if shape == "few_slots":            # slots parked in shared memory, one thread per row converts
+        wl = synth.make_small(51, 2, 8, 2, 128, [[40, 17, 90, 33]], [[2, 0, 3]], [70], [70], name="sum_few")
+        obj_off = [0, 9, 9, 41, 70]
+    elif shape == "many_slots":         # slots parked in the mass buffer, the warp converts row by row
+        pool = [[5 + (i * 7) % 23 for i in range(40)]]
+        wl = synth.make_small(52, 2, 8, 2, 128, pool, [list(range(40))], [100], [100], name="sum_many")
+        obj_off = [3, 10, 64, 65, 97]   # rows 0-2 and 97-99 belong to no object
+    else:                               # objects of two episodes
+        wl = synth.make_small(53, 2, 8, 2, 128, [[30, 60], [5, 5, 250]], [[1, 0], [2, 0]], [40, 50], [40, 50], name="sum_batch")
+        obj_off = [0, 40, 60, 90]
+    n_obj = len(obj_off) - 1
+    with Session(wl, [0, 1]) as s:
+        cs, cq, cn = wl.cu()
+        G = int(max(len(x) for x in wl.sel_local))
+        dev = s.device
+        sums = torch.zeros(n_obj, G + 1, dtype=torch.float32, device=dev)
+        ref_masses = []
+        for li in range(2):
+            q, kn, vn = wl.new_qkv(li, dev)
+            out = torch.empty_like(q)
+            mass = torch.full((q.shape[0], wl.n_q_heads, G + 1), float("nan"), dtype=torch.float32, device=dev)
+            enl.enl_attend(s.cache, li, wl.sel_ids(), q, kn, vn, out if li == 0 else None, mass,
+                           cu_sel=cs if wl.batch > 1 else None, cu_q=cq if wl.batch > 1 else None,
+                           cu_new=cn if wl.batch > 1 else None, n_q=int(cq[-1]), n_new=int(cn[-1]),
+                           flags=0 if li == 0 else enl.ENL_MASS_ONLY, group_mass_sum=sums, obj_off=obj_off)
+            torch.cuda.synchronize()
+            assert enl.enl_cache_status(s.cache) == enl.ENL_OK
+            assert enl.enl_plan_inspect(s.cache)["n_splits"] == 1
+            rm = np.zeros((q.shape[0], wl.n_q_heads, G + 1))
+            for b in range(wl.batch):
+                ro, mo, _ = s.oracle(li, b, q[cq[b]:cq[b + 1]], kn[cn[b]:cn[b + 1]], vn[cn[b]:cn[b + 1]])
+                rm[cq[b]:cq[b + 1], :, :mo.shape[-1]] = mo
+                if li == 0:             # the output is still written without ENL_MASS_ONLY
+                    assert np.abs(out[cq[b]:cq[b + 1]].float().cpu().numpy() - ro).max() <= 2e-2
+                gm = mass[cq[b]:cq[b + 1], :, :mo.shape[-1]].cpu().numpy()
+                assert np.abs(gm - mo).max() <= 1e-3
+            ref_masses.append(rm)
+        n_groups = G                    # the new-token slot is not a group
+        avg = torch.full((n_obj, n_groups), float("nan"), dtype=torch.float32, device=dev)
+        asg = torch.full((n_obj,), -7, dtype=torch.int32, device=dev)
+        thr = 0.05
+        enl.enl_cluster_assign_sums(sums, obj_off, n_groups, wl.n_q_heads, 2, thr, avg, asg)
+        torch.cuda.synchronize()
+        ravg, rasg = orc.cluster_assign(ref_masses, obj_off, n_groups, thr)
+        assert np.abs(avg.cpu().numpy() - ravg).max() < 1e-4, np.abs(avg.cpu().numpy() - ravg).max()
+        got = asg.cpu().numpy()
+        for o in range(n_obj):
+            top = np.sort(ravg[o])[::-1]
+            if abs(top[0] - thr) > 1e-3 and (len(top) < 2 or top[0] - top[1] > 1e-3):
+                assert got[o] == rasg[o], (o, got[o], rasg[o])
+
+
+@pytest.mark.gpu
+def test_mass_only_and_sum_argument_errors():
+    from tests.helpers import Session
+    from paper_2510_18546_b200 import synth
+    wl = synth.make_small(54, 1, 8, 2, 128, [[40, 17]], [[1, 0]], [20], [20], name="sum_err")
+    with Session(wl, [0]) as s:
+        q, kn, vn = wl.new_qkv(0, s.device)
+        out = torch.empty_like(q)
+        mass = torch.zeros(20, 8, 3, dtype=torch.float32, device=s.device)
+        sums = torch.zeros(2, 3, dtype=torch.float32, device=s.device)
+        with pytest.raises(enl.EnlError) as e:      # ENL_MASS_ONLY without a mass buffer
+            enl.enl_attend(s.cache, 0, wl.sel_ids(), q, kn, vn, None, None, flags=enl.ENL_MASS_ONLY)
+        assert e.value.code == enl.ENL_E_INVAL
+        with pytest.raises(enl.EnlError) as e:      # sums without the per-row masses
+            enl.enl_attend(s.cache, 0, wl.sel_ids(), q, kn, vn, out, None, group_mass_sum=sums, obj_off=[0, 5, 20])
+        assert e.value.code == enl.ENL_E_INVAL
+        with pytest.raises(enl.EnlError) as e:      # spans beyond the query rows
+            enl.enl_attend(s.cache, 0, wl.sel_ids(), q, kn, vn, out, mass, group_mass_sum=sums, obj_off=[0, 5, 21])
+        assert e.value.code == enl.ENL_E_INVAL
+        with pytest.raises(enl.EnlError) as e:      # descending spans
+            enl.enl_attend(s.cache, 0, wl.sel_ids(), q, kn, vn, out, mass, group_mass_sum=sums, obj_off=[0, 9, 5])
+        assert e.value.code == enl.ENL_E_INVAL
