@@ -61,7 +61,8 @@ enum {                                            /* return codes               
     ENL_E_TIMEOUT  = -5,   /* a bounded wait inside a kernel expired (see enl_cache_status)    */
     ENL_E_LIMIT    = -6,   /* a size beyond the fixed maxima of enl_attend_static              */
                            /* -7 is not used                                                    */
-    ENL_E_EVICTED  = -8    /* the group's K/V is in the slow tier only (see enl_step_prepare)   */
+    ENL_E_EVICTED  = -8,   /* the group's K/V is in the slow tier only (see enl_step_prepare)   */
+    ENL_E_CORRUPT  = -9    /* enl_cache_selfcheck: a guard page of the pool has been written    */
 };
 
 typedef struct {
@@ -186,6 +187,11 @@ int32_t enl_group_len(const enl_cache_t *c, int32_t group_id, int32_t layer);
 /* Synchronises the device and returns ENL_OK, or ENL_E_TIMEOUT if any kernel of this cache
  * gave up on a bounded wait since the last call (the flag is then cleared). */
 int enl_cache_status(enl_cache_t *c);
+
+/* Synchronises the device and checks the two pages of every layer's K and V pool that no group ever owns
+ * (the all-zero page that stands for "no page" at the low end, a guard page at the high end): a kernel that
+ * wrote outside the pages it was given shows up as ENL_E_CORRUPT.  A debugging aid; ENL_OK otherwise. */
+int enl_cache_selfcheck(enl_cache_t *c);
 
 /*
  * Read-back of the gather plan built by the last enl_attend (host copy), for tests of the

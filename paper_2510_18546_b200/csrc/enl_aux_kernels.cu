@@ -11,14 +11,15 @@ namespace enl {
 namespace {
 
 // k, v: [n_tokens][Hkv][D] bf16 -> pool layer [page][Hkv][16][D]; 16-byte chunks, one per thread-iteration.
-__global__ void page_scatter_kernel(uint4 *__restrict__ kpool, uint4 *__restrict__ vpool,
-                                    const uint4 *__restrict__ k, const uint4 *__restrict__ v,
-                                    const __grid_constant__ PageRun run, int first_pos, int n_tokens,
-                                    int Hkv, int chunks_per_row)
+// The `zero_rows` rows behind the last token (the padding of the group's last page) are cleared: the attention
+// kernels give padded keys probability 0, and 0 times whatever an earlier, longer version of the group left
+// there must stay 0 (a stale non-finite value would not).
+__device__ __forceinline__ void scatter_rows(uint4 *__restrict__ kpool, uint4 *__restrict__ vpool, const uint4 *__restrict__ k,
+                                             const uint4 *__restrict__ v, const PageRun &run, int first_pos, int n_tokens,
+                                             int zero_rows, int Hkv, int chunks_per_row)
 {
-    const long long total = static_cast<long long>(n_tokens) * Hkv * chunks_per_row;
-    pdl_trigger();
-    pdl_wait();                                             // an attention kernel may still be reading these pages
+    const long long total = static_cast<long long>(n_tokens + zero_rows) * Hkv * chunks_per_row;
+    const long long n_src = static_cast<long long>(n_tokens) * Hkv * chunks_per_row;
     for (long long id = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; id < total;
          id += static_cast<long long>(gridDim.x) * blockDim.x) {
         const int ch = static_cast<int>(id % chunks_per_row);
@@ -29,36 +30,33 @@ __global__ void page_scatter_kernel(uint4 *__restrict__ kpool, uint4 *__restrict
         const int page = run.ids[pos / kPageTokens - run.first_page];
         const long long dst = ((static_cast<long long>(page) * Hkv + head) * kPageTokens + pos % kPageTokens) *
                                   chunks_per_row + ch;
-        kpool[dst] = k[id];
-        vpool[dst] = v[id];
+        const bool real = id < n_src;
+        kpool[dst] = real ? k[id] : make_uint4(0u, 0u, 0u, 0u);
+        vpool[dst] = real ? v[id] : make_uint4(0u, 0u, 0u, 0u);
     }
+}
+__global__ void page_scatter_kernel(uint4 *__restrict__ kpool, uint4 *__restrict__ vpool,
+                                    const uint4 *__restrict__ k, const uint4 *__restrict__ v,
+                                    const __grid_constant__ PageRun run, int first_pos, int n_tokens, int zero_rows,
+                                    int Hkv, int chunks_per_row)
+{
+    pdl_trigger();
+    pdl_wait();                                             // an attention kernel may still be reading these pages
+    scatter_rows(kpool, vpool, k, v, run, first_pos, n_tokens, zero_rows, Hkv, chunks_per_row);
 }
 
 // grid (blocks, layers): the same scatter for several layers of one group at once
 __global__ void page_scatter_layers_kernel(uint4 *__restrict__ kpool, uint4 *__restrict__ vpool, long long layer_chunks,
                                            const __grid_constant__ LayerSrc src, long long src_chunk_off,
                                            const __grid_constant__ PageRun run, int first_pos, int n_tokens,
-                                           int Hkv, int chunks_per_row)
+                                           int zero_rows, int Hkv, int chunks_per_row)
 {
-    const long long total = static_cast<long long>(n_tokens) * Hkv * chunks_per_row;
     const uint4 *k = static_cast<const uint4 *>(src.k[blockIdx.y]) + src_chunk_off;
     const uint4 *v = static_cast<const uint4 *>(src.v[blockIdx.y]) + src_chunk_off;
     uint4 *kp = kpool + layer_chunks * blockIdx.y, *vp = vpool + layer_chunks * blockIdx.y;
     pdl_trigger();
     pdl_wait();                                             // an attention kernel may still be reading these pages
-    for (long long id = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; id < total;
-         id += static_cast<long long>(gridDim.x) * blockDim.x) {
-        const int ch = static_cast<int>(id % chunks_per_row);
-        const long long th = id / chunks_per_row;
-        const int head = static_cast<int>(th % Hkv);
-        const int tok = static_cast<int>(th / Hkv);
-        const int pos = first_pos + tok;
-        const int page = run.ids[pos / kPageTokens - run.first_page];
-        const long long dst = ((static_cast<long long>(page) * Hkv + head) * kPageTokens + pos % kPageTokens) *
-                                  chunks_per_row + ch;
-        kp[dst] = k[id];
-        vp[dst] = v[id];
-    }
+    scatter_rows(kp, vp, k, v, run, first_pos, n_tokens, zero_rows, Hkv, chunks_per_row);
 }
 
 __device__ __forceinline__ float ex2f(float x)
@@ -215,15 +213,15 @@ cudaError_t launch_page_copy(const uint8_t *src_k, const uint8_t *src_v, uint8_t
 }
 
 cudaError_t launch_page_scatter(void *kpool_layer, void *vpool_layer, const void *k, const void *v,
-                                const PageRun &run, int first_pos, int n_tokens, int Hkv, int D,
-                                cudaStream_t st)
+                                const PageRun &run, int first_pos, int n_tokens, int zero_rows, int Hkv, int D,
+                                int n_sm, cudaStream_t st)
 {
     if (n_tokens <= 0) return cudaSuccess;
     const int cpr = D * 2 / 16;
-    const long long total = static_cast<long long>(n_tokens) * Hkv * cpr;
+    const long long total = static_cast<long long>(n_tokens + zero_rows) * Hkv * cpr;
     const int threads = 256;
     long long blocks = (total + threads - 1) / threads;
-    if (blocks > 148 * 8) blocks = 148 * 8;
+    if (blocks > n_sm * 8) blocks = n_sm * 8;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(blocks));
     cfg.blockDim = dim3(threads);
@@ -235,21 +233,21 @@ cudaError_t launch_page_scatter(void *kpool_layer, void *vpool_layer, const void
     cfg.numAttrs = 1;
     const cudaError_t e = cudaLaunchKernelEx(&cfg, page_scatter_kernel, static_cast<uint4 *>(kpool_layer),
                                              static_cast<uint4 *>(vpool_layer), static_cast<const uint4 *>(k),
-                                             static_cast<const uint4 *>(v), run, first_pos, n_tokens, Hkv, cpr);
+                                             static_cast<const uint4 *>(v), run, first_pos, n_tokens, zero_rows, Hkv, cpr);
     return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 cudaError_t launch_page_scatter_layers(void *kpool, void *vpool, size_t layer_bytes, int layer0, int n_layers,
                                        const LayerSrc &src, size_t src_off, const PageRun &run, int first_pos,
-                                       int n_tokens, int Hkv, int D, cudaStream_t st)
+                                       int n_tokens, int zero_rows, int Hkv, int D, int n_sm, cudaStream_t st)
 {
     if (n_tokens <= 0 || n_layers <= 0) return cudaSuccess;
     if (n_layers > kScatterLayers) return cudaErrorInvalidValue;
     const int cpr = D * 2 / 16;
-    const long long total = static_cast<long long>(n_tokens) * Hkv * cpr;
+    const long long total = static_cast<long long>(n_tokens + zero_rows) * Hkv * cpr;
     const int threads = 256;
     long long blocks = (total + threads - 1) / threads;
-    const long long cap = std::max(1, 148 * 8 / n_layers);
+    const long long cap = std::max(1, n_sm * 8 / n_layers);
     if (blocks > cap) blocks = cap;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(blocks), static_cast<unsigned>(n_layers));
@@ -264,7 +262,7 @@ cudaError_t launch_page_scatter_layers(void *kpool, void *vpool, size_t layer_by
     uint4 *vp = reinterpret_cast<uint4 *>(static_cast<uint8_t *>(vpool) + layer_bytes * layer0);
     const cudaError_t e = cudaLaunchKernelEx(&cfg, page_scatter_layers_kernel, kp, vp,
                                              static_cast<long long>(layer_bytes / 16), src,
-                                             static_cast<long long>(src_off / 16), run, first_pos, n_tokens, Hkv, cpr);
+                                             static_cast<long long>(src_off / 16), run, first_pos, n_tokens, zero_rows, Hkv, cpr);
     return e != cudaSuccess ? e : cudaGetLastError();
 }
 

@@ -78,6 +78,7 @@ struct enl_cache {
     enl_cache_desc_t d{};
     bool gpu = false;
     int rep = 1;
+    int n_sm = 148;                         // multiprocessors of the device (grid sizes, split counts)
     int64_t n_pages = 0;
     size_t layer_bytes = 0;                 // one layer of one pool
     uint8_t *kpool = nullptr, *vpool = nullptr;
@@ -171,6 +172,7 @@ extern "C" const char *enl_strerror(int code)
         case ENL_E_TIMEOUT: return "a bounded wait inside a kernel expired";
         case ENL_E_LIMIT: return "size beyond the fixed maxima of the entry point that allocates nothing";
         case ENL_E_EVICTED: return "the group is in the slow tier only; enl_step_prepare loads it";
+        case ENL_E_CORRUPT: return "a guard page of the pool has been written";
         default: return "unknown error";
     }
 }
@@ -199,14 +201,15 @@ extern "C" int enl_cache_create(const enl_cache_desc_t *desc, enl_cache_t **out)
     c->d = d;
     c->rep = rep;
     c->gpu = d.device >= 0;
-    // every group may waste up to one page of padding; page 0 stays the all-zero page
-    c->n_pages = (d.max_tokens + kPageTokens - 1) / kPageTokens + d.max_groups + 1;
+    // every group may waste up to one page of padding; page 0 stays the all-zero page, and one guard page that is
+    // never handed out either closes the pool (enl_cache_selfcheck)
+    c->n_pages = (d.max_tokens + kPageTokens - 1) / kPageTokens + d.max_groups + 2;
     if (c->n_pages * d.n_kv_heads * kPageTokens > 0x7fffffffll) { delete c; return ENL_E_INVAL; }
     c->layer_bytes = static_cast<size_t>(c->n_pages) * d.n_kv_heads * kPageTokens * d.head_dim * 2;
     c->groups.resize(d.max_groups);
     c->seen.assign(d.max_groups, 0);
     c->free_pages.reserve(c->n_pages);
-    for (int64_t pg = c->n_pages - 1; pg >= 1; --pg) c->free_pages.push_back(static_cast<int32_t>(pg));
+    for (int64_t pg = c->n_pages - 2; pg >= 1; --pg) c->free_pages.push_back(static_cast<int32_t>(pg));
 
     const int tpc = tokens_per_cta(c);
     c->cap_entries = static_cast<int32_t>(std::min<int64_t>(2 * c->n_pages + kPagesPerTile * (d.max_batch + 1), 0x7ffffff0));
@@ -231,6 +234,11 @@ extern "C" int enl_cache_create(const enl_cache_desc_t *desc, enl_cache_t **out)
     if (cudaGetDeviceCount(&n_dev) != cudaSuccess || d.device >= n_dev) { cudaGetLastError(); delete c; return ENL_E_CUDA; }
     DeviceGuard g(d.device);
     if (!get_encode_fn()) { delete c; return ENL_E_CUDA; }
+    if (cudaDeviceGetAttribute(&c->n_sm, cudaDevAttrMultiProcessorCount, d.device) != cudaSuccess || c->n_sm < 1) {
+        cudaGetLastError();
+        delete c;
+        return ENL_E_CUDA;
+    }
     const size_t pool_bytes = c->layer_bytes * d.n_layers;
     bool okm = cudaMalloc(&c->kpool, pool_bytes) == cudaSuccess && cudaMalloc(&c->vpool, pool_bytes) == cudaSuccess &&
                cudaMalloc(&c->plan_dev, c->plan_bytes) == cudaSuccess &&
@@ -298,6 +306,26 @@ extern "C" int enl_cache_status(enl_cache_t *c)
     return ENL_OK;
 }
 
+extern "C" int enl_cache_selfcheck(enl_cache_t *c)
+{
+    if (!c) return ENL_E_INVAL;
+    if (!c->gpu) return ENL_OK;
+    DeviceGuard g(c->d.device);
+    if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return ENL_E_CUDA; }
+    const size_t page_bytes = static_cast<size_t>(c->d.n_kv_heads) * kPageTokens * c->d.head_dim * 2;
+    std::vector<uint64_t> buf(page_bytes / 8);
+    for (int l = 0; l < c->d.n_layers; ++l)
+        for (int kv = 0; kv < 2; ++kv)
+            for (int end = 0; end < 2; ++end) {
+                const uint8_t *pool = (kv ? c->vpool : c->kpool) + c->layer_bytes * l;
+                const uint8_t *page = pool + (end ? static_cast<size_t>(c->n_pages - 1) * page_bytes : 0);
+                if (cudaMemcpy(buf.data(), page, page_bytes, cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return ENL_E_CUDA; }
+                for (uint64_t w : buf)
+                    if (w != 0) return ENL_E_CORRUPT;
+            }
+    return ENL_OK;
+}
+
 extern "C" int enl_group_store(enl_cache_t *c, int32_t group_id, int32_t layer, int32_t n_tokens, const void *k_dev,
                                const void *v_dev, int32_t mode, void *cuda_stream)
 {
@@ -348,10 +376,11 @@ extern "C" int enl_group_store(enl_cache_t *c, int32_t group_id, int32_t layer, 
         for (int i = run.first_page; i <= last_page; ++i) run.ids[i - run.first_page] = g.pages[i];
         const int end = std::min(new_len, (last_page + 1) * kPageTokens);
         const size_t src_off = static_cast<size_t>(pos - first_pos) * row_bytes;
+        const int zero_rows = end == new_len ? (kPageTokens - new_len % kPageTokens) % kPageTokens : 0;
         if (launch_page_scatter(c->kpool + c->layer_bytes * layer, c->vpool + c->layer_bytes * layer,
                                 static_cast<const uint8_t *>(k_dev) + src_off,
-                                static_cast<const uint8_t *>(v_dev) + src_off, run, pos, end - pos,
-                                c->d.n_kv_heads, c->d.head_dim, st) != cudaSuccess) {
+                                static_cast<const uint8_t *>(v_dev) + src_off, run, pos, end - pos, zero_rows,
+                                c->d.n_kv_heads, c->d.head_dim, c->n_sm, st) != cudaSuccess) {
             cudaGetLastError();
             return ENL_E_CUDA;
         }
@@ -420,8 +449,9 @@ extern "C" int enl_group_store_all_layers(enl_cache_t *c, int32_t group_id, int3
             for (int i = run.first_page; i <= last_page; ++i) run.ids[i - run.first_page] = g.pages[i];
             const int end = std::min(new_len, (last_page + 1) * kPageTokens);
             const size_t src_off = static_cast<size_t>(pos - first_pos) * row_bytes;
+            const int zero_rows = end == new_len ? (kPageTokens - new_len % kPageTokens) % kPageTokens : 0;
             if (launch_page_scatter_layers(c->kpool, c->vpool, c->layer_bytes, layer0, nl, src, src_off, run, pos,
-                                           end - pos, c->d.n_kv_heads, c->d.head_dim, st) != cudaSuccess) {
+                                           end - pos, zero_rows, c->d.n_kv_heads, c->d.head_dim, c->n_sm, st) != cudaSuccess) {
                 cudaGetLastError();
                 return ENL_E_CUDA;
             }
@@ -558,7 +588,7 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
         }
         int n_splits = 1;
         if (decode) {
-            const int slots = 148;                                                // one CTA per SM, one wave
+            const int slots = c->n_sm;                                            // one CTA per SM, one wave
             n_splits = a->split_hint >= 1 ? a->split_hint : std::max(1, slots / (B * d.n_kv_heads));
             n_splits = std::min(std::min(std::max(n_splits, need), fewest), kMaxSplits);
             while (n_splits > need && !fits(n_splits)) --n_splits;
@@ -570,7 +600,7 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
             n_splits = 1;
             if (direct) n_splits = 1;
             else if (a->split_hint >= 1) n_splits = std::min(a->split_hint, std::max(1, min_tiles));   // no CTA without a tile
-            else if (base_items < 120) n_splits = std::max(1, std::min(static_cast<int>(148 / base_items), min_tiles / 2));
+            else if (base_items * 5 < c->n_sm * 4) n_splits = std::max(1, std::min(static_cast<int>(c->n_sm / base_items), min_tiles / 2));
             n_splits = std::min<int64_t>(n_splits, std::max<int64_t>(1, c->cap_items / base_items));
             n_splits = std::min(n_splits, kMaxSplits);
             while (n_splits > 1 && !fits(n_splits)) --n_splits;

@@ -159,9 +159,10 @@ struct PageRun {
     int32_t ids[kScatterPages];   // ids[i] = page holding group positions (first_page + i)*16 ..
     int32_t first_page;           // index within the group of ids[0]
 };
+// zero_rows: rows behind the last token of the run's last page that are cleared (the group ends there)
 cudaError_t launch_page_scatter(void *kpool_layer, void *vpool_layer, const void *k, const void *v,
-                                const PageRun &run, int first_pos, int n_tokens,
-                                int Hkv, int D, cudaStream_t st);
+                                const PageRun &run, int first_pos, int n_tokens, int zero_rows,
+                                int Hkv, int D, int n_sm, cudaStream_t st);
 // The same for up to kScatterLayers layers in one launch: layer l reads k[l] + src_off, v[l] + src_off (bytes)
 // and writes the pool of layer layer0 + l.
 constexpr int kScatterLayers = 64;
@@ -171,7 +172,7 @@ struct LayerSrc {
 };
 cudaError_t launch_page_scatter_layers(void *kpool, void *vpool, size_t layer_bytes, int layer0, int n_layers,
                                        const LayerSrc &src, size_t src_off, const PageRun &run, int first_pos,
-                                       int n_tokens, int Hkv, int D, cudaStream_t st);
+                                       int n_tokens, int zero_rows, int Hkv, int D, int n_sm, cudaStream_t st);
 // Copies whole pages (all kv heads) between two pools of the page format, every layer, K and V: pairs[i] =
 // {source page, destination page}; the pools may be device memory or pinned host memory.
 cudaError_t launch_page_copy(const uint8_t *src_k, const uint8_t *src_v, uint8_t *dst_k, uint8_t *dst_v,

@@ -19,11 +19,11 @@ ENL_BF16 = 1
 ENL_DEVICE_NONE = -1
 ENL_REPLACE, ENL_APPEND = 0, 1
 ENL_PLAN_ONLY, ENL_MASS_ONLY = 1, 2
-ENL_OK, ENL_E_INVAL, ENL_E_NOGROUP, ENL_E_NOMEM, ENL_E_CUDA, ENL_E_TIMEOUT, ENL_E_LIMIT, ENL_E_EVICTED = 0, -1, -2, -3, -4, -5, -6, -8
+ENL_OK, ENL_E_INVAL, ENL_E_NOGROUP, ENL_E_NOMEM, ENL_E_CUDA, ENL_E_TIMEOUT, ENL_E_LIMIT, ENL_E_EVICTED, ENL_E_CORRUPT = 0, -1, -2, -3, -4, -5, -6, -8, -9
 ENL_STATIC_MAX_SEGMENTS, ENL_STATIC_MAX_KEYS, ENL_STATIC_SCRATCH_BYTES = 255, 65536, 4 << 20
 
 EXPORTS = ("enl_cache_create", "enl_group_store", "enl_attend", "enl_cache_free", "enl_strerror",
-           "enl_group_store_all_layers", "enl_group_len", "enl_cache_status", "enl_plan_inspect", "enl_attend_static", "enl_cluster_assign",
+           "enl_group_store_all_layers", "enl_group_len", "enl_cache_status", "enl_cache_selfcheck", "enl_plan_inspect", "enl_attend_static", "enl_cluster_assign",
            "enl_cluster_assign_sums", "enl_select_knapsack", "enl_tier_enable", "enl_group_evict", "enl_step_prepare", "enl_group_resident")
 
 
@@ -97,6 +97,8 @@ def lib() -> ctypes.CDLL:
         L.enl_group_len.restype = ctypes.c_int32
         L.enl_cache_status.argtypes = [ctypes.c_void_p]
         L.enl_cache_status.restype = ctypes.c_int
+        L.enl_cache_selfcheck.argtypes = [ctypes.c_void_p]
+        L.enl_cache_selfcheck.restype = ctypes.c_int
         L.enl_plan_inspect.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p,
                                        ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p,
                                        ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
@@ -309,6 +311,11 @@ def enl_group_len(cache: int, group_id: int, layer: int) -> int:
 
 def enl_cache_status(cache: int) -> int:
     return int(lib().enl_cache_status(cache))
+
+
+def enl_cache_selfcheck(cache: int) -> int:
+    """ENL_OK, or ENL_E_CORRUPT when a guard page of the pool is no longer all zero."""
+    return int(lib().enl_cache_selfcheck(cache))
 
 
 def enl_plan_inspect(cache: int, cap_entries: int = 1 << 16, cap_batch: int = 256):

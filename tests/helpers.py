@@ -44,8 +44,12 @@ class Session:
 
     def close(self):
         if self.cache:
-            enl.enl_cache_free(self.cache)
-            self.cache = None
+            try:
+                # the two pages no group owns (one at either end of every layer's pool) must still be all zero
+                assert enl.enl_cache_selfcheck(self.cache) == enl.ENL_OK, "a kernel wrote outside its pages"
+            finally:
+                enl.enl_cache_free(self.cache)
+                self.cache = None
 
     def __enter__(self):
         return self

@@ -271,3 +271,37 @@ def test_a_large_jump_of_the_row_maximum_is_exact(k_second, jump):
     assert status == enl.ENL_OK
     check_close(out, ro, mass, rm, what=f"jump {jump}")
     assert mass[:, :, 0].abs().max().item() < 1e-6 and (mass[:, :, 1] - 1).abs().max().item() < 1e-3
+
+
+def test_padding_left_by_a_longer_version_of_the_group_is_harmless():
+    """ENL_REPLACE to a shorter length leaves the group's last page partly used.  Whatever the longer version held
+    in the rows behind the new end (here NaN bit patterns) must not reach the result: padded keys get probability
+    0, and 0 x NaN would still be NaN inside the P V product, so the store clears those rows."""
+    wl = synth.make_small(61, 1, 8, 2, 128, [[37, 50]], [[0, 1]], [40], [40], name="stale_padding")
+    with Session(wl, [0], extra_tokens=64) as s:
+        dev = s.device
+        poison = torch.full((48, 2, 128), float("nan"), dtype=torch.bfloat16, device=dev)
+        k, v = wl.pool_kv(0, 0, dev)
+        offs = wl.pool_offsets(0)
+        for g in range(2):                                   # a longer, all-NaN version first, then the real rows
+            enl.enl_group_store(s.cache, g, 0, poison, poison)
+            enl.enl_group_store(s.cache, g, 0, k[offs[g]:offs[g + 1]], v[offs[g]:offs[g + 1]])
+        assert [enl.enl_group_len(s.cache, g, 0) for g in range(2)] == [37, 50]
+        q, kn, vn = wl.new_qkv(0, dev)
+        for split in (0, 2):                                 # the direct path and the pair merge
+            out, mass, _ = s.attend(0, q, kn, vn, split_hint=split)
+            torch.cuda.synchronize()
+            assert enl.enl_cache_status(s.cache) == enl.ENL_OK
+            ro, rm, _ = s.oracle(0, 0, q, kn, vn)
+            check_close(out, ro, mass, rm, what=f"stale padding split {split}")
+        out1, mass1, _ = s.attend(0, q[-1:], kn, vn, n_q=[1], n_new=[40])      # the one-token decode kernel
+        torch.cuda.synchronize()
+        ro1, rm1, _ = s.oracle(0, 0, q[-1:], kn, vn)
+        check_close(out1, ro1, mass1, rm1, what="stale padding decode")
+        # append into the partly used page: the rows behind the new end are cleared again
+        enl.enl_group_store(s.cache, 0, 0, poison, poison)
+        enl.enl_group_store(s.cache, 0, 0, k[offs[0]:offs[0] + 20], v[offs[0]:offs[0] + 20])
+        enl.enl_group_store(s.cache, 0, 0, k[offs[0] + 20:offs[1]], v[offs[0] + 20:offs[1]], mode=enl.ENL_APPEND)
+        out, mass, _ = s.attend(0, q, kn, vn)
+        torch.cuda.synchronize()
+        check_close(out, ro, mass, rm, what="stale padding after append")
