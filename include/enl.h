@@ -21,9 +21,12 @@
  *
  * Every device operation is enqueued on the stream the caller passes (a cudaStream_t cast to
  * void*; NULL = the legacy default stream).  No call synchronises the device except
- * enl_cache_create, enl_cache_free and enl_cache_status.  Validation happens on the host
- * before anything is enqueued: a call that returns an error has enqueued nothing and has
- * left the cache unchanged.
+ * enl_cache_create, enl_cache_free, enl_cache_status and enl_cache_selfcheck.  Validation
+ * happens on the host before anything is enqueued: a call that returns a validation error
+ * (ENL_E_INVAL, ENL_E_NOGROUP, ENL_E_NOMEM, ENL_E_LIMIT, ENL_E_EVICTED) has enqueued nothing
+ * and has left the cache unchanged.  ENL_E_CUDA (a launch or copy that the runtime refused)
+ * can come after the tables were updated and after earlier launches of the same call were
+ * enqueued: treat the cache as unusable then.
  *
  * No position encoding is applied here: cached K is stored as the caller produced it (already
  * rotated at whatever positions the caller assigned to the group), so results do not depend
@@ -87,15 +90,16 @@ typedef struct {
 int enl_cache_create(const enl_cache_desc_t *desc, enl_cache_t **out);
 
 /*
- * Sec. 3.2: write one group's K/V for one layer ("compute KV cache of each group individually"
- * and keep it), or append rows after the group's current end ("concatenate the information of
- * new objects at the end of the group"; existing rows are not touched).
+ * Sec. 3.2: write one group's K/V for one layer (every group's KV cache is computed on its
+ * own and kept), or append rows after the group's current end (newly detected objects join
+ * the end of their group; the rows already there are not touched).
  *   k_dev, v_dev : [n_tokens][n_kv_heads][head_dim] bf16, device; may be NULL only on a
  *                  bookkeeping-only cache.
  *   mode         : ENL_REPLACE sets the group's length for this layer to n_tokens;
  *                  ENL_APPEND adds n_tokens rows after the current length.
  * Pages are shared by all layers of a group, so a group's length must agree across the layers
- * that are attended (checked in enl_attend).  n_tokens = 0 is legal (an empty group).
+ * that are attended: enl_attend uses the length stored for the layer it is given.
+ * n_tokens = 0 is legal (an empty group).
  * Errors: ENL_E_INVAL, ENL_E_NOGROUP (id out of range), ENL_E_NOMEM (pool exhausted; state
  * unchanged), ENL_E_CUDA.
  */
@@ -218,8 +222,8 @@ typedef struct {
 } enl_prepare_stats_t;
 
 /*
- * Sec. 3.2: "we store all the KV cache in the slow memory and only load the selected groups into the
- * device memory", once per planning step rather than once per decoded token.
+ * Sec. 3.2: the KV cache of every group lives in slow memory and only the selected groups are brought
+ * into device memory, once per planning step rather than once per decoded token.
  * enl_tier_enable gives the cache a slow tier: a pinned host pool (same page format) for
  * host_tokens tokens summed over groups (plus one page of slack per group).  From then on a group is in
  * device memory, in the slow tier, or in both.
@@ -266,8 +270,8 @@ typedef struct {
 } enl_cluster_args_t;
 
 /*
- * Sec. 3.3 "Attention-based Memory Clustering": "if the average attention between a newly detected
- * object and an existing group exceeds a specific threshold, we cluster this object into the group";
+ * Sec. 3.3 "Attention-based Memory Clustering": a newly detected object joins an existing group when
+ * the average attention between the two exceeds a threshold, else it opens a new group;
  * the paper leaves open over what the average runs and which group wins when several exceed it: here
  * the mean over the object's token rows, q heads and scored layers of the probability mass on the
  * group, and the group with the largest mean.  An object with an empty span gets average 0.

@@ -1,6 +1,7 @@
 // Clustering reduce (paper, Sec. 3.3 "Attention-based Memory Clustering"): the average attention between a
 // newly detected object and every existing group, over the object's query tokens, all q heads and the few
-// scored layers, and the decision "join the group whose average exceeds the threshold, else open a new group".
+// scored layers, and the decision: the object joins the group whose average exceeds the threshold, else it opens
+// a new group.
 // Input is the per-group mass that enl_attend returns for the scoring pass; this is the reduction that
 // consumes it.  Bandwidth-bound: every mass value is read once, coalesced along the group axis.
 #include <cuda_runtime.h>

@@ -72,6 +72,7 @@ class EnlError(RuntimeError):
 
 
 _lib = None
+_n_layers = {}          # cache handle -> layer count (the all-layers store takes one pointer per layer)
 
 
 def lib() -> ctypes.CDLL:
@@ -153,6 +154,7 @@ def enl_cache_create(n_layers: int, n_q_heads: int, n_kv_heads: int, head_dim: i
     rc = lib().enl_cache_create(ctypes.byref(d), ctypes.byref(h))
     if rc != ENL_OK:
         raise EnlError(rc, "enl_cache_create")
+    _n_layers[int(h.value)] = int(n_layers)
     return h.value
 
 
@@ -175,6 +177,7 @@ def enl_group_store_all_layers(cache: int, group_id: int, ks, vs, mode: int = EN
         n = int(ks[0].shape[0])
         if any(int(t.shape[0]) != n for t in list(ks) + list(vs)):
             raise ValueError("every layer must bring the same number of rows")
+        n_layers = _n_layers.get(int(cache), n_layers)
         if n_layers is not None and (len(ks) != n_layers or len(vs) != n_layers):
             raise ValueError("one K and one V tensor per layer of the cache")
         kp = (ctypes.c_void_p * len(ks))(*[_ptr(t) for t in ks])
@@ -302,6 +305,7 @@ def enl_group_resident(cache: int, group_id: int) -> int:
 
 
 def enl_cache_free(cache: int) -> None:
+    _n_layers.pop(int(cache), None)
     lib().enl_cache_free(cache)
 
 
