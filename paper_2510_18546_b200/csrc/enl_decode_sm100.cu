@@ -7,14 +7,17 @@
 // head -- partial output normalised by the range's own sum, the range's log2-sum-exp and a per-slot
 // log2-sum-exp -- which the split merge kernel turns into the output row and the group masses.
 //
-// Every K and V page is read from HBM exactly once: each of the CTA's 12 warps owns a contiguous run of
-// the CTA's pages and a private ring of TMA stages (one page of one head = 16 rows x D bf16, 128-byte
-// swizzle) fed by its lane 0 in the order K0 V0 K1 V1 ...  Per page, all in registers:
+// Every K and V page is read from HBM exactly once.  The CTA's 12 warps take its pages one at a time from a
+// shared counter (a warp that is served faster by the memory system simply takes more pages: with fixed runs
+// the first warp finished 6-7 us before the last); each warp has a private pair of TMA stages (one page of one
+// head = 16 rows x D bf16, 128-byte swizzle) fed by its lane 0: K and V of the page it works on, refilled with
+// the page it took next as soon as they are read.  Per page, all in registers:
 //   S = Q K^T      mma.sync, A = the rep query rows padded to 16, B = the K page (ldmatrix)
 //   p = exp2(S-m)  running maximum per head kept by the warp, O and the sums rescaled when it grows
 //   O += P V       mma.sync, A = P straight from the S accumulators, B = the V page (ldmatrix.trans)
-// A page belongs to one slot (a selected group, or the new tokens), so the slot sums are running sums
-// that are parked, as log2 values, whenever the slot changes.  No CTA barrier inside the stream.
+// A page belongs to one slot (a selected group, or the new tokens) and a warp's pages come in stream order, so
+// its slot sums are running sums that are parked (slot id + log2 value, in a list of the CTA) whenever the slot
+// changes.  No CTA barrier inside the stream.
 // At the end the warps are merged through shared memory; with several splits the CTA that finishes
 // last for its (episode, kv head) merges the splits' partial results (a counter per pair, reset by
 // that CTA), so a decode step is one launch.
@@ -32,7 +35,7 @@ constexpr int kWarps   = 12;                              // one CTA per SM; 384
 constexpr int kThreads = kWarps * 32;
 constexpr int kStages  = 2;                               // TMA stages per warp: K and V of one page; 96 KB in flight per SM (D = 128)
 constexpr int kMaxRep  = 8;                               // q heads per kv head (rows 8..15 of the MMA stay zero)
-constexpr int kMaxRun  = kDecodeMaxPages / kWarps + 1;    // pages one warp may own
+constexpr int kMaxEnt  = kDecodeMaxPages + kWarps;        // parked slot sums of a CTA: at most one per page and one more per warp
 constexpr float kRescaleThreshold = 8.0f;                 // log2 units
 constexpr unsigned long long kWaitLimitNs = 1000ull * 1000ull * 1000ull;
 
@@ -159,17 +162,19 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 
 constexpr float kNegInf = -__builtin_huge_valf();
 
-// Shared memory: [ring: warp][stage][D*32 B] | per-warp slot log-sums | per-warp (m, l) | split weights | barriers
+// Shared memory: [ring: warp][stage][D*32 B] | parked slot sums | the CTA's page list | slot table | per-warp (m, l) | split weights | barriers
 template <int D>
 struct DecCfg {
     static constexpr int kStageBytes = D * kPageTokens * 2;            // one page of one head: 4 KB (D=128) / 2 KB
     static constexpr int kRingBytes  = kWarps * kStages * kStageBytes;
-    static constexpr int kWslotOff   = kRingBytes;                     // [warp][kMaxRun + 1][kMaxRep] float
-    static constexpr int kWslotBytes = kWarps * (kMaxRun + 1) * kMaxRep * 4;
-    static constexpr int kCslotOff   = kWslotOff + kWslotBytes;        // [kDecodeMaxPages + 1][kMaxRep] float
-    static constexpr int kCslotBytes = (kDecodeMaxPages + 1) * kMaxRep * 4;
+    static constexpr int kEntOff     = kRingBytes;                     // [kMaxEnt][kMaxRep] float, then [kMaxEnt] slot ids
+    static constexpr int kEntBytes   = kMaxEnt * (kMaxRep + 1) * 4;
+    static constexpr int kListOff    = kEntOff + kEntBytes;            // [kDecodeMaxPages] (page id, slot << 8 | valid keys)
+    static constexpr int kListBytes  = kDecodeMaxPages * 8;
+    static constexpr int kCslotOff   = kListOff + kListBytes;          // [kDecodeMaxPages + 1][kMaxRep] x (max, sum)
+    static constexpr int kCslotBytes = (kDecodeMaxPages + 1) * kMaxRep * 8;
     static constexpr int kMiscOff    = kCslotOff + kCslotBytes;
-    // wm[warp][rep], wl[warp][rep], wfirst[warp], wcnt[warp], cm[rep], cl[rep], weights[rep][kMaxSplits], flags[4]
+    // wm[warp][rep], wl[warp][rep], counters[2 * kWarps], cm[rep], cl[rep], weights[rep][kMaxSplits], flags[4]
     static constexpr int kMiscBytes  = (2 * kWarps * kMaxRep + 2 * kWarps + 2 * kMaxRep + kMaxRep * kMaxSplits + 4) * 4;
     static constexpr int kBarOff     = (kMiscOff + kMiscBytes + 15) & ~15;
     static constexpr int kSmemBytes  = kBarOff + kWarps * kStages * 8 + 1024;   // + alignment slack
@@ -189,13 +194,15 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, tq = lane & 3;               // MMA row group and thread-in-group
-    float *wslot = reinterpret_cast<float *>(smem + C::kWslotOff);
-    float *cslot = reinterpret_cast<float *>(smem + C::kCslotOff);
+    float *ent_val = reinterpret_cast<float *>(smem + C::kEntOff);            // [kMaxEnt][kMaxRep]: parked log2 slot sums
+    int *ent_slot = reinterpret_cast<int *>(ent_val + kMaxEnt * kMaxRep);     // [kMaxEnt]: their slots
+    int2 *pg_list = reinterpret_cast<int2 *>(smem + C::kListOff);             // the CTA's pages in stream order
+    int *cmax = reinterpret_cast<int *>(smem + C::kCslotOff);                 // [slot][kMaxRep]: maximum (ordered-int code)
+    float *cslot = reinterpret_cast<float *>(cmax + (kDecodeMaxPages + 1) * kMaxRep);   // [slot][kMaxRep]: sum, then log2-sum
     float *wm = reinterpret_cast<float *>(smem + C::kMiscOff);                // [warp][kMaxRep]
     float *wl = wm + kWarps * kMaxRep;
-    int *wfirst = reinterpret_cast<int *>(wl + kWarps * kMaxRep);             // first slot of the warp's run
-    int *wcnt = wfirst + kWarps;                                              // slots the warp parked
-    float *cm = reinterpret_cast<float *>(wcnt + kWarps);                     // CTA (later: merged) log2-sum-exp reference
+    int *ctrs = reinterpret_cast<int *>(wl + kWarps * kMaxRep);               // [0] next page to hand out, [1] parked entries
+    float *cm = reinterpret_cast<float *>(ctrs + 2 * kWarps);                 // CTA (later: merged) log2-sum-exp reference
     float *cl = cm + kMaxRep;
     float *weights = cl + kMaxRep;                                            // [kMaxRep][kMaxSplits]
     volatile int *flags = reinterpret_cast<volatile int *>(weights + kMaxRep * kMaxSplits);   // [0] abort, [1] last
@@ -226,9 +233,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
     const int pg_beg = static_cast<int>(static_cast<long long>(total) * it.split / p.n_splits);
     const int pg_end = static_cast<int>(static_cast<long long>(total) * (it.split + 1) / p.n_splits);
     const int n_cta = pg_end - pg_beg;                                        // <= kDecodeMaxPages (host guarantees)
-    // this warp's run of pages, CTA-relative [w_beg, w_end)
-    const int w_beg = n_cta * warp / kWarps, w_end = n_cta * (warp + 1) / kWarps;
-    const int n_w = w_end - w_beg;
     const int G = ep.n_slots;
 
     auto entry_meta = [&](int e) -> int {                                     // slot << 8 | valid keys
@@ -237,7 +241,21 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
         return (G << 8) | min(kPageTokens, ep.n_new - i * kPageTokens);
     };
 
-    if (threadIdx.x == 0) { flags[0] = 0; flags[1] = 0; }
+    if (threadIdx.x == 0) { flags[0] = 0; flags[1] = 0; ctrs[0] = kWarps; ctrs[1] = 0; }
+    // the CTA's page list (page id, slot << 8 | valid keys): one coalesced load up front, so that no global load
+    // sits between a stage becoming free and its refill
+    for (int i = threadIdx.x; i < n_cta; i += kThreads) {
+        const int e = pg_beg + i;
+        int2 w;
+        if (e < n_cached) {
+            w.x = __ldg(p.stream_page + ep.stream_off + e);
+            w.y = __ldg(p.stream_meta + ep.stream_off + e);
+        } else {
+            w.x = -1 - (e - n_cached);                                       // new-token page, counted from the end
+            w.y = entry_meta(e);
+        }
+        pg_list[i] = w;
+    }
     if (lane == 0) {
         for (int s = 0; s < kStages; ++s) mbar_init(bar_full(s), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -246,26 +264,12 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
     __syncthreads();
     pdl_trigger();
 
-    // lane j keeps the page id and the meta word of entry j of this warp's run (n_w <= 32): one coalesced
-    // load up front, so that no global load sits between a stage becoming free and its refill
-    int my_page = 0, my_meta = 0;
-    if (lane < n_w) {
-        const int e = pg_beg + w_beg + lane;
-        if (e < n_cached) {
-            my_page = __ldg(p.stream_page + ep.stream_off + e);
-            my_meta = __ldg(p.stream_meta + ep.stream_off + e);
-        } else {
-            my_page = -1 - (e - n_cached);                                   // new-token page, counted from the end
-            my_meta = entry_meta(e);
-        }
-    }
     // so far only shared memory and the gather plan were touched; the caller's tensors and the pool come next
     pdl_wait();
     const uint64_t pol = policy_evict_first();
-    // load i of this warp: K page i/2 (i even) or V page i/2 (i odd); `page` as kept by lane i/2
-    auto issue = [&](int i, int page) {
-        const int st = i % kStages;
-        const bool is_v = i & 1;
+    // K (stage 0) or V (stage 1) of one page into this warp's ring
+    auto issue = [&](bool is_v, int page) {
+        const int st = is_v ? 1 : 0;
         const uint32_t full = bar_full(st), dst = stage_addr(st);
         mbar_expect_tx(full, static_cast<uint32_t>(C::kStageBytes));
         if (page >= 0) {
@@ -281,12 +285,19 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
                 tma_load_3d(dst + hf * (kPageTokens * 128), tm, hf * 64, it.kvh, krow, full, pol);
         }
     };
-    const int n_loads = 2 * n_w;
-    int issued = 0;
-    for (; issued < min(kStages, n_loads); ++issued) {
-        const int pg = __shfl_sync(0xffffffffu, my_page, issued >> 1);
-        if (lane == 0) issue(issued, pg);
+    // the next page of the CTA that nobody has taken yet (CTA-relative index; >= n_cta: none left)
+    auto claim = [&]() -> int {
+        int v = 0;
+        if (lane == 0) v = atomicAdd(&ctrs[0], 1);
+        return __shfl_sync(0xffffffffu, v, 0);
+    };
+    int cur = warp;                                                          // the first round is handed out statically
+    if (cur < n_cta && lane == 0) {
+        const int pg = pg_list[cur].x;
+        issue(false, pg);
+        issue(true, pg);
     }
+    int nxt = claim();
 
     // the query rows of this kv head as the A operand of S = Q K^T (rows >= rep stay zero)
     uint32_t qa[D / 16][2];
@@ -305,17 +316,15 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
                  "l"(p.mass), "r"(p.n_q_total), "r"(p.mass_stride), "r"(p.slot_stride), "r"(p.n_splits), "r"(p.Hq));
     const float scale = p.scale_log2;
     bool ok = true;
-    int consumed = 0;                                                        // loads consumed by this warp
+    int n_done = 0;                                                          // pages this warp has worked through
 
-    // called by the whole warp after it has read stage (consumed % kStages) for the last time
-    auto release_and_refill = [&]() {
-        const int pg = __shfl_sync(0xffffffffu, my_page, (issued >> 1) & 31);   // also orders the warp's reads
-        if (lane == 0 && issued < n_loads) {
+    // called by the whole warp after it has read the K or the V stage for the last time: the page taken next
+    auto refill = [&](bool is_v) {
+        __syncwarp();                                                        // orders the warp's reads before the copy
+        if (lane == 0 && nxt < n_cta) {
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            issue(issued, pg);
+            issue(is_v, pg_list[nxt].x);
         }
-        if (issued < n_loads) ++issued;
-        ++consumed;
     };
 
     float o[kNB][2];
@@ -324,26 +333,25 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
     float z0 = 0.f, z1 = 0.f;               // accumulators of the unused MMA rows 8..15
     float m = kNegInf;                      // running reference maximum of row g (same in the four lanes of a quad)
     float lsum = 0.f, acc = 0.f;            // lane-local parts of the row sum and of the current slot's sum
-    int cur_slot = -1, n_parked = 0;
-    const int slot_first_w = __shfl_sync(0xffffffffu, my_meta, 0) >> 8;
-    float *my_wslot = wslot + warp * (kMaxRun + 1) * kMaxRep;
-    auto park = [&]() {                      // the slot that ends: log2 of its sum, absolute
+    int cur_slot = -1;
+    auto park = [&]() {                      // the slot that ends: its id and the log2 of its sum (absolute) join the CTA's list
         float a = acc;
         a += __shfl_xor_sync(0xffffffffu, a, 1);
         a += __shfl_xor_sync(0xffffffffu, a, 2);
         if (cur_slot >= 0) {
-            if (tq == 0 && g < kMaxRep) my_wslot[n_parked * kMaxRep + g] = (a > 0.f) ? lg2(a) + m : kNegInf;
-            ++n_parked;
+            int e = 0;
+            if (lane == 0) { e = atomicAdd(&ctrs[1], 1); ent_slot[e] = cur_slot; }
+            e = __shfl_sync(0xffffffffu, e, 0);
+            if (tq == 0 && g < kMaxRep) ent_val[e * kMaxRep + g] = (a > 0.f) ? lg2(a) + m : kNegInf;
         }
         acc = 0.f;
     };
 
-    for (int i = 0; i < n_w && ok; ++i) {
+    for (; cur < n_cta && ok; ++n_done) {
         // ---- S = Q K^T ----
-        int st = consumed % kStages;
-        ok = mbar_wait(bar_full(st), static_cast<uint32_t>((consumed / kStages) & 1), abort_flag, p.status);
+        ok = mbar_wait(bar_full(0), static_cast<uint32_t>(n_done & 1), abort_flag, p.status);
         if (!ok) break;
-        uint32_t base = stage_addr(st);
+        uint32_t base = stage_addr(0);
         float c[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
 #pragma unroll
         for (int nb = 0; nb < 2; ++nb) {
@@ -358,13 +366,13 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
                 mma_bf16(c[nb][0], c[nb][1], z0, z1, qa[2 * kq + 1][0], qa[2 * kq + 1][1], b[2], b[3]);
             }
         }
-        const int meta = __shfl_sync(0xffffffffu, my_meta, i);
+        const int meta = pg_list[cur].y;
         const int nv = meta & 0xff, slot = meta >> 8;
         const float s0 = (2 * tq < nv) ? c[0][0] * scale : kNegInf;
         const float s1 = (2 * tq + 1 < nv) ? c[0][1] * scale : kNegInf;
         const float s2 = (8 + 2 * tq < nv) ? c[1][0] * scale : kNegInf;
         const float s3 = (8 + 2 * tq + 1 < nv) ? c[1][1] * scale : kNegInf;
-        release_and_refill();
+        refill(false);
 
         // ---- p = exp2(S - m), sums ----
         float mx = fmaxf(fmaxf(s0, s1), fmaxf(s2, s3));
@@ -392,10 +400,9 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
         const uint32_t a0 = pack_bf16(p0, p1), a2 = pack_bf16(p2, p3);
 
         // ---- O += P V ----
-        st = consumed % kStages;
-        ok = mbar_wait(bar_full(st), static_cast<uint32_t>((consumed / kStages) & 1), abort_flag, p.status);
+        ok = mbar_wait(bar_full(1), static_cast<uint32_t>(n_done & 1), abort_flag, p.status);
         if (!ok) break;
-        base = stage_addr(st);
+        base = stage_addr(1);
         const int row = ((lane >> 3) & 1) * 8 + (lane & 7);                  // token addressed by this lane
 #pragma unroll
         for (int nq = 0; nq < kNB / 2; ++nq) {                               // two 8-channel n-blocks per ldmatrix
@@ -406,22 +413,28 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
             mma_bf16(o[2 * nq][0], o[2 * nq][1], z0, z1, a0, a2, b[0], b[1]);
             mma_bf16(o[2 * nq + 1][0], o[2 * nq + 1][1], z0, z1, a0, a2, b[2], b[3]);
         }
-        release_and_refill();
+        refill(true);
+        cur = nxt;
+        if (cur < n_cta) nxt = claim();
     }
     park();
 
-    // error path only: let this warp's copies in flight land before the CTA retires
-    if (!ok) {
-        for (int f = consumed; f < issued; ++f) {
-            const unsigned long long t0 = global_ns();
-            while (!mbar_try_wait(bar_full(f % kStages), static_cast<uint32_t>((f / kStages) & 1)) &&
-                   global_ns() - t0 < 2000000ull) { }
-        }
+    // error path only: give this warp's copies in flight (at most two pages) time to land before the CTA retires
+    if (!ok && warp < n_cta) {
+        const unsigned long long t0 = global_ns();
+        while (global_ns() - t0 < 50000ull) { }
     }
     lsum += __shfl_xor_sync(0xffffffffu, lsum, 1);
     lsum += __shfl_xor_sync(0xffffffffu, lsum, 2);
     if (tq == 0) { wm[warp * kMaxRep + g] = m; wl[warp * kMaxRep + g] = lsum; }
-    if (lane == 0) { wfirst[warp] = slot_first_w; wcnt[warp] = n_parked; }
+    // slots the CTA's range touched, and their table cleared for the merge of the parked sums
+    int slot_first = 0, n_local = 0;
+    if (n_cta > 0) {
+        slot_first = pg_list[0].y >> 8;
+        n_local = (pg_list[n_cta - 1].y >> 8) - slot_first + 1;
+    }
+    constexpr int kCodeNegInf = static_cast<int>(0x80000000u);               // below the code of every finite value
+    for (int idx = threadIdx.x; idx < n_local * kMaxRep; idx += kThreads) { cmax[idx] = kCodeNegInf; cslot[idx] = 0.f; }
     __syncthreads();                                                         // every stage consumed: the ring is free
     if (*abort_flag) return;
 
@@ -448,28 +461,28 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
         cm[h] = (Lh > 0.f) ? M + lg2(Lh) : kNegInf;                          // log2-sum-exp of the CTA's range
         cl[h] = (Lh > 0.f) ? rcp(Lh) : 0.f;
     }
-    int slot_first = 0x7fffffff, slot_end = 0;                                // slots the CTA's range touched
-#pragma unroll 1
-    for (int w = 0; w < kWarps; ++w)
-        if (wcnt[w] > 0) { slot_first = min(slot_first, wfirst[w]); slot_end = max(slot_end, wfirst[w] + wcnt[w]); }
-    const int n_local = (slot_end > 0) ? slot_end - slot_first : 0;
-    if (n_local == 0) slot_first = 0;
+    // parked sums -> one log2-sum per (slot, head): maximum first (an order-preserving integer code of the float,
+    // so that an integer atomic maximum serves), then the sum of exp2(value - maximum)
+    const int n_ent = ctrs[1];
+    auto code = [](float f) { const int i = __float_as_int(f); return i >= 0 ? i : i ^ 0x7fffffff; };
+    auto decode_code = [](int i) { return __int_as_float(i >= 0 ? i : i ^ 0x7fffffff); };
+    for (int idx = threadIdx.x; idx < n_ent * rep; idx += kThreads) {
+        const int e = idx / rep, h = idx % rep;
+        const float v = ent_val[e * kMaxRep + h];
+        if (v != kNegInf) atomicMax(&cmax[(ent_slot[e] - slot_first) * kMaxRep + h], code(v));
+    }
+    __syncthreads();
+    for (int idx = threadIdx.x; idx < n_ent * rep; idx += kThreads) {
+        const int e = idx / rep, h = idx % rep;
+        const float v = ent_val[e * kMaxRep + h];
+        const int at = (ent_slot[e] - slot_first) * kMaxRep + h;
+        if (v != kNegInf) atomicAdd(&cslot[at], ex2(v - decode_code(cmax[at])));
+    }
+    __syncthreads();
     for (int idx = threadIdx.x; idx < n_local * rep; idx += kThreads) {
-        const int sl = idx / rep, h = idx % rep, s = slot_first + sl;
-        float mxv = kNegInf;
-#pragma unroll 1
-        for (int w = 0; w < kWarps; ++w) {
-            const int j = s - wfirst[w];
-            if (j >= 0 && j < wcnt[w]) mxv = fmaxf(mxv, wslot[(w * (kMaxRun + 1) + j) * kMaxRep + h]);
-        }
-        float sum = 0.f;
-        if (mxv != kNegInf)
-#pragma unroll 1
-            for (int w = 0; w < kWarps; ++w) {
-                const int j = s - wfirst[w];
-                if (j >= 0 && j < wcnt[w]) sum += ex2(wslot[(w * (kMaxRun + 1) + j) * kMaxRep + h] - mxv);
-            }
-        cslot[sl * kMaxRep + h] = (mxv != kNegInf) ? mxv + lg2(sum) : kNegInf;
+        const int at = (idx / rep) * kMaxRep + idx % rep;
+        const float sum = cslot[at];
+        cslot[at] = (sum > 0.f) ? decode_code(cmax[at]) + lg2(sum) : kNegInf;
     }
     __syncthreads();
 
