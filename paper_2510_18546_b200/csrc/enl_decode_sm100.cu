@@ -36,6 +36,7 @@ constexpr int kThreads = kWarps * 32;
 constexpr int kStages  = 2;                               // TMA stages per warp: K and V of one page; 96 KB in flight per SM (D = 128)
 constexpr int kMaxRep  = 8;                               // q heads per kv head (rows 8..15 of the MMA stay zero)
 constexpr int kMaxEnt  = kDecodeMaxPages + kWarps;        // parked slot sums of a CTA: at most one per page and one more per warp
+constexpr int kPrefetchPages = 48;                        // pages per CTA asked into the L2 before the previous kernel has ended
 constexpr float kRescaleThreshold = 8.0f;                 // log2 units
 constexpr unsigned long long kWaitLimitNs = 1000ull * 1000ull * 1000ull;
 
@@ -115,6 +116,12 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *tm,
     asm volatile(
         "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4}], [%5], %6;"
         ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(z), "r"(bar), "l"(pol) : "memory");
+}
+// Brings a box into the L2 without a destination in the SM: it observes nothing, so it may run before the wait for
+// the previous kernel of the stream (the L2 is the point of coherence: a later write to those lines updates them).
+__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap *tm, int x, int y)
+{
+    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(tm), "r"(x), "r"(y) : "memory");
 }
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4])
 {
@@ -263,6 +270,18 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
     }
     __syncthreads();
     pdl_trigger();
+    // While the previous kernel of the stream drains (its CTAs merge their warps and splits for several microseconds
+    // after their streams have ended, and HBM idles meanwhile), ask the first pages of this CTA's range into the L2:
+    // the stream below then starts on hits.
+    {
+        const int n_pf = min(n_cta, kPrefetchPages);
+        for (int i = threadIdx.x; i < n_pf * 2 * kHalves; i += kThreads) {
+            const int pg = pg_list[i / (2 * kHalves)].x;
+            const int r = i % (2 * kHalves);
+            if (pg >= 0)
+                tma_prefetch_2d(r >= kHalves ? &p.tm_vpool : &p.tm_kpool, (r % kHalves) * 64, (pg * p.Hkv + it.kvh) * kPageTokens);
+        }
+    }
 
     // so far only shared memory and the gather plan were touched; the caller's tensors and the pool come next
     pdl_wait();
@@ -445,21 +464,21 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
         for (int nb = 0; nb < kNB; ++nb)
             *reinterpret_cast<float2 *>(obuf + (warp * kMaxRep + g) * D + nb * 8 + 2 * tq) = make_float2(o[nb][0], o[nb][1]);
     }
-    if (threadIdx.x < rep) {
-        const int h = threadIdx.x;
-        float M = kNegInf;
-#pragma unroll 1
-        for (int w = 0; w < kWarps; ++w) M = fmaxf(M, wm[w * kMaxRep + h]);
-        float Lh = 0.f;
-#pragma unroll 1
-        for (int w = 0; w < kWarps; ++w) {
-            const float mw = wm[w * kMaxRep + h];
-            const float f = (mw == kNegInf) ? 0.f : ex2(mw - M);
-            Lh += wl[w * kMaxRep + h] * f;
-            weights[h * kMaxSplits + w] = f;                                 // warp weights, reused below
+    if (warp < rep) {                                                        // warp h takes head h: lane w holds warp w's (m, l)
+        const int h = warp;
+        const float mw = lane < kWarps ? wm[lane * kMaxRep + h] : kNegInf;
+        float M = mw;
+#pragma unroll
+        for (int of = 16; of > 0; of >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, of));
+        const float f = (mw == kNegInf) ? 0.f : ex2(mw - M);
+        float Lh = lane < kWarps ? wl[lane * kMaxRep + h] * f : 0.f;
+#pragma unroll
+        for (int of = 16; of > 0; of >>= 1) Lh += __shfl_xor_sync(0xffffffffu, Lh, of);
+        if (lane < kWarps) weights[h * kMaxSplits + lane] = f;               // warp weights, reused below
+        if (lane == 0) {
+            cm[h] = (Lh > 0.f) ? M + lg2(Lh) : kNegInf;                      // log2-sum-exp of the CTA's range
+            cl[h] = (Lh > 0.f) ? rcp(Lh) : 0.f;
         }
-        cm[h] = (Lh > 0.f) ? M + lg2(Lh) : kNegInf;                          // log2-sum-exp of the CTA's range
-        cl[h] = (Lh > 0.f) ? rcp(Lh) : 0.f;
     }
     // parked sums -> one log2-sum per (slot, head): maximum first (an order-preserving integer code of the float,
     // so that an integer atomic maximum serves), then the sum of exp2(value - maximum)
@@ -493,11 +512,13 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
     for (int ff = threadIdx.x; ff < n_f4; ff += kThreads) {
         const int h = ff / (D / 4);
         float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 1
+        float4 v[kWarps];
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) v[w] = *reinterpret_cast<const float4 *>(obuf + w * kMaxRep * D + ff * 4);
+#pragma unroll
         for (int w = 0; w < kWarps; ++w) {
             const float f = weights[h * kMaxSplits + w];
-            const float4 v = *reinterpret_cast<const float4 *>(obuf + w * kMaxRep * D + ff * 4);
-            a.x += f * v.x; a.y += f * v.y; a.z += f * v.z; a.w += f * v.w;
+            a.x += f * v[w].x; a.y += f * v[w].y; a.z += f * v[w].z; a.w += f * v[w].w;
         }
         const float inv = cl[h];
         a.x *= inv; a.y *= inv; a.z *= inv; a.w *= inv;
@@ -562,10 +583,29 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
         const int k = grp + j * groups;
         pv[j] = (active && k < p.n_splits) ? __ldcg(po4 + k * po_stride4) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
+    // slot range of split k = warp + lane * kWarps, from the plan (the same arithmetic as that split's CTA used)
     int2 my_rng = make_int2(0, 0);
     {
         const int k = warp + lane * kWarps;
-        if (k < p.n_splits) my_rng = __ldcg(p.part_rng + (k * static_cast<int>(gridDim.z) + it.ep) * p.Hkv + it.kvh);
+        if (k < p.n_splits) {
+            const int b0 = static_cast<int>(static_cast<long long>(total) * k / p.n_splits);
+            const int b1 = static_cast<int>(static_cast<long long>(total) * (k + 1) / p.n_splits);
+            if (b1 > b0) {
+                const int s0 = entry_meta(b0) >> 8;
+                my_rng = make_int2(s0, (entry_meta(b1 - 1) >> 8) - s0 + 1);
+            }
+        }
+    }
+    // ... and the slot log-sums: the first 32 (head, slot) pairs of the splits warp and warp + kWarps
+    float xs[2] = {kNegInf, kNegInf};
+    if (p.mass) {
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const int k = warp + j * kWarps;
+            const int first = __shfl_sync(0xffffffffu, my_rng.x, j), cnt = __shfl_sync(0xffffffffu, my_rng.y, j);
+            if (k < p.n_splits && lane < cnt * rep)
+                xs[j] = __ldcg(p.part_slot + (k * split_stride + row_h0 + lane / cnt) * p.slot_stride + first + lane % cnt);
+        }
     }
     for (int h = warp; h < rep; h += kWarps) {                               // weights of the splits: one warp per head
         const float my0 = lane < p.n_splits ? __ldcg(p.part_lse + lane * split_stride + row_h0 + h) : kNegInf;
@@ -591,7 +631,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
         for (int idx = threadIdx.x; idx < rep * (G + 1); idx += kThreads) tab[idx] = 0.f;
     __syncthreads();
 
-    // Round trip 2: the slot log-sums of every split (only the slots its range touched)
+    // the slot log-sums of every split (only the slots its range touched): what was fetched above, then the rest
     if (p.mass && tab_fits) {
         for (int j = 0; warp + j * kWarps < p.n_splits; ++j) {
             const int k = warp + j * kWarps;
@@ -599,7 +639,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
             for (int idx = lane; idx < cnt * rep; idx += 32) {
                 const int h = idx / cnt, sl = idx % cnt;
                 const float lse = cm[h];
-                const float x = __ldcg(p.part_slot + (k * split_stride + row_h0 + h) * p.slot_stride + first + sl);
+                const float x = (j < 2 && idx < 32) ? (j == 0 ? xs[0] : xs[1])
+                                                    : __ldcg(p.part_slot + (k * split_stride + row_h0 + h) * p.slot_stride + first + sl);
                 if (lse != kNegInf && x != kNegInf) atomicAdd(&tab[h * (G + 1) + first + sl], ex2(x - lse));
             }
         }
