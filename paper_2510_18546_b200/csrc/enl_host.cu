@@ -72,6 +72,41 @@ bool encode_map(CUtensorMap *tm, const void *base, int rank, const cuuint64_t *d
 
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
+// Tensor maps of the caller's tensors, kept by (pointer, shape): a planning step calls enl_attend once per layer with
+// tensors that come back step after step, and encoding three maps per call is most of the host time of a call whose
+// gather plan is reused.
+struct MapKey {
+    const void *base;
+    uint64_t d0, d1, d2;
+    uint32_t b0, b1, b2;
+    bool operator==(const MapKey &o) const
+    {
+        return base == o.base && d0 == o.d0 && d1 == o.d1 && d2 == o.d2 && b0 == o.b0 && b1 == o.b1 && b2 == o.b2;
+    }
+};
+struct MapCache {
+    static constexpr int kSlots = 256;
+    MapKey key[kSlots] = {};
+    CUtensorMap map[kSlots];
+    bool used[kSlots] = {};
+    // 3-D bf16 map [d2][d1][d0] with box {b0, b1, b2}
+    bool get(CUtensorMap *out, const void *base, const cuuint64_t *dims, const cuuint64_t *strides, const cuuint32_t *box)
+    {
+        const MapKey k{base, dims[0], dims[1], dims[2], box[0], box[1], box[2]};
+        const size_t h = (reinterpret_cast<uintptr_t>(base) >> 8) * 0x9E3779B97F4A7C15ull >> 56;
+        for (int probe = 0; probe < 4; ++probe) {
+            const int i = static_cast<int>((h + probe) % kSlots);
+            if (used[i] && key[i] == k) { *out = map[i]; return true; }
+        }
+        if (!encode_map(out, base, 3, dims, strides, box)) return false;
+        const int i = static_cast<int>(h % kSlots);
+        key[i] = k;
+        map[i] = *out;
+        used[i] = true;
+        return true;
+    }
+};
+
 }  // namespace
 
 struct enl_cache {
@@ -103,6 +138,7 @@ struct enl_cache {
     bool pairs_ok = false;                  // the device can co-schedule two of the attention kernel's CTAs as a cluster
     std::vector<int32_t> key_sel, key_cu, key_len;   // what the current plan was built from
     int32_t plan_entries = 0, plan_items = 0, plan_splits = 1, plan_batch = 0, plan_max_slots = 0;
+    MapCache maps;                          // tensor maps of the caller's q / k_new / v_new
     std::vector<int32_t> seen;              // duplicate detection stamps
     int32_t stamp = 0;
 
@@ -715,7 +751,7 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
         const cuuint64_t ns[2] = {static_cast<cuuint64_t>(d.head_dim) * 2,
                                   static_cast<cuuint64_t>(d.head_dim) * 2 * d.n_kv_heads};
         const cuuint32_t nb[3] = {64, 1, kPageTokens};
-        if (!encode_map(&dp.tm_knew, a->k_new, 3, nd, ns, nb) || !encode_map(&dp.tm_vnew, a->v_new, 3, nd, ns, nb))
+        if (!c->maps.get(&dp.tm_knew, a->k_new, nd, ns, nb) || !c->maps.get(&dp.tm_vnew, a->v_new, nd, ns, nb))
             return ENL_E_CUDA;
         dp.tm_kpool = c->tm_k[a->layer];
         dp.tm_vpool = c->tm_v[a->layer];
@@ -761,8 +797,8 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
         const cuuint64_t ns[2] = {static_cast<cuuint64_t>(d.head_dim) * 2,
                                   static_cast<cuuint64_t>(d.head_dim) * 2 * d.n_kv_heads};
         const cuuint32_t nb[3] = {64, 1, kTileKeys};
-        if (!encode_map(&p.tm_q, a->q, 3, qd, qs, qb) || !encode_map(&p.tm_knew, a->k_new, 3, nd, ns, nb) ||
-            !encode_map(&p.tm_vnew, a->v_new, 3, nd, ns, nb))
+        if (!c->maps.get(&p.tm_q, a->q, qd, qs, qb) || !c->maps.get(&p.tm_knew, a->k_new, nd, ns, nb) ||
+            !c->maps.get(&p.tm_vnew, a->v_new, nd, ns, nb))
             return ENL_E_CUDA;
     }
     p.tm_kpool = c->tm_k[a->layer];
