@@ -335,21 +335,22 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
     const uint32_t bar_peer_o = bar0 + 8u * (10 + 2 * C::kStages);
     const uint32_t bar_peer_free = bar0 + 8u * (11 + 2 * C::kStages);
     const uint32_t bar_peer_ack = bar0 + 8u * (12 + 2 * C::kStages);
-    // between two segments of a CTA: the softmax warps no longer use the shared memory of the Q tiles (they stage
-    // their output there) / have read the accumulator O_i, which the next segment's first P V overwrites
-    const uint32_t bar_q_free = bar0 + 8u * (13 + 2 * C::kStages);
-    auto bar_o_free   = [&](int i) { return bar0 + 8u * (14 + 2 * C::kStages + i); };
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + C::kBarOff + 8 * (16 + 2 * C::kStages));
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + C::kBarOff + 8 * (13 + 2 * C::kStages));
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
-    // The CTA's work: one or more segments, walked one after the other.  Every role reads the segment's description
-    // itself and keeps its own counters (segments done, key tiles done, ring fills done) for the barrier parities.
-    const int seg_beg = p.cta_first[blockIdx.x], seg_end = p.cta_first[blockIdx.x + 1];
+    // work item
+    const Item it = p.items[blockIdx.x];
+    const EpInfo ep = p.eps[it.ep];
     const int rep = p.rep;
     const int tile_tokens = kTileRows / rep;
-    auto q_tiles_of = [&](const Item &it, const EpInfo &ep) {
-        return (min(it.t0 + kQTiles * tile_tokens, ep.n_q) - it.t0 > tile_tokens) ? 2 : 1;
-    };
+    const int t_hi = min(it.t0 + kQTiles * tile_tokens, ep.n_q);        // exclusive
+    const int n_qt = (t_hi - it.t0 > tile_tokens) ? 2 : 1;
+    const int c_max = ep.n_new - ep.n_q + t_hi - 1;                      // last new key any row sees
+    const int n_new_tiles = c_max / kTileKeys + 1;
+    const int total_tiles = ep.n_ctiles + n_new_tiles;
+    const int j_beg = static_cast<int>(static_cast<long long>(total_tiles) * it.split / p.n_splits);
+    const int j_end = static_cast<int>(static_cast<long long>(total_tiles) * (it.split + 1) / p.n_splits);
+    const int n_tiles = j_end - j_beg;
 
     // ---- set-up ----
     if (threadIdx.x == 0) {
@@ -366,12 +367,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
         mbar_init(bar_peer_o, 1);                                    // this thread's arrival below + 64 KB from the peer
         mbar_init(bar_peer_free, 1);
         mbar_init(bar_peer_ack, 1);
-        mbar_init(bar_q_free, kSoftmaxWarps);
-        mbar_init(bar_o_free(0), 4);
-        mbar_init(bar_o_free(1), 4);
-        if (p.pair_merge) {                                          // one segment per CTA
-            const Item it0 = p.items[seg_beg];
-            const int n_qt = q_tiles_of(it0, p.eps[it0.ep]);
+        if (p.pair_merge) {
             mbar_expect_tx(bar_peer_ml, static_cast<uint32_t>(n_qt * 128 * 16));
             mbar_expect_tx(bar_peer_o, 4u * 16384u);
         }
@@ -400,35 +396,21 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
       asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
       if (warp == kProducerWarp) {
         // ================= TMA producer =================
-        int fill = 0, done = 0;                                     // ring fills and segments so far
-        for (int sg = seg_beg; sg < seg_end && ok; ++sg) {
-            const Item it = p.items[sg];
-            const EpInfo ep = p.eps[it.ep];
-            const int n_qt = q_tiles_of(it, ep);
-            const int j_beg = it.j_beg, j_end = it.j_end;
-            if (j_end <= j_beg) continue;
-            // The Q tiles' shared memory is the previous segment's output staging area: Q is fetched once that is over,
-            // which is after the first fills of the ring (their slots were the previous segment's; its MMAs free them).
-            const int q_at = done > 0 ? min(C::kStages, 2 * (j_end - j_beg)) : 0;
-            const int fill0 = fill;
-            auto load_q = [&]() {
-                if (done > 0) ok = mbar_wait(bar_q_free, static_cast<uint32_t>((done - 1) & 1), abort_flag, p.status);
-                if (ok && lane == 0) {
-                    mbar_expect_tx(bar_q_full, static_cast<uint32_t>(n_qt * C::kTileBytes));
-                    for (int i = 0; i < n_qt; ++i)
-                        for (int hf = 0; hf < C::kHalves; ++hf)
-                            tma_load_3d(q_addr(i) + hf * C::kHalfBytes, &p.tm_q, hf * 64, it.kvh * rep,
-                                        ep.q_off + it.t0 + i * tile_tokens, bar_q_full);
-                }
-            };
-            if (q_at == 0) load_q();
+        if (n_tiles > 0) {
+            if (lane == 0) {
+                mbar_expect_tx(bar_q_full, static_cast<uint32_t>(n_qt * C::kTileBytes));
+                for (int i = 0; i < n_qt; ++i)
+                    for (int hf = 0; hf < C::kHalves; ++hf)
+                        tma_load_3d(q_addr(i) + hf * C::kHalfBytes, &p.tm_q, hf * 64, it.kvh * rep,
+                                    ep.q_off + it.t0 + i * tile_tokens, bar_q_full);
+            }
+            int fill = 0;
             for (int j = j_beg; j < j_end && ok; ++j) {
                 const bool cached = j < ep.n_ctiles;
                 int page = 0;
                 if (cached && lane < kPagesPerTile)
                     page = p.stream_page[ep.stream_off + j * kPagesPerTile + lane];
                 for (int kv = 0; kv < 2; ++kv, ++fill) {
-                    if (q_at > 0 && fill - fill0 == q_at) { load_q(); if (!ok) break; }
                     const int st = fill % C::kStages;
                     if (fill >= C::kStages) {
                         ok = mbar_wait(bar_kv_empty(st), static_cast<uint32_t>((fill / C::kStages - 1) & 1),
@@ -455,21 +437,19 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                     }
                 }
             }
-            if (ok && q_at > 0 && fill - fill0 == q_at) load_q();   // a segment whose fills all came before Q
-            ++done;
-        }
-        // error path only: let the copies already in flight land before the CTA retires
-        if (!ok) {
-            const int first = fill > C::kStages ? fill - C::kStages : 0;
-            for (int f = first; f < fill; ++f) {
-                const unsigned long long t0 = global_ns();
-                while (!mbar_try_wait(bar_kv_full(f % C::kStages), static_cast<uint32_t>((f / C::kStages) & 1)) &&
-                       global_ns() - t0 < 2000000ull) { }
+            // error path only: let the copies already in flight land before the CTA retires
+            if (!ok) {
+                const int first = fill > C::kStages ? fill - C::kStages : 0;
+                for (int f = first; f < fill; ++f) {
+                    const unsigned long long t0 = global_ns();
+                    while (!mbar_try_wait(bar_kv_full(f % C::kStages), static_cast<uint32_t>((f / C::kStages) & 1)) &&
+                           global_ns() - t0 < 2000000ull) { }
+                }
             }
         }
       } else if (warp == kMmaWarp) {
         // ================= MMA issuer =================
-        {
+        if (n_tiles > 0) {
             constexpr uint32_t idesc_qk = make_idesc(kTileKeys, false);
             constexpr uint32_t idesc_pv = make_idesc(D, true);
             auto tmem_s = [&](int i) { return tmem_base + static_cast<uint32_t>(i * 128); };
@@ -519,35 +499,23 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
             auto full_bar = [&](int f) { return bar_kv_full(f % C::kStages); };
             auto full_par = [&](int f) { return static_cast<uint32_t>((f / C::kStages) & 1); };
 
-            // ring fills, segments, and per Q tile the key tiles so far (a segment at the end of an episode may have
-            // one Q tile only: the barriers of the other then see nothing of it)
-            int fbase = 0, done = 0, gt0 = 0, gt1 = 0;
-            for (int sg = seg_beg; sg < seg_end && ok; ++sg) {
-            const Item it = p.items[sg];
-            const int n_qt = q_tiles_of(it, p.eps[it.ep]);
-            const int n_tiles = it.j_end - it.j_beg;
-            if (n_tiles <= 0) continue;
-            ok = mbar_wait(bar_q_full, static_cast<uint32_t>(done & 1), abort_flag, p.status);
-            if (ok) ok = wait_full(fbase);
+            ok = mbar_wait(bar_q_full, 0, abort_flag, p.status);
+            if (ok) ok = wait_full(0);
             if (ok) {
                 tc_fence_after();
-                for (int i = 0; i < n_qt; ++i) issue_qk(i, fbase % C::kStages);
-                commit_to(bar_kv_empty(fbase % C::kStages));
+                for (int i = 0; i < n_qt; ++i) issue_qk(i, 0);
+                commit_to(bar_kv_empty(0));
             }
-            Pending w_v = arm(full_bar(fbase + 1), full_par(fbase + 1));    // V of the first tile
-            Pending w_p = arm(bar_p_half(0, 0), static_cast<uint32_t>(gt0 & 1));  // first half of P_0
+            Pending w_v = arm(full_bar(1), full_par(1));                // V of the first tile
+            Pending w_p = arm(bar_p_half(0, 0), 0u);                    // first half of P_0
             for (int jj = 0; jj < n_tiles && ok; ++jj) {
-                const int fv = fbase + 2 * jj + 1, fk = fbase + 2 * jj + 2;   // ring slots of V_jj and K_{jj+1}
+                const int fv = 2 * jj + 1, fk = 2 * jj + 2;             // ring slots of V_jj and K_{jj+1}
                 const bool more = jj + 1 < n_tiles;
-                const uint32_t par0 = static_cast<uint32_t>((gt0 + jj) & 1), par1 = static_cast<uint32_t>((gt1 + jj) & 1);
+                const uint32_t par = static_cast<uint32_t>(jj & 1);
                 for (int i = 0; i < n_qt; ++i) {
                     const bool last_i = i == n_qt - 1;
-                    const uint32_t par = i ? par1 : par0;
                     if (i == 0) ok = await(w_v);
                     if (ok) ok = await(w_p);
-                    // the first P V of a segment overwrites O_i: the previous segment's rows must have been read out
-                    if (ok && jj == 0 && done > 0)
-                        ok = mbar_wait(bar_o_free(i), static_cast<uint32_t>((done - 1) & 1), abort_flag, p.status);
                     if (!ok) break;
                     tc_fence_after();
                     const Pending w_h1 = arm(bar_p_half(i, 1), par);
@@ -557,7 +525,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                     tc_fence_after();
                     Pending w_k = {0u, 0u, true};
                     if (more && i == 0) w_k = arm(full_bar(fk), full_par(fk));
-                    if (!more && !last_i) w_p = arm(bar_p_half(i + 1, 0), par1);
+                    if (!more && !last_i) w_p = arm(bar_p_half(i + 1, 0), par);
                     issue_pv(i, fv % C::kStages, 1, false);
                     if (last_i) commit_to(bar_kv_empty(fv % C::kStages));
                     if (!more) commit_to(bar_o_done(i));
@@ -567,10 +535,10 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                         tc_fence_after();
                         // what follows Q_i K^T: the next tile's P of this key tile, or (after the last Q tile) V and P_0 of the next
                         if (!last_i) {
-                            w_p = arm(bar_p_half(i + 1, 0), par1);
+                            w_p = arm(bar_p_half(i + 1, 0), par);
                         } else {
                             w_v = arm(full_bar(fv + 2), full_par(fv + 2));
-                            w_p = arm(bar_p_half(0, 0), par0 ^ 1u);
+                            w_p = arm(bar_p_half(0, 0), par ^ 1u);
                         }
                         issue_qk(i, fk % C::kStages);
                         if (last_i) commit_to(bar_kv_empty(fk % C::kStages));
@@ -579,31 +547,19 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
             }
             // pair merge: once every MMA of this CTA has completed, its K/V ring is idle and the peer may write
             // into it (only a CTA that finishes a Q tile receives anything)
-            if (ok && pair && it.piece < n_qt) {
+            if (ok && pair && it.split < n_qt) {
                 for (int i = 0; i < n_qt && ok; ++i) ok = mbar_wait(bar_o_done(i), 0, abort_flag, p.status);
                 if (ok && lane == 0) peer_arrive(peer_addr(bar_peer_free, cluster_rank() ^ 1u));
-            }
-            fbase += 2 * n_tiles;
-            gt0 += n_tiles;
-            if (n_qt == 2) gt1 += n_tiles;
-            ++done;
             }
         }
       }
     } else {
       asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
-      // ================= softmax / epilogue: one thread per query row =================
-      const int i = warp >> 2;                                     // Q tile
-      const int q4 = warp & 3;                                     // TMEM lane quadrant
-      const int r = q4 * 32 + lane;
-      int gt = 0, done = 0, seg_no = 0;                            // key tiles and segments of this Q tile so far; segments
-      for (int sg = seg_beg; sg < seg_end && ok; ++sg) {
-      const Item it = p.items[sg];
-      const EpInfo ep = p.eps[it.ep];
-      const int n_qt = q_tiles_of(it, ep);
-      const int j_beg = it.j_beg, j_end = it.j_end;
-      const int n_tiles = j_end - j_beg;
-      if (i < n_qt) {
+      if ((warp >> 2) < n_qt) {
+        // ================= softmax / epilogue: one thread per query row =================
+        const int i = warp >> 2;                                   // Q tile
+        const int q4 = warp & 3;                                   // TMEM lane quadrant
+        const int r = q4 * 32 + lane;
         const int t = it.t0 + i * tile_tokens + r / rep;           // episode-relative query token
         const int h = it.kvh * rep + r % rep;
         const bool row_valid = t < ep.n_q;
@@ -613,18 +569,15 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
         const uint32_t lane_sel = static_cast<uint32_t>(q4 * 32) << 16;
         const uint32_t t_s = tmem_base + lane_sel + static_cast<uint32_t>(i * 128);
         const uint32_t t_o = tmem_base + lane_sel + static_cast<uint32_t>(256 + i * 128);
-        const bool split_mode = it.n_pieces > 1 && !pair;
+        const bool split_mode = p.n_splits > 1 && !pair;
         const long long grow = static_cast<long long>(ep.q_off) + t;   // global query row
-        // index of the (row, head) pair: in the caller's tensors, or in the partial-result buffers
-        const long long rh = split_mode ? static_cast<long long>(it.part_base + it.piece) * kItemRows + i * kTileRows + r
-                                        : grow * p.Hq + h;
-        const int slot_stride = split_mode ? p.part_stride : p.mass_stride;
+        const long long rh = (split_mode ? (static_cast<long long>(it.split) * p.n_q_total + grow) : grow) * p.Hq + h;
         // Where this row's slot log-sums are parked until the row's total is known: shared memory when the call has few
         // slots (one store per slot end, no round trip to the L2 at the end), else the buffer that takes the result.
         float *slot_out = nullptr;
         if (row_valid) {
-            if (split_mode) { if (p.part_slot) slot_out = p.part_slot + rh * slot_stride; }
-            else if (p.mass) slot_out = p.mass + rh * slot_stride;
+            if (split_mode) { if (p.part_slot) slot_out = p.part_slot + rh * p.mass_stride; }
+            else if (p.mass) slot_out = p.mass + rh * p.mass_stride;
         }
         const bool park_smem = G + 1 <= kParkSlots;
         float *park_row = reinterpret_cast<float *>(smem + C::kParkOff) + i * (kParkSlots * 128) + r;   // + slot * 128
@@ -635,10 +588,10 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
         int shared_slot = -1, skip_slot = -1;
         float bnd = kNegInf;
         if (pair) {
-            const int jb = (it.piece == 0) ? j_end : j_beg;         // first tile of split 1
+            const int jb = (it.split == 0) ? j_end : j_beg;         // first tile of split 1
             const int last0 = (jb > ep.n_ctiles) ? G : (__ldg(p.stream_meta + ep.stream_off + jb * kPagesPerTile - 1) >> 8);
             const int first1 = (jb < ep.n_ctiles) ? (__ldg(p.stream_meta + ep.stream_off + jb * kPagesPerTile) >> 8) : G;
-            if (last0 == first1) { shared_slot = last0; if (it.piece == 1) skip_slot = last0; }
+            if (last0 == first1) { shared_slot = last0; if (it.split == 1) skip_slot = last0; }
         }
         float m = kNegInf, l = 0.f, acc = 0.f;                     // reference (log2 units), row sum, sum of the current slot
         int cur_slot = -1;
@@ -682,7 +635,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                 mask_pages = vis_lo >= kTileKeys ? 0u : (0xffu << (max(vis_lo, 0) / kPageTokens)) & 0xffu;
             }
 
-            ok = mbar_wait(bar_s_full(i), static_cast<uint32_t>((gt + jj) & 1), abort_flag, p.status);
+            ok = mbar_wait(bar_s_full(i), static_cast<uint32_t>(jj & 1), abort_flag, p.status);
             if (!ok) break;
             tc_fence_after();
 
@@ -810,8 +763,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
             const int r2 = q4 * 32 + rr;
             const int t2 = it.t0 + i * tile_tokens + r2 / rep;
             if (t2 >= ep.n_q) return -1;
-            if (split_mode) return (it.part_base + it.piece) * kItemRows + i * kTileRows + r2;
-            return (ep.q_off + t2) * p.Hq + it.kvh * rep + r2 % rep;
+            const int g2 = ep.q_off + t2;
+            return (split_mode ? it.split * p.n_q_total + g2 : g2) * p.Hq + it.kvh * rep + r2 % rep;
         };
         // The warp's 32 rows x 128 bytes leave through the (idle) shared memory of the Q tile: row-per-thread
         // stores would touch 32 different rows per instruction.  Each thread stages its own 128 bytes, 16-byte
@@ -902,7 +855,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
         };
         // slots this CTA walked (all of them without splits)
         int first_slot = 0, last_slot = G;
-        if (it.n_pieces > 1) {
+        if (p.n_splits > 1) {
             first_slot = G + 1;
             last_slot = -1;
             if (n_tiles > 0) {
@@ -919,7 +872,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                 if (p.mass) finish_masses(lse, kNegInf, 0, G);
                 if (n_tiles > 0 && !p.mass_only) {
                     const float inv = (l > 0.f) ? 1.f / l : 0.f;
-                    ok = mbar_wait(bar_o_done(i), static_cast<uint32_t>(done & 1), abort_flag, p.status);
+                    ok = mbar_wait(bar_o_done(i), 0, abort_flag, p.status);
                     if (ok) {
                         tc_fence_after();
 #pragma unroll 1
@@ -949,14 +902,14 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                     for (int rr = 0; rr < 32; ++rr) {               // slots this split did not walk contribute nothing
                         const int ri = __shfl_sync(kFull, my_ridx, rr);
                         if (ri < 0) continue;
-                        float *slots = p.part_slot + static_cast<long long>(ri) * slot_stride;
+                        float *slots = p.part_slot + static_cast<long long>(ri) * p.mass_stride;
                         for (int sl = lane; sl <= G; sl += 32)
                             if (sl < first_slot || sl > last_slot) slots[sl] = kNegInf;
                     }
                 }
                 if (n_tiles > 0) {
                     const float inv = (l > 0.f) ? 1.f / l : 0.f;
-                    ok = mbar_wait(bar_o_done(i), static_cast<uint32_t>(done & 1), abort_flag, p.status);
+                    ok = mbar_wait(bar_o_done(i), 0, abort_flag, p.status);
                     if (ok) {
                         tc_fence_after();
 #pragma unroll 1
@@ -981,8 +934,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                 constexpr uint32_t kRingOff = kQTiles * C::kTileBytes;
                 constexpr uint32_t kExportStageOff = 65536;         // upper half of the ring (4 stages x 32 KB)
                 const uint32_t warp_off = kRingOff + static_cast<uint32_t>(q4 * 16384);
-                if (i != it.piece && n_tiles > 0) {
-                    // This CTA finishes Q tile `it.piece`; the accumulator of the other tile goes to the peer, which
+                if (i != it.split && n_tiles > 0) {
+                    // This CTA finishes Q tile `it.split`; the accumulator of the other tile goes to the peer, which
                     // finishes that one.  It goes as it is (relative to this CTA's own reference; the peer learns the
                     // weight from the row sums above), so that nothing but the last MMA stands before it: staged
                     // row-per-thread in the upper half of this CTA's ring (idle once both tiles' MMAs are done; 16 KB
@@ -1030,7 +983,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                 // written by split 0, which adds the part split 1 sent.  (Before the output: the peer's accumulator is
                 // still on its way.)
                 if (ok && p.mass) finish_masses(pair_lse, pair_bnd, first_slot, last_slot);
-                if (ok && i == it.piece && n_tiles > 0) {
+                if (ok && i == it.split && n_tiles > 0) {
                     // this CTA finishes the tile: its own accumulator and what the peer sent, each with its weight;
                     // thread (warp, lane) reads what thread (warp, lane) of the peer wrote
                     ok = mbar_wait(bar_o_done(i), 0, abort_flag, p.status);
@@ -1066,20 +1019,6 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
               }
             }
         }
-      }
-      // the segment's rows are out: its accumulators and the Q tiles' shared memory may be used again
-      if (n_tiles > 0) {
-          // the warps of a Q tile that the segment does not have say so when the segment's MMAs are over, not before:
-          // running ahead, they would arrive twice in one phase
-          if (i >= n_qt && sg + 1 < seg_end) ok = mbar_wait(bar_o_done(0), static_cast<uint32_t>(seg_no & 1), abort_flag, p.status);
-          ++seg_no;
-          if (ok && sg + 1 < seg_end) {
-              tc_fence_before();
-              __syncwarp();
-              if (lane == 0) { mbar_arrive(bar_o_free(i)); mbar_arrive(bar_q_free); }
-          }
-          if (i < n_qt) { gt += n_tiles; ++done; }
-      }
       }
     }
 
@@ -1129,15 +1068,15 @@ bool attention_pairs_supported()
     return n > 0;
 }
 
-cudaError_t launch_attention(const AttnParams &p, int head_dim, int n_ctas, cudaStream_t st)
+cudaError_t launch_attention(const AttnParams &p, int head_dim, int n_items, cudaStream_t st)
 {
-    if (n_ctas <= 0) return cudaSuccess;
+    if (n_items <= 0) return cudaSuccess;
     cudaError_t e;
-    if (p.pair_merge && (head_dim != 128 || (n_ctas & 1))) return cudaErrorInvalidValue;
+    if (p.pair_merge && (head_dim != 128 || p.n_splits != 2 || (n_items & 1))) return cudaErrorInvalidValue;
     if (head_dim == 128)
-        e = launch_pdl(attn_kernel<128>, dim3(n_ctas), dim3(kThreads), Cfg<128>::kSmemBytes, st, p, p.pair_merge ? 2u : 1u);
+        e = launch_pdl(attn_kernel<128>, dim3(n_items), dim3(kThreads), Cfg<128>::kSmemBytes, st, p, p.pair_merge ? 2u : 1u);
     else if (head_dim == 64)
-        e = launch_pdl(attn_kernel<64>, dim3(n_ctas), dim3(kThreads), Cfg<64>::kSmemBytes, st, p);
+        e = launch_pdl(attn_kernel<64>, dim3(n_items), dim3(kThreads), Cfg<64>::kSmemBytes, st, p);
     else
         return cudaErrorInvalidValue;
     return e != cudaSuccess ? e : cudaGetLastError();

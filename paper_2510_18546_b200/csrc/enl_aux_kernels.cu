@@ -74,40 +74,25 @@ __global__ void combine_kernel(const CombineParams p)
     constexpr int V = D / 32;                               // channels per lane
     const int lane = threadIdx.x & 31;
     const long long rh = blockIdx.x * static_cast<long long>(blockDim.x >> 5) + (threadIdx.x >> 5);
-    const long long n_rh = static_cast<long long>(p.n_q_total) * p.Hq;
+    const long long split_stride = static_cast<long long>(p.n_q_total) * p.Hq;
     pdl_trigger();
-    if (rh >= n_rh) return;
+    pdl_wait();                                             // the partial results come from the previous kernel
+    if (rh >= split_stride) return;
     const int row = static_cast<int>(rh / p.Hq);
     const float ninf = -__builtin_huge_valf();
-    // Where the pieces of this (row, head) lie: piece k at index first + k * step of the partial buffers.  By item:
-    // the row's item for this kv head, block (part_base + k) of kItemRows rows, the row's place in the item's two Q
-    // tiles.  An item in one piece was written by the attention kernel itself.
-    long long first = rh, step = n_rh;
-    int n_splits = p.n_splits;
-    if (p.row_item) {
-        const int h = static_cast<int>(rh - static_cast<long long>(row) * p.Hq);
-        const int2 ip = p.item_part[p.row_item[row] + h / p.rep];
-        if (ip.y <= 1) return;
-        const int local = p.row_local[row];
-        first = static_cast<long long>(ip.x) * kItemRows + (local / p.tile_tokens) * kTileRows +
-                (local % p.tile_tokens) * p.rep + h % p.rep;
-        step = kItemRows;
-        n_splits = ip.y;
-    }
-    pdl_wait();                                             // the partial results come from the previous kernel
 
     // Few splits (the usual case): every load of the warp -- log-sum-exps, partial outputs, the first 32 slot
     // log-sums -- is issued before anything is computed, so the warp pays one memory round trip, not five.
-    if (n_splits <= 4) {
-        const float *slot0 = p.part_slot ? p.part_slot + first * p.slot_stride + lane : nullptr;
+    if (p.n_splits <= 4) {
+        const float *slot0 = p.part_slot ? p.part_slot + rh * p.slot_stride + lane : nullptr;
         const int G = p.mass ? p.row_slots[row] : -1;
         float lv[4], sv[4], ov[4][V];
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-            const bool on = k < n_splits;
-            lv[k] = on ? __ldcg(p.part_lse + first + k * step) : ninf;
-            sv[k] = (on && p.mass && lane <= G) ? __ldcg(slot0 + k * step * p.slot_stride) : ninf;
-            const float *src = p.part_o + (first + (on ? k : 0) * step) * D + lane * V;
+            const bool on = k < p.n_splits;
+            lv[k] = on ? __ldcg(p.part_lse + k * split_stride + rh) : ninf;
+            sv[k] = (on && p.mass && lane <= G) ? __ldcg(slot0 + k * split_stride * p.slot_stride) : ninf;
+            const float *src = p.part_o + ((on ? k : 0) * split_stride + rh) * D + lane * V;
             if constexpr (V == 4) {
                 const float4 t = __ldcg(reinterpret_cast<const float4 *>(src));
                 ov[k][0] = t.x; ov[k][1] = t.y; ov[k][2] = t.z; ov[k][3] = t.w;
@@ -145,8 +130,8 @@ __global__ void combine_kernel(const CombineParams p)
             }
             for (int s = lane + 32; s <= G; s += 32) {                      // more than 32 slots: the rest, as below
                 float w = 0.f;
-                for (int k = 0; k < n_splits; ++k) {
-                    const float v = __ldcg(p.part_slot + (first + k * step) * p.slot_stride + s);
+                for (int k = 0; k < p.n_splits; ++k) {
+                    const float v = __ldcg(p.part_slot + (k * split_stride + rh) * p.slot_stride + s);
                     if (v != ninf) w += ex2f(v - lse);
                 }
                 p.mass[rh * p.mass_stride + s] = w;
@@ -156,8 +141,8 @@ __global__ void combine_kernel(const CombineParams p)
     }
 
     // every lane needs every split's log-sum-exp: lane k loads split k (and k + 32), then shuffles
-    float my0 = lane < n_splits ? p.part_lse[first + lane * step] : ninf;
-    float my1 = lane + 32 < n_splits ? p.part_lse[first + (lane + 32) * step] : ninf;
+    float my0 = lane < p.n_splits ? p.part_lse[lane * split_stride + rh] : ninf;
+    float my1 = lane + 32 < p.n_splits ? p.part_lse[(lane + 32) * split_stride + rh] : ninf;
     float mx = fmaxf(my0, my1);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
@@ -171,10 +156,10 @@ __global__ void combine_kernel(const CombineParams p)
     float acc[V];
 #pragma unroll
     for (int x = 0; x < V; ++x) acc[x] = 0.f;
-    for (int k = 0; k < n_splits; ++k) {
+    for (int k = 0; k < p.n_splits; ++k) {
         const float w = __shfl_sync(0xffffffffu, k < 32 ? w0 : w1, k & 31);
         if (w != 0.f) {
-            const float *src = p.part_o + (first + k * step) * D + lane * V;
+            const float *src = p.part_o + (k * split_stride + rh) * D + lane * V;
             if constexpr (V == 4) {
                 const float4 v = *reinterpret_cast<const float4 *>(src);
                 acc[0] += w * v.x; acc[1] += w * v.y; acc[2] += w * v.z; acc[3] += w * v.w;
@@ -193,8 +178,8 @@ __global__ void combine_kernel(const CombineParams p)
         const int G = p.row_slots[row];
         for (int s = lane; s <= G; s += 32) {
             float w = 0.f;
-            for (int k = 0; k < n_splits; ++k) {
-                const float v = p.part_slot[(first + k * step) * p.slot_stride + s];
+            for (int k = 0; k < p.n_splits; ++k) {
+                const float v = p.part_slot[(k * split_stride + rh) * p.slot_stride + s];
                 if (v != ninf) w += ex2f(v - lse);
             }
             p.mass[rh * p.mass_stride + s] = w;

@@ -125,11 +125,7 @@ struct enl_cache {
     // gather plan: host image (pinned when there is a GPU), device copy, capacities
     int32_t cap_entries = 0, cap_items = 0;
     uint8_t *plan_host = nullptr, *plan_dev = nullptr;
-    // fixed regions; the segment list, the CTAs' first segments and the items' partial blocks follow the episodes at
-    // offsets of the current plan (off_items .. off_head_end travel in one copy), the per-row arrays likewise
-    size_t off_eps = 0, off_items = 0, off_stream = 0, off_meta = 0, off_rows = 0, plan_bytes = 0;
-    size_t off_ctafirst = 0, off_itempart = 0, off_head_end = 0;
-    size_t off_rowslots = 0, off_rowitem = 0, off_rowlocal = 0, off_rowobj = 0, off_rows_end = 0;
+    size_t off_eps = 0, off_items = 0, off_stream = 0, off_meta = 0, off_rowslots = 0, off_rowobj = 0, plan_bytes = 0;
     cudaEvent_t plan_copied = nullptr;
     bool plan_valid = false, plan_on_device = false;
     uint64_t plan_epoch = 0;
@@ -139,8 +135,6 @@ struct enl_cache {
     std::vector<int32_t> key_obj;           // object spans the row -> object map was built from
     bool plan_decode = false;               // the plan is for the one-token decode kernel
     bool plan_pair = false;                 // two splits whose CTAs merge inside the attention kernel (cluster of two)
-    bool plan_merge = false;                // some item is cut into pieces that the merge kernel puts together
-    int32_t plan_ctas = 0, plan_blocks = 0; // CTAs of the attention launch; partial-result blocks in the scratch buffer
     bool pairs_ok = false;                  // the device can co-schedule two of the attention kernel's CTAs as a cluster
     std::vector<int32_t> key_sel, key_cu, key_len;   // what the current plan was built from
     int32_t plan_entries = 0, plan_items = 0, plan_splits = 1, plan_batch = 0, plan_max_slots = 0;
@@ -169,10 +163,6 @@ struct enl_cache {
     int32_t *h_meta() { return reinterpret_cast<int32_t *>(plan_host + off_meta); }
     int32_t *h_rowslots() { return reinterpret_cast<int32_t *>(plan_host + off_rowslots); }
     int32_t *h_rowobj() { return reinterpret_cast<int32_t *>(plan_host + off_rowobj); }
-    int32_t *h_rowitem() { return reinterpret_cast<int32_t *>(plan_host + off_rowitem); }
-    int32_t *h_rowlocal() { return reinterpret_cast<int32_t *>(plan_host + off_rowlocal); }
-    int32_t *h_ctafirst() { return reinterpret_cast<int32_t *>(plan_host + off_ctafirst); }
-    int2 *h_itempart() { return reinterpret_cast<int2 *>(plan_host + off_itempart); }
 };
 
 namespace {
@@ -263,11 +253,11 @@ extern "C" int enl_cache_create(const enl_cache_desc_t *desc, enl_cache_t **out)
     auto align256 = [](size_t x) { return (x + 255) & ~static_cast<size_t>(255); };
     c->off_eps = 0;
     c->off_items = align256(c->off_eps + sizeof(EpInfo) * d.max_batch);
-    // segments (at most two per item when the launch is cut evenly), one first-segment index per CTA, one int2 per item
-    c->off_stream = align256(c->off_items + (sizeof(Item) + sizeof(int32_t) + sizeof(int2)) * (c->cap_items + 1) + 1024);
+    c->off_stream = align256(c->off_items + sizeof(Item) * c->cap_items);
     c->off_meta = align256(c->off_stream + sizeof(int32_t) * c->cap_entries);
-    c->off_rows = align256(c->off_meta + sizeof(int32_t) * c->cap_entries);
-    c->plan_bytes = align256(c->off_rows + 4 * (sizeof(int32_t) * d.max_q_tokens + 256));
+    c->off_rowslots = align256(c->off_meta + sizeof(int32_t) * c->cap_entries);
+    c->off_rowobj = align256(c->off_rowslots + sizeof(int32_t) * d.max_q_tokens);
+    c->plan_bytes = align256(c->off_rowobj + sizeof(int32_t) * d.max_q_tokens);
 
     if (!c->gpu) {
         c->plan_host = new (std::nothrow) uint8_t[c->plan_bytes];
@@ -520,6 +510,7 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
     if (a->batch < 1 || a->batch > d.max_batch) return ENL_E_INVAL;
     if (a->n_sel < 0 || a->n_q < 1 || a->n_new < a->n_q || a->n_q > d.max_q_tokens) return ENL_E_INVAL;
     if (a->n_sel > 0 && !a->sel_ids) return ENL_E_INVAL;
+    if (a->split_hint < 0) return ENL_E_INVAL;
     const int B = a->batch;
     if (B > 1 && (!a->cu_sel || !a->cu_q || !a->cu_new)) return ENL_E_INVAL;
     const int32_t one_sel[2] = {0, a->n_sel}, one_q[2] = {0, a->n_q}, one_new[2] = {0, a->n_new};
@@ -598,8 +589,8 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
     if (!reuse) {
         // size check first, so that a failed call leaves the previous plan intact
         const int tpc = tokens_per_cta(c);
-        int64_t n_entries = 0, base_items = 0, all_tiles = 0;
-        int min_tiles = 0x7fffffff, max_tiles = 1;
+        int64_t n_entries = 0, base_items = 0;
+        int min_tiles = 0x7fffffff;
         for (int b = 0; b < B; ++b) {
             int64_t e = 0;
             for (int s = cu_sel[b]; s < cu_sel[b + 1]; ++s) e += std::max(1, ceil_div(sel_len[s], kPageTokens));
@@ -610,9 +601,6 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
             // fewest tiles any CTA of this episode walks: its first token block
             const int c_first = nn - nq + std::min(tpc, nq) - 1;
             min_tiles = std::min<int64_t>(min_tiles, e / kPagesPerTile + c_first / kTileKeys + 1);
-            max_tiles = std::max<int64_t>(max_tiles, e / kPagesPerTile + (nn - 1) / kTileKeys + 1);
-            for (int t0 = 0; t0 < nq; t0 += tpc)
-                all_tiles += (e / kPagesPerTile + (nn - nq + std::min(t0 + tpc, nq) - 1) / kTileKeys + 1) * d.n_kv_heads;
         }
         if (n_entries > c->cap_entries || base_items > c->cap_items) return ENL_E_NOMEM;
 
@@ -644,44 +632,18 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
                 static_cast<int64_t>(B) * d.n_kv_heads * n_splits > c->cap_items)
                 decode = false;                                                    // too long for one merge: general kernel
         }
-        // The general kernel's launch.  Whole: one CTA per item (two Q tiles of one kv head over all their key tiles).
-        // Uniform (a positive hint): every item in n_splits equal pieces, one CTA each.  Even (the default when it pays,
-        // or a negative hint = that many CTAs): the key tiles of all items, laid end to end, are cut into equal runs, one
-        // per CTA and at most one CTA per SM, so that the launch is one full wave whatever the number of items; a CTA
-        // walks the segments of its run one after the other, and an item that was cut leaves partial results.
-        int even_ctas = 0;
-        const int64_t part_floats = static_cast<int64_t>(kItemRows) * per_rh;    // one partial block
         if (!decode) {
             n_splits = 1;
-            if (direct) {
-                n_splits = 1;
-            } else if (a->split_hint >= 1) {
-                n_splits = std::min(a->split_hint, std::max(1, min_tiles));   // no CTA without a tile
-                n_splits = std::min<int64_t>(n_splits, std::max<int64_t>(1, c->cap_items / base_items));
-                n_splits = std::min(n_splits, kMaxSplits);
-                while (n_splits > 1 && !fits(n_splits)) --n_splits;
-            } else {
-                // at least three key tiles per CTA on average, and no item in more pieces than the merge kernel takes
-                int64_t n = a->split_hint < 0 ? -static_cast<int64_t>(a->split_hint)
-                                              : std::min<int64_t>(c->n_sm, std::max<int64_t>(base_items, all_tiles / 3));
-                n = std::min<int64_t>(n, all_tiles);
-                const int64_t min_run = (max_tiles + kMaxSplits - 3) / (kMaxSplits - 2);
-                n = std::max<int64_t>(1, std::min<int64_t>(n, all_tiles / min_run));
-                const bool cuts = a->split_hint < 0 || n > base_items || base_items > c->n_sm;
-                if (cuts && base_items + n <= c->cap_items) even_ctas = static_cast<int>(n);
-            }
+            if (direct) n_splits = 1;
+            else if (a->split_hint >= 1) n_splits = std::min(a->split_hint, std::max(1, min_tiles));   // no CTA without a tile
+            else if (base_items * 5 < c->n_sm * 4) n_splits = std::max(1, std::min(static_cast<int>(c->n_sm / base_items), min_tiles / 2));
+            n_splits = std::min<int64_t>(n_splits, std::max<int64_t>(1, c->cap_items / base_items));
+            n_splits = std::min(n_splits, kMaxSplits);
+            while (n_splits > 1 && !fits(n_splits)) --n_splits;
         }
 
         if (c->gpu && cudaEventSynchronize(c->plan_copied) != cudaSuccess) { cudaGetLastError(); return ENL_E_CUDA; }
         c->plan_valid = false;
-        {
-            const size_t stride = (sizeof(int32_t) * a->n_q + 255) & ~static_cast<size_t>(255);
-            c->off_rowslots = c->off_rows;
-            c->off_rowitem = c->off_rows + stride;
-            c->off_rowlocal = c->off_rows + 2 * stride;
-            c->off_rowobj = c->off_rows + 3 * stride;
-            c->off_rows_end = c->off_rows + (has_sum ? 4 : 3) * stride;
-        }
         EpInfo *eps = c->h_eps();
         int32_t *stream = c->h_stream();
         int32_t *smeta = c->h_meta();
@@ -720,115 +682,29 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
         } else {
             c->key_obj.clear();
         }
-        // Items in the order of the rows (episode, token block, kv head), then heaviest first (late token blocks see
-        // more new-token tiles).  The decode kernel derives its work from the grid and takes nothing from here.
-        struct Work { int32_t ep, kvh, t0, tiles, index; };
+        // CTAs, heaviest first (late token blocks see more new-token tiles)
+        struct Work { Item it; int tiles; };
         std::vector<Work> work;
-        work.reserve(static_cast<size_t>(base_items));
-        int32_t *rowitem = c->h_rowitem(), *rowlocal = c->h_rowlocal();
+        work.reserve(static_cast<size_t>(base_items) * n_splits);
+        for (int b = 0; b < B && decode; ++b)
+            for (int h = 0; h < d.n_kv_heads; ++h)
+                for (int sp = 0; sp < n_splits; ++sp) work.push_back({Item{b, h, 0, sp}, eps[b].n_ctiles});
         for (int b = 0; b < B && !decode; ++b) {
             const EpInfo &e = eps[b];
             for (int t0 = 0; t0 < e.n_q; t0 += tpc) {
                 const int t_hi = std::min(t0 + tpc, e.n_q);
                 const int tiles = e.n_ctiles + (e.n_new - e.n_q + t_hi - 1) / kTileKeys + 1;
-                for (int t = t0; t < t_hi; ++t) {
-                    rowitem[e.q_off + t] = static_cast<int32_t>(work.size());
-                    rowlocal[e.q_off + t] = t - t0;
-                }
                 for (int h = 0; h < d.n_kv_heads; ++h)
-                    work.push_back({b, h, t0, tiles, static_cast<int32_t>(work.size())});
+                    for (int sp = 0; sp < n_splits; ++sp) work.push_back({Item{b, h, t0, sp}, tiles});
             }
         }
-        const size_t n_base = work.size();
         std::stable_sort(work.begin(), work.end(), [](const Work &x, const Work &y) { return x.tiles > y.tiles; });
-        // segments, the CTAs' first segments, the items' partial blocks
-        std::vector<Item> segs;
-        std::vector<int32_t> cta_first;
-        std::vector<int2> item_part(n_base, make_int2(0, 1));
-        int32_t n_blocks = 0, max_pieces = 1;
-        if (decode) {
-            max_pieces = n_splits;
-        } else if (even_ctas > 0) {
-            // run c covers tiles [cut(c), cut(c + 1)) of the items laid end to end; a cut that would leave a piece of
-            // one tile moves to the item's border
-            std::vector<int64_t> start(n_base + 1, 0);
-            for (size_t k = 0; k < n_base; ++k) start[k + 1] = start[k] + work[k].tiles;
-            const int64_t T = start[n_base];
-            std::vector<int64_t> cut(even_ctas + 1);
-            size_t k = 0;
-            for (int cta = 0; cta <= even_ctas; ++cta) {
-                int64_t pos = T * cta / even_ctas;
-                while (k + 1 < n_base && start[k + 1] <= pos) ++k;
-                if (pos - start[k] == 1) pos = start[k];
-                else if (start[k + 1] - pos == 1) pos = start[k + 1];
-                cut[cta] = cta > 0 ? std::max(pos, cut[cta - 1]) : 0;
-            }
-            cut[even_ctas] = T;
-            k = 0;
-            std::vector<int32_t> pieces(n_base, 0);
-            for (int cta = 0; cta < even_ctas; ++cta) {
-                cta_first.push_back(static_cast<int32_t>(segs.size()));
-                int64_t pos = cut[cta];
-                while (pos < cut[cta + 1]) {
-                    while (start[k + 1] <= pos) ++k;
-                    const int64_t end = std::min(cut[cta + 1], start[k + 1]);
-                    segs.push_back(Item{work[k].ep, work[k].kvh, work[k].t0, static_cast<int32_t>(pos - start[k]),
-                                        static_cast<int32_t>(end - start[k]), pieces[k]++, 0, 0});
-                    pos = end;
-                }
-            }
-            cta_first.push_back(static_cast<int32_t>(segs.size()));
-            for (size_t i = 0; i < n_base; ++i) {
-                if (pieces[i] > 1) { item_part[work[i].index] = make_int2(n_blocks, pieces[i]); n_blocks += pieces[i]; }
-                max_pieces = std::max(max_pieces, pieces[i]);
-            }
-            for (Item &sg : segs) {                       // the item of a segment: same (episode, kv head, token block)
-                const int2 ip = item_part[rowitem[eps[sg.ep].q_off + sg.t0] + sg.kvh];
-                sg.part_base = ip.x;
-                sg.n_pieces = ip.y;
-            }
-            // more pieces than the merge kernel takes, or partial results beyond the scratch buffer: whole items instead
-            if (max_pieces > kMaxSplits || n_blocks * part_floats * 4 + 16 > d.scratch_bytes) {
-                segs.clear();
-                cta_first.clear();
-                std::fill(item_part.begin(), item_part.end(), make_int2(0, 1));
-                n_blocks = 0;
-                max_pieces = 1;
-                even_ctas = 0;
-            }
-        }
-        if (!decode && even_ctas == 0) {
-            const bool in_scratch = n_splits > 1;
-            for (size_t i = 0; i < n_base; ++i) {
-                const Work &w = work[i];
-                for (int sp = 0; sp < n_splits; ++sp) {
-                    cta_first.push_back(static_cast<int32_t>(segs.size()));
-                    segs.push_back(Item{w.ep, w.kvh, w.t0, static_cast<int32_t>(static_cast<int64_t>(w.tiles) * sp / n_splits),
-                                        static_cast<int32_t>(static_cast<int64_t>(w.tiles) * (sp + 1) / n_splits), sp, n_splits,
-                                        in_scratch ? n_blocks : 0});
-                }
-                if (in_scratch) { item_part[w.index] = make_int2(n_blocks, n_splits); n_blocks += n_splits; }
-            }
-            cta_first.push_back(static_cast<int32_t>(segs.size()));
-            max_pieces = n_splits;
-        }
-        // the head of the plan: episodes, segments, first segments, partial blocks
-        {
-            auto align256 = [](size_t x) { return (x + 255) & ~static_cast<size_t>(255); };
-            c->off_ctafirst = align256(c->off_items + sizeof(Item) * segs.size());
-            c->off_itempart = align256(c->off_ctafirst + sizeof(int32_t) * cta_first.size());
-            c->off_head_end = align256(c->off_itempart + sizeof(int2) * n_base);
-            if (c->off_head_end > c->off_stream) return ENL_E_NOMEM;      // cannot happen: the capacities were checked above
-            if (!segs.empty()) std::memcpy(c->h_items(), segs.data(), sizeof(Item) * segs.size());
-            if (!cta_first.empty()) std::memcpy(c->h_ctafirst(), cta_first.data(), sizeof(int32_t) * cta_first.size());
-            if (n_base) std::memcpy(c->h_itempart(), item_part.data(), sizeof(int2) * n_base);
-        }
+        Item *items = c->h_items();
+        for (size_t i = 0; i < work.size(); ++i) items[i] = work[i].it;
 
         c->plan_entries = ne;
-        c->plan_ctas = decode ? 0 : static_cast<int32_t>(cta_first.size()) - 1;
-        c->plan_items = decode ? static_cast<int32_t>(static_cast<int64_t>(B) * d.n_kv_heads * n_splits) : c->plan_ctas;
-        c->plan_blocks = n_blocks;
-        c->plan_splits = max_pieces;
+        c->plan_items = static_cast<int32_t>(work.size());
+        c->plan_splits = n_splits;
         c->plan_batch = B;
         c->plan_max_slots = max_slots;
         c->plan_epoch = c->epoch;
@@ -839,9 +715,7 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
         // Two splits of a head_dim-128 call are launched as clusters of two CTAs, which exchange their partial
         // results through distributed shared memory: no scratch round trip and no merge kernel.  Every CTA must
         // have at least one tile, and the items of a pair must be neighbours (they are: same tile count, stable sort).
-        c->plan_pair = !decode && even_ctas == 0 && n_splits == 2 && d.head_dim == 128 && min_tiles >= 2 &&
-                       (c->pairs_ok || !c->gpu);
-        c->plan_merge = !decode && !c->plan_pair && n_blocks > 0;
+        c->plan_pair = !decode && n_splits == 2 && d.head_dim == 128 && min_tiles >= 2 && (c->pairs_ok || !c->gpu);
         c->key_sel.assign(a->sel_ids, a->sel_ids + a->n_sel);
         c->key_cu = cu_key;
         c->key_len = sel_len;
@@ -853,14 +727,16 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
     if (!c->plan_on_device) {
         // one copy covers episodes, items, stream and row->slots (unused gaps travel too; they are small)
         const size_t ent_bytes = sizeof(int32_t) * c->plan_entries;
-        bool okc = cudaMemcpyAsync(c->plan_dev, c->plan_host, c->off_head_end, cudaMemcpyHostToDevice, st) == cudaSuccess &&
+        bool okc = cudaMemcpyAsync(c->plan_dev, c->plan_host, c->off_stream, cudaMemcpyHostToDevice, st) == cudaSuccess &&
                    (ent_bytes == 0 ||
                     (cudaMemcpyAsync(c->plan_dev + c->off_stream, c->plan_host + c->off_stream, ent_bytes,
                                      cudaMemcpyHostToDevice, st) == cudaSuccess &&
                      cudaMemcpyAsync(c->plan_dev + c->off_meta, c->plan_host + c->off_meta, ent_bytes,
                                      cudaMemcpyHostToDevice, st) == cudaSuccess)) &&
-                   cudaMemcpyAsync(c->plan_dev + c->off_rows, c->plan_host + c->off_rows, c->off_rows_end - c->off_rows,
-                                   cudaMemcpyHostToDevice, st) == cudaSuccess &&
+                   cudaMemcpyAsync(c->plan_dev + c->off_rowslots, c->plan_host + c->off_rowslots,
+                                   sizeof(int32_t) * a->n_q, cudaMemcpyHostToDevice, st) == cudaSuccess &&
+                   (!has_sum || cudaMemcpyAsync(c->plan_dev + c->off_rowobj, c->plan_host + c->off_rowobj,
+                                                sizeof(int32_t) * a->n_q, cudaMemcpyHostToDevice, st) == cudaSuccess) &&
                    cudaEventRecord(c->plan_copied, st) == cudaSuccess;
         if (!okc) { cudaGetLastError(); c->plan_valid = false; return ENL_E_CUDA; }
         c->plan_on_device = true;
@@ -928,7 +804,6 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
     p.tm_kpool = c->tm_k[a->layer];
     p.tm_vpool = c->tm_v[a->layer];
     p.items = reinterpret_cast<const Item *>(c->plan_dev + c->off_items);
-    p.cta_first = reinterpret_cast<const int32_t *>(c->plan_dev + c->off_ctafirst);
     p.eps = reinterpret_cast<const EpInfo *>(c->plan_dev + c->off_eps);
     p.stream_page = reinterpret_cast<const int32_t *>(c->plan_dev + c->off_stream);
     p.stream_meta = reinterpret_cast<const int32_t *>(c->plan_dev + c->off_meta);
@@ -940,39 +815,36 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
     p.Hkv = d.n_kv_heads;
     p.rep = c->rep;
     p.mass_stride = a->mass_stride;
-    p.part_stride = slot_stride;                     // the partial slot buffer is packed
+    p.n_splits = c->plan_splits;
     p.pair_merge = c->plan_pair ? 1 : 0;
     p.scale_log2 = 1.4426950408889634f / sqrtf(static_cast<float>(d.head_dim));
     p.mass_sum = a->group_mass_sum;
     p.row_obj = has_sum ? reinterpret_cast<const int32_t *>(c->plan_dev + c->off_rowobj) : nullptr;
     p.sum_stride = a->sum_stride;
     p.mass_only = mass_only ? 1 : 0;
-    if (c->plan_merge) {
-        const size_t rows = static_cast<size_t>(c->plan_blocks) * kItemRows;
+    const bool scratch_merge = p.n_splits > 1 && !c->plan_pair;
+    if (scratch_merge) {
+        const size_t rows = static_cast<size_t>(p.n_splits) * a->n_q * d.n_q_heads;
         p.part_o = c->scratch;
         p.part_lse = c->scratch + rows * d.head_dim;
         p.part_slot = has_mass ? c->scratch + rows * (d.head_dim + 1) : nullptr;
+        p.mass_stride = slot_stride;                 // the partial slot buffer is packed
     }
-    if (launch_attention(p, d.head_dim, c->plan_ctas, st) != cudaSuccess) { cudaGetLastError(); return ENL_E_CUDA; }
-    if (c->plan_merge) {
-        CombineParams cp = {};
+    if (launch_attention(p, d.head_dim, c->plan_items, st) != cudaSuccess) { cudaGetLastError(); return ENL_E_CUDA; }
+    if (scratch_merge) {
+        CombineParams cp;
         cp.part_o = p.part_o;
         cp.part_lse = p.part_lse;
         cp.part_slot = p.part_slot;
         cp.out = a->out;
         cp.mass = a->group_mass;
         cp.row_slots = reinterpret_cast<const int32_t *>(c->plan_dev + c->off_rowslots);
-        cp.row_item = reinterpret_cast<const int32_t *>(c->plan_dev + c->off_rowitem);
-        cp.row_local = reinterpret_cast<const int32_t *>(c->plan_dev + c->off_rowlocal);
-        cp.item_part = reinterpret_cast<const int2 *>(c->plan_dev + c->off_itempart);
-        cp.rep = c->rep;
-        cp.tile_tokens = kTileRows / c->rep;
         cp.n_q_total = a->n_q;
         cp.Hq = d.n_q_heads;
         cp.D = d.head_dim;
         cp.slot_stride = slot_stride;
         cp.mass_stride = a->mass_stride;
-        cp.n_splits = c->plan_splits;
+        cp.n_splits = p.n_splits;
         if (launch_combine(cp, st) != cudaSuccess) { cudaGetLastError(); return ENL_E_CUDA; }
     }
     return ENL_OK;
@@ -1205,7 +1077,7 @@ extern "C" int enl_plan_inspect(const enl_cache_t *cc, int32_t cap_entries, int3
     if (n_entries) *n_entries = c->plan_entries;
     if (n_splits) *n_splits = c->plan_splits;
     if (n_items) *n_items = c->plan_items;
-    if (merge_kind) *merge_kind = c->plan_decode ? 3 : c->plan_pair ? 2 : c->plan_merge ? 1 : 0;
+    if (merge_kind) *merge_kind = c->plan_decode ? 3 : c->plan_pair ? 2 : c->plan_splits > 1 ? 1 : 0;
     const int32_t *s = c->h_stream(), *m = c->h_meta();
     for (int i = 0; i < c->plan_entries && i < cap_entries; ++i) {
         if (stream_pages) stream_pages[i] = s[i];

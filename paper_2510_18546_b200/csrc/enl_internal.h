@@ -24,18 +24,12 @@ struct EpInfo {
     int32_t pad;
 };
 
-// One segment of work of the attention launch: two Q tiles of one (episode, kv head) over a range of the
-// episode's key tiles.  An "item" is the pair of Q tiles over ALL its key tiles; it is cut into n_pieces segments
-// (1 = whole).  A CTA walks one or more segments one after the other.
-constexpr int kItemRows = kQTiles * kTileRows;   // (row, head) pairs of an item: the unit of the partial-result buffers
+// One CTA of the attention launch.
 struct Item {
     int32_t ep;             // episode
     int32_t kvh;            // kv head
-    int32_t t0;             // first query token (episode-relative) of the two Q tiles
-    int32_t j_beg, j_end;   // key tiles [j_beg, j_end) of the item's stream
-    int32_t piece;          // index of this segment among the item's pieces
-    int32_t n_pieces;       // 1: the segment writes the item's final rows; more: partial results, merged afterwards
-    int32_t part_base;      // first partial block of the item (piece k uses block part_base + k, kItemRows rows each)
+    int32_t t0;             // first query token (episode-relative) of the CTA's two Q tiles
+    int32_t split;          // KV split index in [0, n_splits)
 };
 
 // Kernel parameters (passed by value as a __grid_constant__).
@@ -45,22 +39,21 @@ struct AttnParams {
     CUtensorMap tm_vnew;
     CUtensorMap tm_kpool;   // [pages*Hkv*16][D] box {64, 16}   (one layer)
     CUtensorMap tm_vpool;
-    const Item   *items;          // segments
-    const int32_t *cta_first;     // [CTAs + 1]: CTA c walks segments cta_first[c] .. cta_first[c + 1] - 1
+    const Item   *items;
     const EpInfo *eps;
     const int32_t *stream_page;   // KV stream: page id of every entry
     const int32_t *stream_meta;   // KV stream: slot << 8 | valid tokens
     void   *out;            // bf16 [n_q][Hq][D]
     float  *mass;           // fp32 or null
-    float  *part_o;         // pieces: [block][kItemRows][D] fp32 (normalised by the piece's own sum)
-    float  *part_lse;       // pieces: [block][kItemRows] log2-sum-exp of the piece
-    float  *part_slot;      // pieces: [block][kItemRows][mass_stride] per-slot log2-sum-exp
+    float  *part_o;         // split mode: [split][row][Hq][D] fp32 (normalised by the split's own sum)
+    float  *part_lse;       // split mode: [split][row][Hq] log2-sum-exp of the split
+    float  *part_slot;      // split mode: [split][row][Hq][mass_stride] per-slot log2-sum-exp
     int32_t *status;        // device word: nonzero = a bounded wait expired
     int32_t n_q_total;      // rows over the batch
     int32_t Hq, Hkv, rep;   // rep = Hq / Hkv
-    int32_t mass_stride;    // row stride of mass
-    int32_t part_stride;    // row stride of part_slot
-    int32_t pair_merge;     // 1: two pieces per item, launched as clusters of two CTAs that merge through distributed shared memory
+    int32_t mass_stride;
+    int32_t n_splits;
+    int32_t pair_merge;     // 1: two splits, launched as clusters of two CTAs that merge through distributed shared memory
     float   scale_log2;     // log2(e) / sqrt(D)
     float  *mass_sum;       // fp32 [n_obj][sum_stride] or null: per object the masses summed over its rows and the q heads (added to)
     const int32_t *row_obj; // [n_q_total]: object of every query row, -1 = none (only with mass_sum)
@@ -102,16 +95,10 @@ struct CombineParams {
     void  *out;
     float *mass;
     const int32_t *row_slots;   // [n_q_total]: G_b of the row's episode
-    // Partial results by item (the attention kernel): row -> first item of its token block (kv head 0) and its token
-    // within the block; item -> (first partial block, pieces).  All null: uniform layout [split][row][head] with
-    // n_splits splits for every row (the entry point that allocates nothing).
-    const int32_t *row_item, *row_local;
-    const int2 *item_part;
     int32_t n_q_total, Hq, D;
     int32_t slot_stride;        // row stride of part_slot
     int32_t mass_stride;        // row stride of mass
     int32_t n_splits;
-    int32_t rep, tile_tokens;   // q heads per kv head, query tokens per Q tile
 };
 
 // Programmatic dependent launch: a kernel launched this way may start (set-up only) while the previous kernel
@@ -161,7 +148,7 @@ inline cudaError_t launch_pdl_n(void (*kernel)(KArgs...), dim3 grid, dim3 block,
 #endif
 
 // launchers (defined in the .cu files of the kernels)
-cudaError_t launch_attention(const AttnParams &p, int head_dim, int n_ctas, cudaStream_t st);
+cudaError_t launch_attention(const AttnParams &p, int head_dim, int n_items, cudaStream_t st);
 cudaError_t launch_combine(const CombineParams &p, cudaStream_t st);
 cudaError_t launch_decode(const DecodeParams &p, int head_dim, int batch, cudaStream_t st);
 cudaError_t prepare_decode(int head_dim);

@@ -229,7 +229,7 @@ extern "C" int enl_attend_static(const enl_static_args_t *a, void *cuda_stream)
     else static_partial_kernel<64><<<grid, kThreads, 0, st>>>(p, seg);
     if (cudaGetLastError() != cudaSuccess) return ENL_E_CUDA;
 
-    enl::CombineParams cp = {};
+    enl::CombineParams cp;
     cp.part_o = p.part_o;
     cp.part_lse = p.part_lse;
     cp.part_slot = p.part_slot;

@@ -64,10 +64,8 @@ SMALL = {
 }
 
 
-# split > 0: every item in that many pieces; split < 0: the launch cut evenly over that many CTAs (one CTA walks all
-# segments, one after the other, when it is -1)
 @pytest.mark.parametrize("name", sorted(SMALL))
-@pytest.mark.parametrize("split", [0, 2, 5, -1, -3, -7])
+@pytest.mark.parametrize("split", [0, 2, 5])
 def test_small_shapes(name, split):
     c = SMALL[name]
     wl = synth.make_small(7, 1, c["Hq"], c["Hkv"], c["D"], c["pool"], c["sel"], c["n_q"], c["n_new"], name=name)
