@@ -791,7 +791,10 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
         // Masses: parked log-sums -> shares of the row's total.  ref / extra: per row (held by the row's thread) the
         // log-sum-exp of the whole row and, in a pair, the other split's part of the slot in which the splits meet.
         // Few slots: they were parked in shared memory.  Otherwise (the scoring pass has a thousand slots) the warp takes
-        // its rows one after the other, lanes over the slots (coalesced), eight rows' loads in flight.
+        // 96 slots at a time, lanes over the slots (coalesced), the loads of all its 32 rows in flight together: the
+        // cost is one memory round trip (some 3000 cycles while other CTAs stream their keys) per 96 slots.  Up to
+        // eight slots left over at the end (the new tokens' slot after 64 groups, say) are taken row by lane
+        // instead, each thread converting its own row; their loads are in flight with the first round's.
         // With mass_sum (Sec. 3.3 consumes only averages over an object's tokens and the q heads) the masses of the
         // warp's rows that belong to one object are added up on the way, lane by slot, and leave as one atomic add per
         // object and slot.
@@ -813,44 +816,69 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                 return;
             }
             __syncwarp();                                           // the parked values of all lanes are visible
+            const int n_left = (last - first + 1) & 31;
+            const int n_tail = (!p.mass_sum && n_left <= 8) ? n_left : 0;
+            const int last_wide = last - n_tail;
+            float *tail_slots = p.mass + static_cast<long long>(my_ridx) * p.mass_stride + last_wide + 1;
+            float tv[8];
+#pragma unroll
+            for (int x = 0; x < 8; ++x)
+                tv[x] = (x < n_tail && my_ridx >= 0 && last_wide + 1 + x != skip_slot) ? __ldcg(tail_slots + x) : kNegInf;
+            constexpr int kChunks = 3;                              // 32-slot chunks whose loads are in flight together
 #pragma unroll 1
-            for (int s0 = first + lane; s0 - lane <= last; s0 += 32) {
+            for (int sb = first + lane; sb - lane <= last_wide; sb += 32 * kChunks) {
+              float v[kChunks][32];
+#pragma unroll
+              for (int ck = 0; ck < kChunks; ++ck) {
+                const int s0 = sb + 32 * ck;
+                const bool mine = s0 <= last_wide && s0 != skip_slot;
+#pragma unroll
+                for (int x = 0; x < 32; ++x) {
+                    const int ri = __shfl_sync(kFull, my_ridx, x);
+                    v[ck][x] = (mine && ri >= 0) ? __ldcg(p.mass + static_cast<long long>(ri) * p.mass_stride + s0) : kNegInf;
+                }
+              }
+#pragma unroll
+              for (int ck = 0; ck < kChunks; ++ck) {
+                const int s0 = sb + 32 * ck;
+                if (s0 - lane > last_wide) break;                   // warp-uniform
+                const bool mine = s0 <= last_wide && s0 != skip_slot;
                 float run = 0.f;                                    // this slot's sum over the rows of the current object
                 int run_obj = -1;
-#pragma unroll 1
-                for (int r0 = 0; r0 < 32; r0 += 8) {
-                    float v[8];
-                    float *dst[8];
 #pragma unroll
-                    for (int x = 0; x < 8; ++x) {
-                        const int ri = __shfl_sync(kFull, my_ridx, r0 + x);
-                        dst[x] = (ri >= 0 && s0 <= last && s0 != skip_slot)
-                                     ? p.mass + static_cast<long long>(ri) * p.mass_stride + s0 : nullptr;
-                        v[x] = dst[x] ? __ldcg(dst[x]) : kNegInf;
+                for (int x = 0; x < 32; ++x) {
+                    const int ri = __shfl_sync(kFull, my_ridx, x);
+                    const float ref = __shfl_sync(kFull, ref_mine, x);
+                    const float extra = (shared_slot >= 0) ? __shfl_sync(kFull, extra_mine, x) : kNegInf;   // the same in all lanes
+                    float w = 0.f;
+                    if (mine && ri >= 0) {
+                        w = (ref != kNegInf) ? ex2(v[ck][x] - ref) : 0.f;
+                        if (s0 == shared_slot && ref != kNegInf) w += ex2(extra - ref);
+                        p.mass[static_cast<long long>(ri) * p.mass_stride + s0] = w;
                     }
-#pragma unroll
-                    for (int x = 0; x < 8; ++x) {
-                        const float ref = __shfl_sync(kFull, ref_mine, r0 + x);
-                        const float extra = __shfl_sync(kFull, extra_mine, r0 + x);
-                        const int obj = __shfl_sync(kFull, my_obj, r0 + x);
-                        float w = 0.f;
-                        if (dst[x]) {
-                            w = (ref != kNegInf) ? ex2(v[x] - ref) : 0.f;
-                            if (s0 == shared_slot && ref != kNegInf) w += ex2(extra - ref);
-                            *dst[x] = w;
+                    if (p.mass_sum) {                               // warp-uniform: obj is the same in every lane
+                        const int obj = __shfl_sync(kFull, my_obj, x);
+                        if (obj != run_obj) {
+                            if (run_obj >= 0 && mine)
+                                atomicAdd(p.mass_sum + static_cast<long long>(run_obj) * p.sum_stride + s0, run);
+                            run = 0.f;
+                            run_obj = obj;
                         }
-                        if (p.mass_sum) {                           // warp-uniform: obj is the same in every lane
-                            if (obj != run_obj) {
-                                if (run_obj >= 0 && s0 <= last)
-                                    atomicAdd(p.mass_sum + static_cast<long long>(run_obj) * p.sum_stride + s0, run);
-                                run = 0.f;
-                                run_obj = obj;
-                            }
-                            run += w;
-                        }
+                        run += w;
                     }
                 }
-                if (run_obj >= 0 && s0 <= last) atomicAdd(p.mass_sum + static_cast<long long>(run_obj) * p.sum_stride + s0, run);
+                if (run_obj >= 0 && mine) atomicAdd(p.mass_sum + static_cast<long long>(run_obj) * p.sum_stride + s0, run);
+              }
+            }
+            if (n_tail > 0 && my_ridx >= 0) {
+#pragma unroll
+                for (int x = 0; x < 8; ++x) {
+                    const int sl = last_wide + 1 + x;
+                    if (x >= n_tail || sl == skip_slot) continue;
+                    float w = (ref_mine != kNegInf) ? ex2(tv[x] - ref_mine) : 0.f;
+                    if (sl == shared_slot && ref_mine != kNegInf) w += ex2(extra_mine - ref_mine);
+                    tail_slots[x] = w;
+                }
             }
         };
         // slots this CTA walked (all of them without splits)
