@@ -791,10 +791,11 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
         // Masses: parked log-sums -> shares of the row's total.  ref / extra: per row (held by the row's thread) the
         // log-sum-exp of the whole row and, in a pair, the other split's part of the slot in which the splits meet.
         // Few slots: they were parked in shared memory.  Otherwise (the scoring pass has a thousand slots) the warp takes
-        // 96 slots at a time, lanes over the slots (coalesced), the loads of all its 32 rows in flight together: the
-        // cost is one memory round trip (some 3000 cycles while other CTAs stream their keys) per 96 slots.  Up to
-        // eight slots left over at the end (the new tokens' slot after 64 groups, say) are taken row by lane
-        // instead, each thread converting its own row; their loads are in flight with the first round's.
+        // 32 slots at a time, lanes over the slots (coalesced), the loads of all its 32 rows in flight together: the
+        // cost is one memory round trip (some 3000 cycles while other CTAs stream their keys) per 32 slots; three
+        // such chunks in flight at once measured slower.  Up to eight slots left over at the end (the new tokens'
+        // slot after 64 groups, say) are taken row by lane instead, each thread converting its own row; their loads
+        // are in flight with the first chunk's.
         // With mass_sum (Sec. 3.3 consumes only averages over an object's tokens and the q heads) the masses of the
         // warp's rows that belong to one object are added up on the way, lane by slot, and leave as one atomic add per
         // object and slot.
@@ -824,7 +825,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
 #pragma unroll
             for (int x = 0; x < 8; ++x)
                 tv[x] = (x < n_tail && my_ridx >= 0 && last_wide + 1 + x != skip_slot) ? __ldcg(tail_slots + x) : kNegInf;
-            constexpr int kChunks = 3;                              // 32-slot chunks whose loads are in flight together
+            constexpr int kChunks = 1;                              // 32-slot chunks whose loads are in flight together
 #pragma unroll 1
             for (int sb = first + lane; sb - lane <= last_wide; sb += 32 * kChunks) {
               float v[kChunks][32];
