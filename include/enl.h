@@ -305,6 +305,29 @@ int enl_cluster_assign_sums(const float *mass_sum, int32_t sum_stride, int32_t n
 int enl_select_knapsack(int32_t n, const float *prob, float threshold, const int64_t *mem_bytes,
                         int64_t budget_bytes, int64_t quantum, int32_t *sel_out);
 
+/* ---- optional: rotary position encoding of rows before they are stored ------------------------ */
+
+#define ENL_ROPE_MAX_HEAD_DIM 256
+
+/*
+ * Sec. 3.2 mentions position encoding by citation only: every group keeps the positions it was
+ * computed with, and appended tokens continue them.  The attention and the store take K (and Q)
+ * as given; no call of the path rotates anything.  A caller that holds un-rotated rows can rotate
+ * them here, in place, before enl_group_store / enl_attend: rotary position embedding as published
+ * (Su et al., "RoFormer"), channel pair j of every head turned by the angle pos * base^(-2j/D):
+ *   (x1, x2) -> (x1 cos - x2 sin, x2 cos + x1 sin),
+ * the pair being channels (2j, 2j+1) if interleaved != 0, else (j, j + D/2).  The paper fixes
+ * neither the base nor the pairing; both are the caller's.
+ *   rows      : device bf16 [n][n_heads][head_dim], 4-byte aligned, rotated in place
+ *   positions : device int32 [n], or NULL: row i then has position first_pos + i
+ * Angles are formed in double precision and reduced before sine and cosine are taken in fp32;
+ * results are rounded to bf16.  Enqueued on the stream; allocates nothing.
+ * Errors: ENL_E_INVAL (null rows, n < 0, n_heads < 1, odd head_dim, base <= 0), ENL_E_LIMIT
+ * (head_dim > ENL_ROPE_MAX_HEAD_DIM), ENL_E_CUDA.
+ */
+int enl_rope_rotate(void *rows, int32_t n, int32_t n_heads, int32_t head_dim, const int32_t *positions,
+                    int32_t first_pos, double base, int32_t interleaved, void *cuda_stream);
+
 /* ---- an entry point that allocates nothing ------------------------------------------------ */
 
 #define ENL_STATIC_MAX_SEGMENTS  255                 /* cached segments per call                      */

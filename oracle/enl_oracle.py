@@ -215,6 +215,23 @@ def knapsack_bruteforce(prob: Sequence[float], threshold: float, mem_bytes: Sequ
     return best, arg
 
 
+def rope_rotate(rows: np.ndarray, positions: Sequence[int], base: float, interleaved: bool) -> np.ndarray:
+    """Rotary position embedding as published (Su et al., "RoFormer"; Sec. 3.2 of the paper only cites it): in every
+    head, channel pair j -- (2j, 2j+1) when ``interleaved``, else (j, j + D/2) -- of the row at position pos is turned
+    by the angle pos * base^(-2j/D).  ``rows`` is float64 [n][heads][D]; returns a new array."""
+    x = np.asarray(rows, dtype=np.float64)
+    n, heads, d = x.shape
+    out = np.empty_like(x)
+    for i in range(n):
+        for j in range(d // 2):
+            ang = float(positions[i]) * float(base) ** (-2.0 * j / d)
+            cs, sn = np.cos(ang), np.sin(ang)
+            i1, i2 = (2 * j, 2 * j + 1) if interleaved else (j, j + d // 2)
+            out[i, :, i1] = x[i, :, i1] * cs - x[i, :, i2] * sn
+            out[i, :, i2] = x[i, :, i2] * cs + x[i, :, i1] * sn
+    return out
+
+
 class TierModel:
     """Residency book-keeping of the slow tier (Sec. 3.2 / 3.4): which groups are in device memory, under a
     device budget in pages, with least-recently-selected eviction.  Plain Python; the reference for the hit /

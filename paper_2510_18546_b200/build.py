@@ -7,7 +7,7 @@ import subprocess
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libenl.so")
-SOURCES = ["enl_host.cu", "enl_attn_sm100.cu", "enl_decode_sm100.cu", "enl_aux_kernels.cu", "enl_static_scratch.cu", "enl_cluster.cu", "enl_select.cpp"]
+SOURCES = ["enl_host.cu", "enl_attn_sm100.cu", "enl_decode_sm100.cu", "enl_aux_kernels.cu", "enl_static_scratch.cu", "enl_cluster.cu", "enl_rope.cu", "enl_select.cpp"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-shared"]
 

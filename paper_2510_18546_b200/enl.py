@@ -24,7 +24,7 @@ ENL_STATIC_MAX_SEGMENTS, ENL_STATIC_MAX_KEYS, ENL_STATIC_SCRATCH_BYTES = 255, 65
 
 EXPORTS = ("enl_cache_create", "enl_group_store", "enl_attend", "enl_cache_free", "enl_strerror",
            "enl_group_store_all_layers", "enl_group_len", "enl_cache_status", "enl_cache_selfcheck", "enl_plan_inspect", "enl_attend_static", "enl_cluster_assign",
-           "enl_cluster_assign_sums", "enl_select_knapsack", "enl_tier_enable", "enl_group_evict", "enl_step_prepare", "enl_group_resident")
+           "enl_cluster_assign_sums", "enl_select_knapsack", "enl_rope_rotate", "enl_tier_enable", "enl_group_evict", "enl_step_prepare", "enl_group_resident")
 
 
 class CacheDesc(ctypes.Structure):
@@ -115,6 +115,9 @@ def lib() -> ctypes.CDLL:
         L.enl_select_knapsack.argtypes = [ctypes.c_int32, ctypes.c_void_p, ctypes.c_float, ctypes.c_void_p,
                                           ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p]
         L.enl_select_knapsack.restype = ctypes.c_int
+        L.enl_rope_rotate.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p,
+                                      ctypes.c_int32, ctypes.c_double, ctypes.c_int32, ctypes.c_void_p]
+        L.enl_rope_rotate.restype = ctypes.c_int
         L.enl_tier_enable.argtypes = [ctypes.c_void_p, ctypes.c_int64]
         L.enl_tier_enable.restype = ctypes.c_int
         L.enl_group_evict.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p]
@@ -276,6 +279,16 @@ def enl_select_knapsack(prob: Sequence[float], threshold: float, mem_bytes: Sequ
     if rc < 0:
         raise EnlError(rc, "enl_select_knapsack")
     return out[:rc].copy()
+
+
+def enl_rope_rotate(rows, positions=None, first_pos: int = 0, base: float = 10000.0, interleaved: bool = False,
+                    stream: int = 0) -> None:
+    """Rotates ``rows`` (device bf16 [n][heads][D]) in place; ``positions`` is a device int32 tensor [n] or None."""
+    n, heads, d = (int(x) for x in rows.shape)
+    rc = lib().enl_rope_rotate(_ptr(rows), n, heads, d, _ptr(positions), int(first_pos), float(base),
+                               1 if interleaved else 0, stream or None)
+    if rc != ENL_OK:
+        raise EnlError(rc, "enl_rope_rotate")
 
 
 def enl_tier_enable(cache: int, host_tokens: int) -> None:

@@ -1,6 +1,7 @@
 """The rows next to the hot path: the clustering reduce that consumes the group mass (Sec. 3.3), the retrieval
 knapsack that produces the select list (Sec. 3.4, Eq. 1-2), and the group-append compute step (Sec. 3.2)."""
 import itertools
+import math
 
 import numpy as np
 import pytest
@@ -255,3 +256,71 @@ def test_mass_only_and_sum_argument_errors():
         with pytest.raises(enl.EnlError) as e:      # descending spans
             enl.enl_attend(s.cache, 0, wl.sel_ids(), q, kn, vn, out, mass, group_mass_sum=sums, obj_off=[0, 9, 5])
         assert e.value.code == enl.ENL_E_INVAL
+
+
+# ---- rotary position helper (Sec. 3.2 cites the embedding; base and pairing are the caller's) ----
+
+def test_rope_oracle_pins():
+    """What the mathematics fixes: position 0 is the identity; a pair's norm is kept; the first pair (frequency 1)
+    turns by the position itself, counter-clockwise; pair j turns by pos * base^(-2j/D); rotations add up; and the
+    property the embedding exists for: <R_m q, R_n k> depends on m - n only."""
+    rng = np.random.default_rng(3)
+    d = 16
+    x = rng.standard_normal((5, 2, d))
+    for inter in (False, True):
+        pair = (lambda j: (2 * j, 2 * j + 1)) if inter else (lambda j: (j, j + d // 2))
+        assert np.array_equal(orc.rope_rotate(x, [0] * 5, 10000.0, inter), x)
+        y = orc.rope_rotate(x, [3, 1, 4, 1, 5], 10000.0, inter)
+        for j in range(d // 2):
+            i1, i2 = pair(j)
+            assert np.allclose(y[..., i1] ** 2 + y[..., i2] ** 2, x[..., i1] ** 2 + x[..., i2] ** 2, rtol=1e-12)
+        # unit vector along the first channel of a pair: the angle it ends at
+        e = np.zeros((1, 1, d))
+        for j in (0, 3, d // 2 - 1):
+            i1, i2 = pair(j)
+            e[:] = 0.0
+            e[0, 0, i1] = 1.0
+            r = orc.rope_rotate(e, [7], 100.0, inter)
+            want = (7.0 * 100.0 ** (-2.0 * j / d)) % (2 * math.pi)
+            assert math.isclose(math.atan2(r[0, 0, i2], r[0, 0, i1]) % (2 * math.pi), want, abs_tol=1e-12)
+            assert np.count_nonzero(np.abs(r) > 1e-15) <= 2
+        a = orc.rope_rotate(orc.rope_rotate(x, [2] * 5, 50.0, inter), [9] * 5, 50.0, inter)
+        assert np.allclose(a, orc.rope_rotate(x, [11] * 5, 50.0, inter), atol=1e-12)
+        q, k = rng.standard_normal((1, 1, d)), rng.standard_normal((1, 1, d))
+        dots = [float((orc.rope_rotate(q, [m], 10000.0, inter) * orc.rope_rotate(k, [n], 10000.0, inter)).sum())
+                for m, n in ((5, 2), (13, 10), (3, 0))]
+        assert max(dots) - min(dots) < 1e-12
+    # the two pairings differ (a transposed pairing would not pass both branches above with the same data)
+    assert not np.allclose(orc.rope_rotate(x, [3] * 5, 10000.0, False), orc.rope_rotate(x, [3] * 5, 10000.0, True))
+
+
+def test_rope_argument_errors():
+    enl_build.build_library()
+    L = enl.lib()
+    assert L.enl_rope_rotate(None, 1, 1, 64, None, 0, 10000.0, 0, None) == enl.ENL_E_INVAL
+    assert L.enl_rope_rotate(16, 1, 1, 63, None, 0, 10000.0, 0, None) == enl.ENL_E_INVAL      # odd head_dim
+    assert L.enl_rope_rotate(16, 1, 0, 64, None, 0, 10000.0, 0, None) == enl.ENL_E_INVAL
+    assert L.enl_rope_rotate(16, 1, 1, 64, None, 0, 0.0, 0, None) == enl.ENL_E_INVAL          # base must be positive
+    assert L.enl_rope_rotate(16, 1, 1, 512, None, 0, 10000.0, 0, None) == enl.ENL_E_LIMIT
+    assert L.enl_rope_rotate(16, 0, 1, 64, None, 0, 10000.0, 0, None) == enl.ENL_OK           # nothing to do
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("d,heads,inter", [(128, 8, False), (128, 8, True), (64, 2, False), (32, 3, True)])
+def test_rope_rotate_matches_oracle(d, heads, inter):
+    """Rows rotated by the library against the float64 oracle: contiguous positions from a large offset (the angle
+    must be reduced in double) and a position list; then stored and attended like any other K."""
+    dev = torch.device("cuda:0")
+    g = torch.Generator().manual_seed(5)
+    n = 77
+    x = (torch.randn(n, heads, d, generator=g) * 0.5).to(torch.bfloat16)
+    for positions, first in ((None, 100000), (torch.randint(0, 4096, (n,), generator=g).to(torch.int32), 0)):
+        rows = x.clone().to(dev)
+        pos_host = list(range(first, first + n)) if positions is None else positions.tolist()
+        enl.enl_rope_rotate(rows, None if positions is None else positions.to(dev), first_pos=first, base=10000.0,
+                            interleaved=inter)
+        torch.cuda.synchronize()
+        want = orc.rope_rotate(x.double().numpy(), pos_host, 10000.0, inter)
+        got = rows.float().cpu().numpy().astype(np.float64)
+        # one bf16 rounding of a value of that size, plus fp32 sine / cosine
+        assert np.all(np.abs(got - want) <= np.abs(want) * 2.0 ** -8 + 1e-5), np.abs(got - want).max()
