@@ -305,3 +305,29 @@ def test_padding_left_by_a_longer_version_of_the_group_is_harmless():
         out, mass, _ = s.attend(0, q, kn, vn)
         torch.cuda.synchronize()
         check_close(out, ro, mass, rm, what="stale padding after append")
+
+
+def test_split_that_sees_no_key_after_calls_that_left_other_data_in_the_scratch():
+    """Eight zero-length groups come first, so the first 128-key tile of the stream holds no key at all, and with
+    three splits over five tiles the first split is exactly that tile: its log-sum-exp is -inf and its weight in
+    the merge is 0.  The scratch buffer is never cleared; the calls before (another split count, a one-token decode
+    call) leave -inf and unrelated partial results where this call's partial outputs go."""
+    wl = synth.make_small(71, 1, 8, 2, 128, [[0] * 8 + [300, 40]], [list(range(10))], [64], [64], name="empty_split")
+    with Session(wl, [0]) as s:
+        q, kn, vn = wl.new_qkv(0, s.device)
+        ro, rm, _ = s.oracle(0, 0, q, kn, vn)
+        ro1, rm1, _ = s.oracle(0, 0, q[-1:], kn, vn)
+        for split in (5, 1):
+            out, mass, _ = s.attend(0, q, kn, vn, split_hint=split)
+            torch.cuda.synchronize()
+            check_close(out, ro, mass, rm, what=f"empty first tile, split {split}")
+        out1, mass1, _ = s.attend(0, q[-1:], kn, vn, n_q=[1], n_new=[64])
+        torch.cuda.synchronize()
+        check_close(out1, ro1, mass1, rm1, what="empty first tile, decode")
+        out, mass, _ = s.attend(0, q, kn, vn, split_hint=3)
+        torch.cuda.synchronize()
+        assert enl.enl_cache_status(s.cache) == enl.ENL_OK
+        p = enl.enl_plan_inspect(s.cache)
+        assert p["merge_kind"] == 1 and p["n_splits"] == 3
+        check_close(out, ro, mass, rm, what="empty first tile, split 3")
+        assert mass[:, :, :8].abs().max().item() == 0.0          # zero-length groups: mass exactly 0
