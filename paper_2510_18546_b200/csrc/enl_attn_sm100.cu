@@ -10,8 +10,8 @@
 //   p   = exp2(S * c - m)    one thread per row, fp32; padding and causally hidden columns -> 0
 //   O_i += P_i V             tcgen05.mma, P (bf16) read from TMEM, V from shared memory
 // The row sum of p is split by the slot (selected group, or the new tokens) each 16-key page belongs
-// to; when a slot ends its log2-sum-exp is parked in the mass buffer, and after the last tile the
-// warp turns those into probabilities.  With KV splits every split writes partial results that a
+// to; when a slot ends its log2-sum-exp is parked (in shared memory for calls with few slots, else in
+// the mass buffer), and after the last tile the parked values are turned into probabilities.  With KV splits every split writes partial results that a
 // second kernel merges, or (two splits, head_dim 128) the two CTAs of a cluster merge in place.
 //
 // Roles (12 warps): warps 0-3 are the softmax warpgroup of Q tile 0, warps 4-7 that of Q tile 1: one

@@ -5,7 +5,7 @@
 // episode, one kv head and one range of the episode's key stream (16-token pages of the selected groups
 // in list order, then the new-token keys), the partial attention of the rep q heads that read this kv
 // head -- partial output normalised by the range's own sum, the range's log2-sum-exp and a per-slot
-// log2-sum-exp -- which the split merge kernel turns into the output row and the group masses.
+// log2-sum-exp -- which the split merge at the end of the kernel turns into the output row and the group masses.
 //
 // Every K and V page is read from HBM exactly once.  The CTA's 12 warps take its pages one at a time from a
 // shared counter (a warp that is served faster by the memory system simply takes more pages: with fixed runs
