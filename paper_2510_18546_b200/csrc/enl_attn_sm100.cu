@@ -201,6 +201,17 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *tm,
         "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
         ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
 }
+// Bring a box into the L2 without a destination in the SM: nothing is observed, so these may run before the wait for
+// the previous kernel of the stream (the L2 is the point of coherence: a later write to those lines updates them).
+__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap *tm, int x, int y)
+{
+    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(tm), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tma_prefetch_3d(const CUtensorMap *tm, int x, int y, int z)
+{
+    asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];"
+                 ::"l"(tm), "r"(x), "r"(y), "r"(z) : "memory");
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after()  { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 // D[tmem] (+)= A[smem] * B[smem] and D[tmem] (+)= A[tmem] * B[smem].  The whole warp executes the surrounding code
@@ -388,6 +399,27 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
     // everything above touched only shared memory, TMEM and the gather plan; from here on the caller's tensors,
     // the pool and the scratch are read and written, so the previous kernel of the stream must have finished
     pdl_trigger();
+    // While the previous kernel drains, ask what the first S tile needs into the L2: the Q tiles and the first two
+    // key tiles' K and V (cached pages; new-token tiles only when the stream starts with them).
+    // (Only CTAs of the first wave wait for the previous kernel; for the others this would be loads issued twice.)
+    if (warp == kProducerWarp && n_tiles > 0 && static_cast<int>(blockIdx.x) < p.first_wave) {
+        if (lane < n_qt * C::kHalves)
+            tma_prefetch_3d(&p.tm_q, (lane % C::kHalves) * 64, it.kvh * rep, ep.q_off + it.t0 + (lane / C::kHalves) * tile_tokens);
+        for (int j = j_beg; j < min(j_beg + 2, j_end); ++j) {
+            if (j < ep.n_ctiles) {
+                if (lane < kPagesPerTile) {
+                    const int row = (p.stream_page[ep.stream_off + j * kPagesPerTile + lane] * p.Hkv + it.kvh) * kPageTokens;
+                    for (int hf = 0; hf < C::kHalves; ++hf) {
+                        tma_prefetch_2d(&p.tm_kpool, hf * 64, row);
+                        tma_prefetch_2d(&p.tm_vpool, hf * 64, row);
+                    }
+                }
+            } else if (lane < 2 * C::kHalves) {
+                tma_prefetch_3d(lane < C::kHalves ? &p.tm_knew : &p.tm_vnew, (lane % C::kHalves) * 64, it.kvh,
+                                ep.new_off + (j - ep.n_ctiles) * kTileKeys);
+            }
+        }
+    }
     pdl_wait();
 
     bool ok = true;

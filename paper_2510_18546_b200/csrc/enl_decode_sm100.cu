@@ -283,6 +283,16 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
         }
     }
 
+    // ... and the query rows of this kv head (rep x D bf16, contiguous): whatever the kernel before writes there, the
+    // L2 holds the current data, and the loads after the wait then need not go to HBM before the first S
+    {
+        const uint8_t *qb = reinterpret_cast<const uint8_t *>(p.q) +
+                            (static_cast<long long>(ep.q_off) * p.Hq + it.kvh * rep) * D * 2;
+        const int q_bytes = rep * D * 2;
+        if (static_cast<int>(threadIdx.x) * 128 < q_bytes)
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(qb + threadIdx.x * 128) : "memory");
+    }
+
     // so far only shared memory and the gather plan were touched; the caller's tensors and the pool come next
     pdl_wait();
     const uint64_t pol = policy_evict_first();

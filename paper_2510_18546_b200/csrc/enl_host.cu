@@ -822,6 +822,7 @@ extern "C" int enl_attend(enl_cache_t *c, const enl_attend_args_t *a, void *cuda
     p.row_obj = has_sum ? reinterpret_cast<const int32_t *>(c->plan_dev + c->off_rowobj) : nullptr;
     p.sum_stride = a->sum_stride;
     p.mass_only = mass_only ? 1 : 0;
+    p.first_wave = c->n_sm;
     const bool scratch_merge = p.n_splits > 1 && !c->plan_pair;
     if (scratch_merge) {
         const size_t rows = static_cast<size_t>(p.n_splits) * a->n_q * d.n_q_heads;

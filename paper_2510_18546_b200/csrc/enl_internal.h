@@ -59,6 +59,7 @@ struct AttnParams {
     const int32_t *row_obj; // [n_q_total]: object of every query row, -1 = none (only with mass_sum)
     int32_t sum_stride;
     int32_t mass_only;      // 1: the output rows are not written
+    int32_t first_wave;     // CTAs that start while the previous kernel of the stream may still run (the number of SMs)
 };
 
 // Decode (one query token per episode): pages of the key stream one CTA may cover, and the most splits
