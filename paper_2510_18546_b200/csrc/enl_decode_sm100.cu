@@ -181,8 +181,9 @@ struct DecCfg {
     static constexpr int kCslotOff   = kListOff + kListBytes;          // [kDecodeMaxPages + 1][kMaxRep] x (max, sum)
     static constexpr int kCslotBytes = (kDecodeMaxPages + 1) * kMaxRep * 8;
     static constexpr int kMiscOff    = kCslotOff + kCslotBytes;
-    // wm[warp][rep], wl[warp][rep], counters[2 * kWarps], cm[rep], cl[rep], weights[rep][kMaxSplits], flags[4]
-    static constexpr int kMiscBytes  = (2 * kWarps * kMaxRep + 2 * kWarps + 2 * kMaxRep + kMaxRep * kMaxSplits + 4) * 4;
+    // wm[warp][rep], wl[warp][rep], counters[2 * kWarps], cm[rep], cl[rep], weights[rep][kMaxSplits], flags[4],
+    // slot ranges of the splits [kMaxSplits] x (first, count)
+    static constexpr int kMiscBytes  = (2 * kWarps * kMaxRep + 2 * kWarps + 2 * kMaxRep + kMaxRep * kMaxSplits + 4 + 2 * kMaxSplits) * 4;
     static constexpr int kBarOff     = (kMiscOff + kMiscBytes + 15) & ~15;
     static constexpr int kSmemBytes  = kBarOff + kWarps * kStages * 8 + 1024;   // + alignment slack
 };
@@ -214,6 +215,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
     float *weights = cl + kMaxRep;                                            // [kMaxRep][kMaxSplits]
     volatile int *flags = reinterpret_cast<volatile int *>(weights + kMaxRep * kMaxSplits);   // [0] abort, [1] last
     volatile int *abort_flag = flags;
+    int2 *rng_tab = reinterpret_cast<int2 *>(const_cast<int *>(flags) + 4);   // [split]: first slot and slots of its page range
     const uint32_t bar0 = sbase + C::kBarOff;
     auto bar_full = [&](int s) { return bar0 + 8u * (warp * kStages + s); };
     auto stage_addr = [&](int s) { return sbase + static_cast<uint32_t>((warp * kStages + s) * C::kStageBytes); };
@@ -249,6 +251,20 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
     };
 
     if (threadIdx.x == 0) { flags[0] = 0; flags[1] = 0; ctrs[0] = kWarps; ctrs[1] = 0; }
+    // The slot range of every split of this (episode, kv head), from the plan (the same arithmetic as that split's
+    // CTA uses): whichever CTA merges the splits at the end then needs no memory round trip to learn where each
+    // split's slot sums lie.
+    if (static_cast<int>(threadIdx.x) < p.n_splits && p.n_splits > 1) {
+        const int k = threadIdx.x;
+        const int b0 = static_cast<int>(static_cast<long long>(total) * k / p.n_splits);
+        const int b1 = static_cast<int>(static_cast<long long>(total) * (k + 1) / p.n_splits);
+        int2 r = make_int2(0, 0);
+        if (b1 > b0) {
+            const int s0 = entry_meta(b0) >> 8;
+            r = make_int2(s0, (entry_meta(b1 - 1) >> 8) - s0 + 1);
+        }
+        rng_tab[k] = r;
+    }
     // the CTA's page list (page id, slot << 8 | valid keys): one coalesced load up front, so that no global load
     // sits between a stage becoming free and its refill
     for (int i = threadIdx.x; i < n_cta; i += kThreads) {
@@ -593,18 +609,11 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
         const int k = grp + j * groups;
         pv[j] = (active && k < p.n_splits) ? __ldcg(po4 + k * po_stride4) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
-    // slot range of split k = warp + lane * kWarps, from the plan (the same arithmetic as that split's CTA used)
+    // slot range of split k = warp + lane * kWarps (worked out from the plan at the start of the kernel)
     int2 my_rng = make_int2(0, 0);
     {
         const int k = warp + lane * kWarps;
-        if (k < p.n_splits) {
-            const int b0 = static_cast<int>(static_cast<long long>(total) * k / p.n_splits);
-            const int b1 = static_cast<int>(static_cast<long long>(total) * (k + 1) / p.n_splits);
-            if (b1 > b0) {
-                const int s0 = entry_meta(b0) >> 8;
-                my_rng = make_int2(s0, (entry_meta(b1 - 1) >> 8) - s0 + 1);
-            }
-        }
+        if (k < p.n_splits) my_rng = rng_tab[k];
     }
     // ... and the slot log-sums: the first 32 (head, slot) pairs of the splits warp and warp + kWarps
     float xs[2] = {kNegInf, kNegInf};
