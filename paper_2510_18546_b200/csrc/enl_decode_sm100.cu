@@ -484,11 +484,14 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
     if (*abort_flag) return;
 
     // ---- merge the warps: reference maximum, sum, output, slot log-sums of the CTA ----
-    float *obuf = reinterpret_cast<float *>(smem);                           // [warp][kMaxRep][D]
+    // [warp][kMaxRep][D + 8]: with rows D floats apart the eight rows a warp stores together would share their banks
+    constexpr int kORow = D + 8;
+    static_assert(kWarps * kMaxRep * kORow * 4 <= C::kRingBytes, "the warps' outputs fit the idle ring");
+    float *obuf = reinterpret_cast<float *>(smem);
     if (g < rep) {
 #pragma unroll
         for (int nb = 0; nb < kNB; ++nb)
-            *reinterpret_cast<float2 *>(obuf + (warp * kMaxRep + g) * D + nb * 8 + 2 * tq) = make_float2(o[nb][0], o[nb][1]);
+            *reinterpret_cast<float2 *>(obuf + (warp * kMaxRep + g) * kORow + nb * 8 + 2 * tq) = make_float2(o[nb][0], o[nb][1]);
     }
     if (warp < rep) {                                                        // warp h takes head h: lane w holds warp w's (m, l)
         const int h = warp;
@@ -540,7 +543,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
         float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
         float4 v[kWarps];
 #pragma unroll
-        for (int w = 0; w < kWarps; ++w) v[w] = *reinterpret_cast<const float4 *>(obuf + w * kMaxRep * D + ff * 4);
+        for (int w = 0; w < kWarps; ++w)
+            v[w] = *reinterpret_cast<const float4 *>(obuf + (w * kMaxRep + h) * kORow + (ff % (D / 4)) * 4);
 #pragma unroll
         for (int w = 0; w < kWarps; ++w) {
             const float f = weights[h * kMaxSplits + w];
