@@ -178,8 +178,8 @@ struct DecCfg {
     static constexpr int kEntBytes   = kMaxEnt * (kMaxRep + 1) * 4;
     static constexpr int kListOff    = kEntOff + kEntBytes;            // [kDecodeMaxPages] (page id, slot << 8 | valid keys)
     static constexpr int kListBytes  = kDecodeMaxPages * 8;
-    static constexpr int kCslotOff   = kListOff + kListBytes;          // [kDecodeMaxPages + 1][kMaxRep] x (max, sum)
-    static constexpr int kCslotBytes = (kDecodeMaxPages + 1) * kMaxRep * 8;
+    static constexpr int kCslotOff   = kListOff + kListBytes;          // [kDecodeMaxPages + 1][kMaxRep] slot sums
+    static constexpr int kCslotBytes = (kDecodeMaxPages + 1) * kMaxRep * 4;
     static constexpr int kMiscOff    = kCslotOff + kCslotBytes;
     // wm[warp][rep], wl[warp][rep], counters[2 * kWarps], cm[rep], cl[rep], weights[rep][kMaxSplits], flags[4],
     // slot ranges of the splits [kMaxSplits] x (first, count)
@@ -205,8 +205,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
     float *ent_val = reinterpret_cast<float *>(smem + C::kEntOff);            // [kMaxEnt][kMaxRep]: parked log2 slot sums
     int *ent_slot = reinterpret_cast<int *>(ent_val + kMaxEnt * kMaxRep);     // [kMaxEnt]: their slots
     int2 *pg_list = reinterpret_cast<int2 *>(smem + C::kListOff);             // the CTA's pages in stream order
-    int *cmax = reinterpret_cast<int *>(smem + C::kCslotOff);                 // [slot][kMaxRep]: maximum (ordered-int code)
-    float *cslot = reinterpret_cast<float *>(cmax + (kDecodeMaxPages + 1) * kMaxRep);   // [slot][kMaxRep]: sum, then log2-sum
+    float *cslot = reinterpret_cast<float *>(smem + C::kCslotOff);            // [slot][kMaxRep]: sum of shares, then log2-sum
     float *wm = reinterpret_cast<float *>(smem + C::kMiscOff);                // [warp][kMaxRep]
     float *wl = wm + kWarps * kMaxRep;
     int *ctrs = reinterpret_cast<int *>(wl + kWarps * kMaxRep);               // [0] next page to hand out, [1] parked entries
@@ -478,8 +477,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
         slot_first = pg_list[0].y >> 8;
         n_local = (pg_list[n_cta - 1].y >> 8) - slot_first + 1;
     }
-    constexpr int kCodeNegInf = static_cast<int>(0x80000000u);               // below the code of every finite value
-    for (int idx = threadIdx.x; idx < n_local * kMaxRep; idx += kThreads) { cmax[idx] = kCodeNegInf; cslot[idx] = 0.f; }
+    for (int idx = threadIdx.x; idx < n_local * kMaxRep; idx += kThreads) cslot[idx] = 0.f;
     __syncthreads();                                                         // every stage consumed: the ring is free
     if (*abort_flag) return;
 
@@ -509,28 +507,21 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
             cl[h] = (Lh > 0.f) ? rcp(Lh) : 0.f;
         }
     }
-    // parked sums -> one log2-sum per (slot, head): maximum first (an order-preserving integer code of the float,
-    // so that an integer atomic maximum serves), then the sum of exp2(value - maximum)
-    const int n_ent = ctrs[1];
-    auto code = [](float f) { const int i = __float_as_int(f); return i >= 0 ? i : i ^ 0x7fffffff; };
-    auto decode_code = [](int i) { return __int_as_float(i >= 0 ? i : i ^ 0x7fffffff); };
-    for (int idx = threadIdx.x; idx < n_ent * rep; idx += kThreads) {
-        const int e = idx / rep, h = idx % rep;
-        const float v = ent_val[e * kMaxRep + h];
-        if (v != kNegInf) atomicMax(&cmax[(ent_slot[e] - slot_first) * kMaxRep + h], code(v));
-    }
     __syncthreads();
+    // parked sums -> one log2-sum per (slot, head).  The reference is the log2-sum-exp of the CTA's whole range: no
+    // slot's sum exceeds it, so the shares exp2(value - reference) are at most 1 and add up without a maximum pass
+    // (a share below 2^-126 counts as nothing).
+    const int n_ent = ctrs[1];
     for (int idx = threadIdx.x; idx < n_ent * rep; idx += kThreads) {
         const int e = idx / rep, h = idx % rep;
         const float v = ent_val[e * kMaxRep + h];
-        const int at = (ent_slot[e] - slot_first) * kMaxRep + h;
-        if (v != kNegInf) atomicAdd(&cslot[at], ex2(v - decode_code(cmax[at])));
+        if (v != kNegInf) atomicAdd(&cslot[(ent_slot[e] - slot_first) * kMaxRep + h], ex2(v - cm[h]));
     }
     __syncthreads();
     for (int idx = threadIdx.x; idx < n_local * rep; idx += kThreads) {
         const int at = (idx / rep) * kMaxRep + idx % rep;
         const float sum = cslot[at];
-        cslot[at] = (sum > 0.f) ? decode_code(cmax[at]) + lg2(sum) : kNegInf;
+        cslot[at] = (sum > 0.f) ? cm[idx % rep] + lg2(sum) : kNegInf;
     }
     __syncthreads();
 
