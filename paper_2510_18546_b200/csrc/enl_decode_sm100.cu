@@ -517,13 +517,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
         const float v = ent_val[e * kMaxRep + h];
         if (v != kNegInf) atomicAdd(&cslot[(ent_slot[e] - slot_first) * kMaxRep + h], ex2(v - cm[h]));
     }
-    __syncthreads();
-    for (int idx = threadIdx.x; idx < n_local * rep; idx += kThreads) {
-        const int at = (idx / rep) * kMaxRep + idx % rep;
-        const float sum = cslot[at];
-        cslot[at] = (sum > 0.f) ? cm[idx % rep] + lg2(sum) : kNegInf;
-    }
-    __syncthreads();
+    // (the barrier that ends this pass comes after the output merge below, which does not depend on it)
 
     const bool single = p.n_splits == 1;
     const long long row_h0 = static_cast<long long>(ep.q_off) * p.Hq + it.kvh * rep;          // + h: (row, head) index
@@ -552,27 +546,27 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
             *reinterpret_cast<float4 *>(p.part_o + rh0 * D + ff * 4) = a;
         }
     }
+    if (!single) {
+        if (threadIdx.x < rep) p.part_lse[rh0 + threadIdx.x] = cm[threadIdx.x];
+        if (threadIdx.x == 0)
+            p.part_rng[(it.split * static_cast<int>(gridDim.z) + it.ep) * p.Hkv + it.kvh] = make_int2(slot_first, n_local);
+    }
+    __syncthreads();                                                         // every share has been added
     if (single) {
+        // the CTA saw the whole stream: a slot's share of the range is its mass
         if (p.mass)
             for (int idx = threadIdx.x; idx < rep * (G + 1); idx += kThreads) {
                 const int h = idx / (G + 1), s = idx % (G + 1);
-                const float lse = cm[h];
-                float v = 0.f;
-                if (s >= slot_first && s < slot_first + n_local && lse != kNegInf) {
-                    const float x = cslot[(s - slot_first) * kMaxRep + h];
-                    if (x != kNegInf) v = ex2(x - lse);
-                }
-                p.mass[(row_h0 + h) * p.mass_stride + s] = v;
+                const bool mine = s >= slot_first && s < slot_first + n_local;
+                p.mass[(row_h0 + h) * p.mass_stride + s] = mine ? cslot[(s - slot_first) * kMaxRep + h] : 0.f;
             }
         return;
     }
-    if (threadIdx.x < rep) p.part_lse[rh0 + threadIdx.x] = cm[threadIdx.x];
-    if (threadIdx.x == 0)
-        p.part_rng[(it.split * static_cast<int>(gridDim.z) + it.ep) * p.Hkv + it.kvh] = make_int2(slot_first, n_local);
-    if (p.part_slot)                                                         // only the slots this range touched
+    if (p.part_slot)                                                         // only the slots this range touched, as log2-sums
         for (int idx = threadIdx.x; idx < rep * n_local; idx += kThreads) {
             const int h = idx / n_local, sl = idx % n_local;
-            p.part_slot[(rh0 + h) * p.slot_stride + slot_first + sl] = cslot[sl * kMaxRep + h];
+            const float sum = cslot[sl * kMaxRep + h];
+            p.part_slot[(rh0 + h) * p.slot_stride + slot_first + sl] = (sum > 0.f) ? cm[h] + lg2(sum) : kNegInf;
         }
 
     // ---- the last CTA of this (episode, kv head) merges the splits ----
