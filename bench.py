@@ -38,7 +38,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 NCU_TRAFFIC_BYTES = {
     "planner": 15.43e6 + 0.0,         # attn_kernel<128> incl. the in-kernel split merge, profiles/attn_kernel_planner.md
     "long": 45.18e6 + 1.80e6,         # attn_kernel<128>, one launch, profiles/attn_kernel_planner.md
-    "decode": 140.67e6 + 3.38e6,      # decode_kernel<128>, profiles/decode_kernel_decode.md
+    "decode": 140.67e6 + 4.71e6,      # decode_kernel<128>, profiles/decode_kernel_decode.md
 }
 
 
